@@ -1,0 +1,462 @@
+"""Pins of the CPU oracle against things it does not define itself.
+
+Every reference value here comes from a textbook softmax attention written in this
+file, finite differences of it, closed-form algebra, or brute force on tiny inputs.
+A planted mistake in the oracle (dropped term, wrong sign, transposed operand,
+missing count bias) must fail at least one of these.
+"""
+import itertools
+import math
+
+import numpy as np
+import pytest
+
+from oracle import kvs_oracle as oc
+
+RNG = np.random.default_rng(20240607)
+
+
+# ------------------------------------------------------------------ independent reference
+def ref_attention_output(q, K, V):
+    """Textbook single-query softmax attention, written independently of the oracle."""
+    logits = np.array([float(np.dot(q, K[i])) for i in range(K.shape[0])]) / math.sqrt(K.shape[1])
+    w = np.exp(logits - np.max(logits))
+    w = w / np.sum(w)
+    out = np.zeros(V.shape[1])
+    for i in range(K.shape[0]):
+        out += w[i] * V[i]
+    return out, w
+
+
+def loss_linear(E, q, K, V):
+    out, _ = ref_attention_output(q, K, V)
+    return float(np.dot(E, out))
+
+
+def fd_grad(E, q, K, V, i, h=1e-5):
+    g = np.zeros(K.shape[1])
+    for a in range(K.shape[1]):
+        Kp, Km = K.copy(), K.copy()
+        Kp[i, a] += h
+        Km[i, a] -= h
+        g[a] = (loss_linear(E, q, Kp, V) - loss_linear(E, q, Km, V)) / (2 * h)
+    return g
+
+
+def fd_hessian_block(E, q, K, V, i, j, h=1e-4):
+    d = K.shape[1]
+    H = np.zeros((d, d))
+    for a in range(d):
+        for b in range(d):
+            acc = 0.0
+            for sa, sb in ((1, 1), (1, -1), (-1, 1), (-1, -1)):
+                Kx = K.copy()
+                Kx[i, a] += sa * h
+                Kx[j, b] += sb * h
+                acc += sa * sb * loss_linear(E, q, Kx, V)
+            H[a, b] = acc / (4 * h * h)
+    return H
+
+
+def tiny_problem(n=6, d=3, dv=3, seed=0):
+    r = np.random.default_rng(seed)
+    return (r.standard_normal(dv), r.standard_normal(d), r.standard_normal((n, d)),
+            r.standard_normal((n, dv)))
+
+
+# ------------------------------------------------------------------ bf16 conversion
+def test_bf16_roundtrip_and_rne():
+    allbits = np.arange(0x0080, 0x7F80, dtype=np.uint16)           # all positive normals
+    assert np.array_equal(oc.f64_to_bf16(oc.bf16_to_f64(allbits)), allbits)
+    neg = allbits | np.uint16(0x8000)
+    assert np.array_equal(oc.f64_to_bf16(oc.bf16_to_f64(neg)), neg)
+    # exact ties go to the even mantissa; just above a tie goes up
+    lo = oc.bf16_to_f64(np.array([0x3F80, 0x3F81], dtype=np.uint16))   # 1.0, 1.0078125
+    assert oc.f64_to_bf16(np.array([(lo[0] + lo[1]) / 2]))[0] == 0x3F80
+    hi = oc.bf16_to_f64(np.array([0x3F82], dtype=np.uint16))
+    assert oc.f64_to_bf16(np.array([(lo[1] + hi[0]) / 2]))[0] == 0x3F82
+    assert oc.f64_to_bf16(np.array([(lo[0] + lo[1]) / 2 + 1e-12]))[0] == 0x3F81
+    # carry into the exponent
+    top = oc.bf16_to_f64(np.array([0x3FFF], dtype=np.uint16))[0]      # 1.9921875
+    assert oc.f64_to_bf16(np.array([top + 0.005]))[0] == 0x4000       # -> 2.0
+    # float32 semantics agree on random values
+    x = RNG.standard_normal(10000) * 5
+    f32 = x.astype(np.float32).astype(np.float64)                     # exact in f32 first
+    u = f32.astype(np.float32).view(np.uint32)
+    want = ((u + 0x7FFF + ((u >> 16) & 1)) >> 16).astype(np.uint16)
+    assert np.array_equal(oc.f64_to_bf16(f32), want)
+    assert oc.f64_to_bf16(np.array([0.0, -0.0])).tolist() == [0, 0x8000]
+
+
+# ------------------------------------------------------------------ Section 4.1 pins
+def test_attention_matches_textbook():
+    E, q, K, V = tiny_problem(7, 4, 5, 1)
+    _, alpha, o = oc.attention(q, K, V)
+    o_ref, a_ref = ref_attention_output(q, K, V)
+    assert np.allclose(alpha, a_ref, rtol=0, atol=1e-15)
+    assert np.allclose(o, o_ref, rtol=0, atol=1e-15)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_key_gradient_vs_finite_differences(seed):
+    E, q, K, V = tiny_problem(6, 3, 3, seed)
+    for i in range(K.shape[0]):
+        g = oc.key_gradient(E, q, K, V, i)
+        assert np.allclose(g, fd_grad(E, q, K, V, i), rtol=1e-6, atol=1e-9)
+
+
+@pytest.mark.parametrize("seed", [0, 3])
+def test_hessian_blocks_vs_finite_differences(seed):
+    E, q, K, V = tiny_problem(5, 3, 3, seed)
+    for m in (0, 2, 3):
+        h11, h22, h12 = oc.hessian_blocks(E, q, K, V, m)
+        scale = max(np.abs(h11).max(), np.abs(h22).max(), np.abs(h12).max())
+        assert np.allclose(h11, fd_hessian_block(E, q, K, V, m, m), atol=2e-6 * max(scale, 1))
+        assert np.allclose(h22, fd_hessian_block(E, q, K, V, m + 1, m + 1), atol=2e-6 * max(scale, 1))
+        assert np.allclose(h12, fd_hessian_block(E, q, K, V, m, m + 1), atol=2e-6 * max(scale, 1))
+        # symmetry of the coupling block h^{m+1,m} = h^{m,m+1} (rank one in q q^T)
+        assert np.allclose(h12, fd_hessian_block(E, q, K, V, m + 1, m).T, atol=2e-6 * max(scale, 1))
+
+
+def test_c_vectors_recovered_from_fd_hessian_with_unit_E():
+    """With E = unit vector a, the Hessian scalar is component a of c_ij: the brute-force
+    Hessian therefore pins every component and the sign of c11, c22 and c12."""
+    _, q, K, V = tiny_problem(5, 2, 3, 11)
+    m = 1
+    _, alpha, o = ref_attention_output(q, K, V)[1], None, None
+    out, w = ref_attention_output(q, K, V)
+    c11, c22, c12 = oc.c_vectors(w[m], w[m + 1], V[m], V[m + 1], out)
+    qq = np.outer(q, q) / K.shape[1]
+    for a in range(V.shape[1]):
+        E = np.zeros(V.shape[1])
+        E[a] = 1.0
+        for blk, cvec in (((m, m), c11), ((m + 1, m + 1), c22), ((m, m + 1), c12)):
+            H = fd_hessian_block(E, q, K, V, *blk)
+            coef = float(np.sum(H * qq) / np.sum(qq * qq))
+            assert abs(coef - cvec[a]) < 5e-7, (blk, a, coef, cvec[a])
+
+
+def test_softmax_second_derivative_identity():
+    """d2 alpha_i / dz_i^2 = alpha_i(1-alpha_i)(1-2 alpha_i); the paper's diagonal coefficient
+    alpha(1-2 alpha) is what multiplies (v_i - o) once the d o/dz term is included.  Check the
+    resulting d s_i/d e_j of Section 4.1 by finite differences in logit space."""
+    r = np.random.default_rng(5)
+    z = r.standard_normal(5)
+    V = r.standard_normal((5, 3))
+
+    def s_vec(zz, i):
+        a = np.exp(zz - zz.max())
+        a /= a.sum()
+        return a[i] * (V[i] - a @ V)
+
+    a = np.exp(z - z.max())
+    a /= a.sum()
+    o = a @ V
+    h = 1e-6
+    for i, j in itertools.product(range(3), range(3)):
+        zp, zm = z.copy(), z.copy()
+        zp[j] += h
+        zm[j] -= h
+        fd = (s_vec(zp, i) - s_vec(zm, i)) / (2 * h)
+        if i == j:
+            c, _, _ = oc.c_vectors(a[i], a[i], V[i], V[i], o)
+            assert np.allclose(fd, c, atol=1e-8)
+        else:
+            _, _, c = oc.c_vectors(a[i], a[j], V[i], V[j], o)
+            assert np.allclose(fd, c, atol=1e-8)
+
+
+# ------------------------------------------------------------------ Section 4.2 pins
+@pytest.mark.parametrize("seed", [0, 4, 9])
+def test_linear_system_and_weight_form(seed):
+    E, q, K, V = tiny_problem(6, 4, 3, seed)
+    m = 2
+    h11, h22, h12 = oc.hessian_blocks(E, q, K, V, m)
+    Mmat = h11 + 2 * h12 + h22
+    Nvec = h11 @ K[m] + h12 @ (K[m] + K[m + 1]) + h22 @ K[m + 1]
+    kstar = oc.projected_solution(E, q, K, V, m)
+    assert np.allclose(Mmat @ kstar, Nvec, atol=1e-12)
+    # minimum-norm solution equals numpy's pseudo-inverse solution
+    assert np.allclose(kstar, np.linalg.pinv(Mmat) @ Nvec, atol=1e-9)
+    out, w = ref_attention_output(q, K, V)
+    c11, c22, c12 = oc.c_vectors(w[m], w[m + 1], V[m], V[m + 1], out)
+    wm, wn = oc.exact_weights(E, c11, c22, c12)
+    assert abs(wm + wn - 1.0) < 1e-12
+    kw = wm * K[m] + wn * K[m + 1]
+    # same component along q (the only direction the rank-one system constrains)
+    assert abs(float(q @ kw) - float(q @ kstar)) < 1e-10
+    assert np.allclose(Mmat @ kw, Nvec, atol=1e-12)
+
+
+def test_norm_form_equals_exact_weights_when_cosines_align():
+    """d_v = 1, residuals of one sign, alpha < 1/2: cos(E,c11) = cos(E,c22) = -cos(E,c12)
+    holds exactly, so the gradient-free weight equals the exact one."""
+    r = np.random.default_rng(3)
+    n = 8
+    K = r.standard_normal((n, 4)) * 0.3
+    q = r.standard_normal(4)
+    V = r.uniform(0.0, 0.2, size=(n, 1))
+    m = 3
+    V[m] = 2.0
+    V[m + 1] = 3.0          # both far above o: same-sign residuals
+    out, w = ref_attention_output(q, K, V)
+    assert w[m] < 0.5 and w[m + 1] < 0.5 and V[m] > out and V[m + 1] > out
+    c11, c22, c12 = oc.c_vectors(w[m], w[m + 1], V[m], V[m + 1], out)
+    for E in (np.array([1.0]), np.array([-2.5])):
+        wm, _ = oc.exact_weights(E, c11, c22, c12)
+        wn = oc.norm_form_weight(np.linalg.norm(c11), np.linalg.norm(c22), np.linalg.norm(c12))
+        assert abs(wm - wn) < 1e-12
+
+
+def test_norm_form_weight_closed_form_and_guards():
+    assert oc.norm_form_weight(3.0, 1.0, 0.5) == pytest.approx((3 - 0.5) / (3 - 1 + 1))
+    assert oc.norm_form_weight(1.0, 3.0, 0.5) == pytest.approx((1 - 0.5) / 3)
+    assert oc.norm_form_weight(1.0, 1.0, 1.0) == 0.5            # zero denominator
+    assert oc.norm_form_weight(0.0, 0.0, 0.0) == 0.5
+    assert oc.norm_form_weight(1.0, 5.0, 2.0) == 0.0            # (1-2)/(1-4+5) < 0 -> clip
+    assert oc.norm_form_weight(5.0, 1.0, 2.0) == 1.0            # (5-2)/(2) > 1 -> clip
+    assert oc.norm_form_weight(float("nan"), 1.0, 0.1) == 0.5
+
+
+# ------------------------------------------------------------------ window statistics
+def _rand_bf16(shape, r, scale=1.0):
+    x = (r.standard_normal(shape) * scale).astype(np.float32)
+    u = x.view(np.uint32)
+    return ((u + 0x7FFF + ((u >> 16) & 1)) >> 16).astype(np.uint16)
+
+
+def test_window_stats_against_per_query_definitions():
+    """N1, N12 and A are sums over the window queries of per-query quantities that are
+    themselves pinned above (c-vectors).  Rebuild them query by query with the textbook
+    attention, with the causal mask expressed by truncating the key list."""
+    r = np.random.default_rng(8)
+    n, d, G, W = 20, 6, 2, 3
+    Kb, Vb, Qb = _rand_bf16((n, d), r), _rand_bf16((n, d), r), _rand_bf16((G, W, d), r)
+    c = np.ones(n)
+    Kf, Vf, Qf = oc.bf16_to_f64(Kb), oc.bf16_to_f64(Vb), oc.bf16_to_f64(Qb)
+    scale = 0.37
+    alpha, o, vbar = oc.window_probabilities(Kf, Vf, c, Qf, W, scale, True)
+    A, N1 = oc.slot_stats(alpha, o, vbar)
+    off, P = 2, 6
+    N12, cosv, score = oc.pair_stats(Kf, alpha, o, vbar, A, off, P, 0)
+    A_ref, N1_ref, N12_ref = np.zeros(n), np.zeros(n), np.zeros(P)
+    for g in range(G):
+        for i in range(W):
+            vis = n - W + i + 1                                   # slots 0..n-W+i
+            qeff = Qf[g, i] * scale * math.sqrt(d)                 # textbook divides by sqrt(d)
+            out, w = ref_attention_output(qeff, Kf[:vis], Vf[:vis])
+            assert np.allclose(alpha[g * W + i, :vis], w, atol=1e-15)
+            assert np.all(alpha[g * W + i, vis:] == 0)
+            A_ref[:vis] += w
+            for j in range(vis):
+                c11, _, _ = oc.c_vectors(w[j], w[j], Vf[j], Vf[j], out)
+                N1_ref[j] += np.linalg.norm(c11)
+            for p in range(P):
+                j = off + 2 * p
+                if j + 1 < vis:
+                    _, _, c12 = oc.c_vectors(w[j], w[j + 1], Vf[j], Vf[j + 1], out)
+                    N12_ref[p] += np.linalg.norm(c12)
+    assert np.allclose(A, A_ref, atol=1e-14)
+    assert np.allclose(N1, N1_ref, atol=1e-14)
+    assert np.allclose(N12, N12_ref, atol=1e-14)
+    for p in range(P):
+        j = off + 2 * p
+        cs = float(Kf[j] @ Kf[j + 1]) / math.sqrt(float(Kf[j] @ Kf[j]) * float(Kf[j + 1] @ Kf[j + 1]))
+        assert abs(cosv[p] - cs) < 1e-14
+        assert abs(score[p] - (A_ref[j] + A_ref[j + 1]) * max(0.0, 1 - cs)) < 1e-14
+    _, _, score1 = oc.pair_stats(Kf, alpha, o, vbar, A, off, P, 1)
+    assert np.allclose(score1, A_ref[off:off + 2 * P:2] + A_ref[off + 1:off + 2 * P:2], atol=1e-14)
+
+
+def test_merged_slot_equals_its_expanded_tokens():
+    """A slot with count c, value sum S and key k must behave exactly like c tokens that all
+    have key k and whose values sum to S: same o, same total mass.  Pins ln(c) and S/c."""
+    r = np.random.default_rng(12)
+    n, d, G, W = 9, 4, 1, 2
+    Kf = r.standard_normal((n, d))
+    V = r.standard_normal((n + 2, d))
+    Q = r.standard_normal((G, W, d))
+    # expanded cache: slot 2 is three tokens with the same key
+    K_exp = np.concatenate([Kf[:2], Kf[2:3], Kf[2:3], Kf[2:3], Kf[3:]], axis=0)
+    a_exp, o_exp, _ = oc.window_probabilities(K_exp, V, np.ones(n + 2), Q, W, 0.5, False)
+    Vsum = np.concatenate([V[:2], V[2:5].sum(0, keepdims=True), V[5:]], axis=0)
+    c = np.ones(n)
+    c[2] = 3
+    a_m, o_m, vbar = oc.window_probabilities(Kf, Vsum, c, Q, W, 0.5, False)
+    assert np.allclose(o_m, o_exp, atol=1e-14)
+    assert np.allclose(a_m[:, 2], a_exp[:, 2:5].sum(1), atol=1e-14)
+    assert np.allclose(a_m[:, 3:], a_exp[:, 5:], atol=1e-14)
+    assert np.allclose(vbar[2], V[2:5].mean(0), atol=1e-15)
+
+
+def test_causal_mask_positions():
+    r = np.random.default_rng(2)
+    n, d, G, W = 10, 4, 2, 4
+    alpha, _, _ = oc.window_probabilities(r.standard_normal((n, d)), r.standard_normal((n, d)),
+                                          np.ones(n), r.standard_normal((G, W, d)), W, 1.0, True)
+    for g in range(G):
+        for i in range(W):
+            row = alpha[g * W + i]
+            assert np.all(row[: n - W + i + 1] > 0) and np.all(row[n - W + i + 1:] == 0)
+            assert abs(row.sum() - 1) < 1e-14
+
+
+# ------------------------------------------------------------------ selection / schedule
+def test_select_pairs_brute_force_with_ties():
+    r = np.random.default_rng(4)
+    for trial in range(50):
+        P = int(r.integers(1, 12))
+        score = r.integers(0, 4, size=P).astype(np.float64)        # many ties
+        R = int(r.integers(0, P + 1))
+        want = sorted(range(P), key=lambda p: (score[p], p))[:R]
+        mask = oc.select_pairs(score, R)
+        assert mask.sum() == R and sorted(np.nonzero(mask)[0].tolist()) == sorted(want)
+
+
+def test_round_plan_closed_forms():
+    # the paper's operating regime: budget 2048 + chunk 512, sink 32 -> one round of 512 merges
+    plan = oc.full_plan(2560, 2048, 32, 32, 0.5)
+    assert plan == [(2560, 32, (2560 - 32 - 32) // 2, 512)]
+    # parity alternates, every round removes R, ends exactly on the budget
+    plan = oc.full_plan(4096, 1024, 32, 32, 0.5)
+    n = 4096
+    for r, (nr, off, P, R) in enumerate(plan):
+        assert nr == n and off == 32 + r % 2 and P == (n - off - 32) // 2
+        assert R == min(n - 1024, max(1, P // 2))
+        n -= R
+    assert n == 1024 and len(plan) == 5
+    assert len(oc.full_plan(32768, 2048, 32, 64, 0.5)) == 10
+    assert len(oc.full_plan(131072, 4096, 32, 128, 0.5)) == 13
+    with pytest.raises(ValueError):
+        oc.full_plan(70, 10, 32, 32, 0.5)        # protected regions exceed the budget
+    assert oc.full_plan(100, 100, 32, 32, 0.5) == []
+    assert oc.round_plan(100, 99, 32, 32, 0.01, 0) == (32, 18, 1)     # at least one pair
+
+
+# ------------------------------------------------------------------ merge + compaction
+def test_apply_merge_bookkeeping():
+    r = np.random.default_rng(6)
+    n, d, off, P = 30, 8, 3, 10
+    Kb, Vb = _rand_bf16((n, d), r, 3.0), _rand_bf16((n, d), r, 3.0)
+    c = r.integers(1, 5, size=n)
+    mask = np.zeros(P, dtype=np.uint8)
+    mask[[0, 3, 4, 9]] = 1
+    w = r.uniform(0, 1, size=P)
+    Kn, Vn, cn, idx = oc.apply_merge(Kb, Vb, c, off, mask, w)
+    assert Kn.shape[0] == n - 4 and cn.sum() == c.sum()
+    Kf, Vf = oc.bf16_to_f64(Kb), oc.bf16_to_f64(Vb)
+    # monotone, stable map; right members land on their partner
+    assert np.all(np.diff(idx) >= 0) and idx[0] == 0 and idx[-1] == n - 5
+    for p in range(P):
+        j = off + 2 * p
+        if mask[p]:
+            assert idx[j] == idx[j + 1]
+            want = Kf[j + 1] + w[p] * (Kf[j] - Kf[j + 1])
+            got = oc.bf16_to_f64(Kn[idx[j]])
+            # round to nearest: error at most half a bf16 ulp, and ulp <= |x| 2^-7
+            assert np.all(np.abs(got - want) <= np.abs(want) * 2.0 ** -8)
+            vs = Vf[j] + Vf[j + 1]
+            assert np.all(np.abs(oc.bf16_to_f64(Vn[idx[j]]) - vs) <= np.abs(vs) * 2.0 ** -8)
+            assert cn[idx[j]] == c[j] + c[j + 1]
+        else:
+            assert idx[j + 1] == idx[j] + 1
+            assert np.array_equal(Kn[idx[j]], Kb[j]) and np.array_equal(Kn[idx[j + 1]], Kb[j + 1])
+            assert np.array_equal(Vn[idx[j]], Vb[j]) and cn[idx[j + 1]] == c[j + 1]
+    # untouched prefix and suffix are bit-identical and keep their order
+    assert np.array_equal(Kn[:off], Kb[:off]) and np.array_equal(Vn[-(n - off - 2 * P):], Vb[off + 2 * P:])
+    # total value mass is conserved up to the bf16 rounding of the merged rows
+    assert np.allclose(oc.bf16_to_f64(Vn).sum(0), Vf.sum(0), atol=4 * 2.0 ** -7 * 12)
+
+
+def test_merge_unit_invariants_and_identical_keys():
+    r = np.random.default_rng(7)
+    n, d, G, W, sink, budget = 120, 8, 2, 4, 5, 40
+    Kb, Vb, Qb = _rand_bf16((n, d), r), _rand_bf16((n, d), r), _rand_bf16((G, W, d), r)
+    # plant identical neighbours: they have cosine 1 -> score 0 -> merged first, K unchanged
+    for j in (sink + 2, sink + 10, sink + 20):
+        Kb[j + 1] = Kb[j]
+    trace = []
+    Kn, Vn, cn = oc.merge_unit(Kb, Vb, np.ones(n, dtype=np.int64), Qb, budget, window=W, sink=sink,
+                               trace=trace)
+    assert Kn.shape[0] == budget and Vn.shape[0] == budget and cn.sum() == n
+    assert np.array_equal(Kn[:sink], Kb[:sink]) and np.array_equal(Vn[:sink], Vb[:sink])
+    assert np.array_equal(Kn[-W:], Kb[-W:]) and np.array_equal(cn[-W:], np.ones(W))
+    st = trace[0]
+    for j in (sink + 2, sink + 10, sink + 20):
+        p = (j - st["off"]) // 2
+        assert st["score"][p] <= 1e-12 and st["mask"][p] == 1
+    for t in trace:
+        assert t["mask"].sum() == t["R"]
+        assert np.all((t["w"] >= 0) & (t["w"] <= 1))
+    # one round by hand: merging identical keys returns that key, bit for bit
+    K1, V1, c1 = oc.merge_unit(Kb, Vb, np.ones(n, dtype=np.int64), Qb, budget, window=W, sink=sink,
+                               max_rounds=1)
+    assert np.array_equal(K1[sink + 2], Kb[sink + 2]) and c1[sink + 2] == 2
+
+
+def test_value_sum_merge_is_lossless_for_identical_keys():
+    """Decode over a cache in which identical-key neighbours were merged (value sum, count 2)
+    equals textbook attention over the unmerged cache."""
+    r = np.random.default_rng(9)
+    n, d = 16, 8
+    Kb, Vb = _rand_bf16((n, d), r), _rand_bf16((n, d), r)
+    Kb[5] = Kb[4]
+    Kb[11] = Kb[10]
+    qb = _rand_bf16((2, 3, d), r)
+    Kf, Vf, qf = oc.bf16_to_f64(Kb), oc.bf16_to_f64(Vb), oc.bf16_to_f64(qb)
+    keep = np.ones(n, dtype=bool)
+    keep[[5, 11]] = False
+    Vsum = Vf.copy()
+    Vsum[4] += Vf[5]
+    Vsum[10] += Vf[11]
+    c = np.ones(n, dtype=np.int64)
+    c[[4, 10]] = 2
+    # value sums of two bf16 numbers need not be bf16; keep them exact by using float input bits
+    Vsum_bits = oc.f64_to_bf16(Vsum[keep])
+    exact = np.array_equal(oc.bf16_to_f64(Vsum_bits), Vsum[keep])
+    out, lse = oc.decode_attention(qb, Kb[keep], Vsum_bits, c[keep])
+    for g in range(2):
+        for t in range(3):
+            ref, w = ref_attention_output(qf[g, t], Kf, Vf)
+            tol = 1e-13 if exact else 2e-2
+            assert np.allclose(out[g, t], ref, atol=tol)
+            e = Kf @ qf[g, t] / math.sqrt(d)
+            assert abs(lse[g, t] - (np.log(np.sum(np.exp(e - e.max()))) + e.max())) < 1e-12
+
+
+def test_decode_counts_one_is_textbook_attention():
+    r = np.random.default_rng(10)
+    n, d = 33, 16
+    Kb, Vb, qb = _rand_bf16((n, d), r), _rand_bf16((n, d), r), _rand_bf16((3, 2, d), r)
+    out, _ = oc.decode_attention(qb, Kb, Vb, np.ones(n, dtype=np.int64))
+    for g in range(3):
+        for t in range(2):
+            ref, _ = ref_attention_output(oc.bf16_to_f64(qb)[g, t], oc.bf16_to_f64(Kb), oc.bf16_to_f64(Vb))
+            assert np.allclose(out[g, t], ref, atol=1e-13)
+
+
+def test_forced_mask_is_followed():
+    r = np.random.default_rng(13)
+    n, d, G, W, sink, budget = 60, 8, 1, 4, 4, 50
+    Kb, Vb, Qb = _rand_bf16((n, d), r), _rand_bf16((n, d), r), _rand_bf16((G, W, d), r)
+    off, P, R = oc.round_plan(n, budget, sink, W, 0.5, 0)
+    forced = np.zeros(P, dtype=np.uint8)
+    forced[:R] = 1
+    Kn, Vn, cn = oc.merge_unit(Kb, Vb, np.ones(n, dtype=np.int64), Qb, budget, window=W, sink=sink,
+                               forced_masks=[forced])
+    assert np.array_equal(cn[sink:sink + R], np.full(R, 2))
+
+
+def test_n1_is_a_norm_when_attention_is_peaked():
+    """alpha > 1/2 makes (1 - 2 alpha) negative; N1 sums NORMS of c_jj, so it uses |1 - 2 alpha|."""
+    r = np.random.default_rng(14)
+    n, d = 5, 4
+    Kf = r.standard_normal((n, d)) * 0.1
+    Q = r.standard_normal((1, 1, d))
+    Kf[1] = 6.0 * Q[0, 0] / np.linalg.norm(Q[0, 0])          # one dominant key
+    V = r.standard_normal((n, d))
+    alpha, o, vbar = oc.window_probabilities(Kf, V, np.ones(n), Q, 1, 1.0, False)
+    assert alpha[0, 1] > 0.5
+    _, N1 = oc.slot_stats(alpha, o, vbar)
+    c11, _, _ = oc.c_vectors(alpha[0, 1], alpha[0, 1], V[1], V[1], o[0])
+    assert N1[1] > 0 and abs(N1[1] - np.linalg.norm(c11)) < 1e-14
