@@ -1,0 +1,188 @@
+/*
+ * kvs.h - C ABI of the B200 (sm_100a) KV-merge library, libkvs.so.
+ *
+ * The library implements the KV-merge pass of KVSlimmer: for every (sequence, KV head)
+ * it computes observation-window attention, reduces the forward-only statistics that the
+ * closed-form exact Hessian of an adjacent key pair needs, scores and selects adjacent
+ * pairs, merges keys with the closed-form weights and values by summation, and compacts
+ * the cache in place to the token budget.  A split-K attention over the merged cache
+ * closes the loop.
+ *
+ * General conventions
+ *   - Every pointer marked DEVICE is device memory owned by the caller; HOST pointers are
+ *     ordinary host memory.  The library allocates no device memory, never synchronises
+ *     the stream and never throws.
+ *   - All compute calls are asynchronous on `cuda_stream` (a cudaStream_t passed as
+ *     void*; NULL is the legacy default stream).
+ *   - Errors the host can detect return a code before anything is enqueued and leave all
+ *     buffers untouched.  Errors only the device can detect (a bounded wait that ran out)
+ *     set *status_dev to a kvs_status_t value; the pass then finishes without touching
+ *     further cache memory.  status_dev may be NULL.
+ *   - bf16 tensors are passed as void* to 16-bit words; layouts are row major with the
+ *     head dimension (128) innermost and contiguous.
+ *   - A cache "slot" is a triple (key, value SUM, count).  A fresh token has count 1 and
+ *     its value as the sum.  A merged slot stands for `count` original tokens: it enters
+ *     attention with the logit bias ln(count) and the mean value sum/count.
+ */
+#ifndef KVS_H_
+#define KVS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  KVS_OK = 0,
+  KVS_ERR_INVALID_ARG = 1,        /* NULL pointer, non-positive size, bad stride ...        */
+  KVS_ERR_UNSUPPORTED = 2,        /* head_dim != 128, group*window > 1024, ...              */
+  KVS_ERR_WORKSPACE = 3,          /* workspace smaller than kvs_workspace_size() asks       */
+  KVS_ERR_BUDGET_UNREACHABLE = 4, /* a round has no candidate pair left above the budget    */
+  KVS_ERR_CUDA = 5,               /* a CUDA runtime call failed; see kvs_last_error_string  */
+  KVS_ERR_TIMEOUT = 6             /* device side: a bounded wait ran out                    */
+} kvs_status_t;
+
+typedef struct {
+  int32_t batch;         /* B sequences                                                      */
+  int32_t n_q_heads;     /* Hq; must be a multiple of n_kv_heads                             */
+  int32_t n_kv_heads;    /* Hkv                                                              */
+  int32_t head_dim;      /* must be 128                                                      */
+  int32_t window;        /* W: the observation queries are the last W positions              */
+  int32_t sink;          /* leading slots that are never merged (the paper keeps 32)         */
+  int32_t recent;        /* trailing slots never merged; >= window when causal               */
+  int32_t causal;        /* 1: window query i attends to slots <= n - W + i                  */
+  float   softmax_scale; /* multiplies <q,k> inside the logit (1/sqrt(128))                  */
+  float   round_frac;    /* fraction of the candidate pairs merged per round, in (0,1]       */
+  int32_t score_mode;    /* 0: attention mass * (1 - cosine)   1: attention mass only        */
+  int32_t first_round;   /* index of the first round executed (sets the pair parity)         */
+  int64_t k_stride_b, k_stride_h, k_stride_t; /* K element strides: sequence, head, slot     */
+  int64_t v_stride_b, v_stride_h, v_stride_t; /* V element strides; k/v_stride_t >= 128      */
+} kvs_params_t;
+
+/* Library version (major*100 + minor). */
+int kvs_version(void);
+
+/* Text of the most recent error on the calling thread ("" if none). */
+const char* kvs_last_error_string(void);
+
+/* Number of kernels this library has launched since it was loaded (host counter). */
+uint64_t kvs_launch_count(void);
+
+/*
+ * Round schedule of one sequence (host only, no CUDA call).
+ * Operation: the chunk schedule of Section 3.1 ("merge chunk_size adjacent pairs in one
+ * step"), repeated until the budget is met.  Round r of a cache with n slots uses the
+ * aligned candidate pairs (off+2p, off+2p+1), off = sink + (r mod 2),
+ * P = floor((n - off - recent)/2), and merges R = min(n - budget, max(1, floor(round_frac*P))).
+ *   n, budget      current slot count and target
+ *   max_rounds     capacity of the output arrays (HOST, may be NULL to count only)
+ *   n_r/off_r/P_r/R_r  HOST int32[max_rounds] out
+ *   n_rounds       HOST out: rounds needed
+ * Returns KVS_ERR_BUDGET_UNREACHABLE if a round has P == 0, KVS_ERR_WORKSPACE if
+ * max_rounds is too small (n_rounds is still set).
+ */
+kvs_status_t kvs_round_plan(const kvs_params_t* params, int32_t n, int32_t budget,
+                            int32_t max_rounds, int32_t* n_r, int32_t* off_r, int32_t* P_r,
+                            int32_t* R_r, int32_t* n_rounds);
+
+/*
+ * Bytes of DEVICE workspace that kvs_merge_layer / kvs_compact / kvs_window_stats need for
+ * caches of up to max_seq_len slots, and kvs_decode_attn for up to max_new query tokens
+ * (pass 0 if decode is not used).  Host only.
+ */
+kvs_status_t kvs_workspace_size(const kvs_params_t* params, int32_t max_seq_len,
+                                int32_t max_new, size_t* bytes);
+
+/*
+ * The whole merge pass of one decoder layer, in place  [Section 4: Eqs. attn_def_vec,
+ * c11_def-c12_def, kstar_final; Section 3.1: v* = v_m + v_{m+1} and the chunk schedule].
+ *   K, V       DEVICE bf16 [B,Hkv,Nmax,128] (strides in params); V holds value SUMS
+ *   counts     DEVICE int32 [B,Hkv,Nmax] contiguous; 1 for fresh tokens
+ *   q_win      DEVICE bf16 [B,Hq,W,128] contiguous: queries of the last W positions
+ *   seq_len    HOST int32[B]: slots in use per sequence (<= n_max)
+ *   budget     HOST int32[B]: target slot count per sequence
+ *   n_max      Nmax, the slot capacity that the counts layout uses
+ *   new_len    HOST int32[B] out: min(seq_len, budget); written before the call returns
+ *   workspace  DEVICE, >= kvs_workspace_size(params, max seq_len, 0); 256-byte aligned
+ * A sequence with seq_len <= budget is left untouched.  Slots at index >= new_len[b] are
+ * unspecified afterwards.  Rounds run back to back on the stream with no host sync.
+ */
+kvs_status_t kvs_merge_layer(const kvs_params_t* params, void* K, void* V, int32_t* counts,
+                             const void* q_win, const int32_t* seq_len, const int32_t* budget,
+                             int32_t n_max, int32_t* new_len, void* workspace,
+                             size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
+
+/*
+ * One round of merge + stable in-place compaction with a caller-supplied decision
+ * [Eq. kstar_final for the key, v* = v_m + v_{m+1} for the value sum].
+ *   merge_mask DEVICE uint8 [B,Hkv,Nmax/2]: 1 where candidate pair p is merged; pair p of
+ *              sequence b covers slots (off+2p, off+2p+1), off = sink + (first_round mod 2)
+ *   w_left     DEVICE fp32 [B,Hkv,Nmax/2]: weight of the left key of pair p:
+ *              K* = bf16(K_right + w (K_left - K_right))
+ *   seq_len    HOST int32[B]; new_len HOST int32[B] out = seq_len - (pairs merged) is NOT
+ *              computed here: the caller passes n_merge HOST int32[B], the number of ones in
+ *              each sequence's mask (per head, equal for all heads), and gets
+ *              new_len = seq_len - n_merge
+ *   new_index  optional DEVICE int32 [B,Hkv,Nmax] out: old slot -> new slot (the right
+ *              member of a merged pair maps to its partner's new slot)
+ * Compaction indices and counts are exact integer work: the same mask gives the same
+ * result bit for bit.
+ */
+kvs_status_t kvs_compact(const kvs_params_t* params, void* K, void* V, int32_t* counts,
+                         const uint8_t* merge_mask, const float* w_left,
+                         const int32_t* seq_len, const int32_t* n_merge, int32_t n_max,
+                         int32_t* new_len, int32_t* new_index, void* workspace,
+                         size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
+
+/*
+ * Attention of new queries over a (merged) cache, split along the slots and combined
+ * [Eq. attn_def_vec with merged slots: numerator uses value sums, denominator weights
+ * each slot by its count]:
+ *   out_q = sum_j exp(s_qj) Vsum_j / sum_j c_j exp(s_qj),  s_qj = softmax_scale <q, K_j>.
+ * No causal mask.
+ *   q_new      DEVICE bf16 [B,Hq,n_new,128] contiguous
+ *   out        DEVICE bf16 [B,Hq,n_new,128] contiguous
+ *   lse        optional DEVICE fp32 [B,Hq,n_new]: ln sum_j c_j exp(s_qj)
+ *   seq_len    HOST int32[B]: slots in use
+ * (n_q_heads / n_kv_heads) * n_new must be <= 1024.
+ */
+kvs_status_t kvs_decode_attn(const kvs_params_t* params, const void* q_new, int32_t n_new,
+                             const void* K, const void* V, const int32_t* counts,
+                             const int32_t* seq_len, int32_t n_max, void* out, float* lse,
+                             void* workspace, size_t workspace_bytes, int32_t* status_dev,
+                             void* cuda_stream);
+
+/*
+ * Diagnostic export: the statistics and the decision of ONE round (params->first_round)
+ * without modifying the cache  [Eqs. attn_def_vec, c11_def-c12_def, kstar_final].
+ *   A, N1      optional DEVICE fp32 [B,Hkv,Nmax]: attention mass and summed |c_jj| per slot
+ *              (defined for candidate slots off <= j < off+2P; others are not written)
+ *   N12, cosv, score, w   optional DEVICE fp32 [B,Hkv,Nmax/2] per candidate pair
+ *   mask       optional DEVICE uint8 [B,Hkv,Nmax/2]: the R pairs with smallest (score, p)
+ *   o_win      optional DEVICE fp32 [B,Hkv,G*W,128]: attention output of the window queries
+ *   lse_win    optional DEVICE fp32 [B,Hkv,G*W]: ln sum_j c_j exp(s_qj) of the window queries
+ */
+kvs_status_t kvs_window_stats(const kvs_params_t* params, const void* K, const void* V,
+                              const int32_t* counts, const void* q_win, const int32_t* seq_len,
+                              const int32_t* budget, int32_t n_max, float* A, float* N1,
+                              float* N12, float* cosv, float* score, float* w, uint8_t* mask,
+                              float* o_win, float* lse_win, void* workspace,
+                              size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
+
+/*
+ * Per-kernel device timing for benchmarks.  Between kvs_profile_begin() and
+ * kvs_profile_end() every kernel launch of this library is bracketed by CUDA events on the
+ * launching stream.  kvs_profile_end() synchronises those events and returns, for each
+ * kernel kind k < n_kinds, the summed device time in milliseconds and the launch count.
+ * kvs_profile_kind_name(k) names kind k (NULL past the last).  Not thread safe.
+ */
+kvs_status_t kvs_profile_begin(void);
+kvs_status_t kvs_profile_end(int32_t n_kinds, float* ms, int32_t* launches);
+const char* kvs_profile_kind_name(int32_t kind);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVS_H_ */

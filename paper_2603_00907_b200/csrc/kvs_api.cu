@@ -1,0 +1,568 @@
+// C ABI of libkvs.so: argument checks, the host round scheduler, the workspace layout and
+// the launch sequence of each entry point.  No device memory is allocated here and the
+// stream is never synchronised.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <atomic>
+#include <vector>
+
+#include "kvs_internal.h"
+
+namespace {
+
+thread_local char g_err[256] = "";
+std::atomic<uint64_t> g_launches{0};
+
+kvs_status_t fail(kvs_status_t code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+// ------------------------------------------------------------------------------- profiling
+struct ProfRec { int kind; cudaEvent_t a, b; };
+struct Profiler {
+  bool on = false;
+  std::vector<ProfRec> recs;
+  std::vector<cudaEvent_t> pool;
+  size_t used = 0;
+  cudaEvent_t get() {
+    if (used == pool.size()) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+      pool.push_back(e);
+    }
+    return pool[used++];
+  }
+} g_prof;
+
+template <class F>
+cudaError_t launch(int kind, cudaStream_t st, F&& f) {
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (!g_prof.on) return f();
+  cudaEvent_t a = g_prof.get(), b = g_prof.get();
+  if (!a || !b) return f();
+  cudaEventRecord(a, st);
+  cudaError_t e = f();
+  cudaEventRecord(b, st);
+  g_prof.recs.push_back({kind, a, b});
+  return e;
+}
+
+const char* kKindNames[KVS_K_COUNT] = {"attn_partials", "combine", "hessian_stats",
+                                       "select", "merge_compact", "misc"};
+
+// ------------------------------------------------------------------------------- validation
+kvs_status_t check_params(const kvs_params_t* p) {
+  if (!p) return fail(KVS_ERR_INVALID_ARG, "params is NULL");
+  if (p->batch <= 0 || p->n_q_heads <= 0 || p->n_kv_heads <= 0)
+    return fail(KVS_ERR_INVALID_ARG, "batch and head counts must be positive");
+  if (p->head_dim != KVS_D) return fail(KVS_ERR_UNSUPPORTED, "head_dim must be 128");
+  if (p->n_q_heads % p->n_kv_heads) return fail(KVS_ERR_INVALID_ARG, "n_q_heads %% n_kv_heads != 0");
+  if (p->window <= 0) return fail(KVS_ERR_INVALID_ARG, "window must be positive");
+  if (p->sink < 0 || p->recent < 0) return fail(KVS_ERR_INVALID_ARG, "sink/recent must be >= 0");
+  if (p->causal && p->recent < p->window)
+    return fail(KVS_ERR_INVALID_ARG, "causal window needs recent >= window");
+  if (!(p->round_frac > 0.f && p->round_frac <= 1.f))
+    return fail(KVS_ERR_INVALID_ARG, "round_frac must be in (0,1]");
+  if (!(p->softmax_scale > 0.f) || !isfinite(p->softmax_scale))
+    return fail(KVS_ERR_INVALID_ARG, "softmax_scale must be positive and finite");
+  if (p->score_mode != 0 && p->score_mode != 1) return fail(KVS_ERR_INVALID_ARG, "score_mode must be 0 or 1");
+  if (p->first_round < 0) return fail(KVS_ERR_INVALID_ARG, "first_round must be >= 0");
+  const int G = p->n_q_heads / p->n_kv_heads;
+  if ((int64_t)G * p->window > KVS_MAX_M)
+    return fail(KVS_ERR_UNSUPPORTED, "group * window must be <= %d", KVS_MAX_M);
+  return KVS_OK;
+}
+
+kvs_status_t check_strides(const kvs_params_t* p) {
+  const int64_t s[6] = {p->k_stride_b, p->k_stride_h, p->k_stride_t,
+                        p->v_stride_b, p->v_stride_h, p->v_stride_t};
+  for (int i = 0; i < 6; ++i)
+    if (s[i] < 0 || (s[i] % 8)) return fail(KVS_ERR_INVALID_ARG, "strides must be non-negative multiples of 8 elements");
+  if (p->k_stride_t < KVS_D || p->v_stride_t < KVS_D)
+    return fail(KVS_ERR_INVALID_ARG, "slot stride must be >= 128");
+  return KVS_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ------------------------------------------------------------------------------- schedule
+void round_plan(const kvs_params_t* p, int n, int budget, int r, int* off, int* P, int* R) {
+  *off = p->sink + (r & 1);
+  int cand = (n - *off - p->recent) / 2;
+  if (n - *off - p->recent < 0) cand = 0;
+  *P = cand > 0 ? cand : 0;
+  if (*P == 0) { *R = 0; return; }
+  // floor(round_frac * P) evaluated in double from the float parameter
+  int want = (int)floor((double)p->round_frac * (double)*P);
+  if (want < 1) want = 1;
+  const int excess = n - budget;
+  *R = excess < want ? excess : want;
+}
+
+// ------------------------------------------------------------------------------- workspace
+size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct WsLayout {
+  size_t part_ml, part_o, qstat, o, score, w, mask, tile_prefix, sync, total;
+  int splits_max, M_max, pair_stride, tile_stride, U;
+  size_t sync_bytes;
+};
+
+int splits_bound(int M, int Hkv) {
+  const int nqblk = (M + 127) / 128;
+  int s = (2 * 148 + nqblk * Hkv - 1) / (nqblk * Hkv);
+  if (s < 1) s = 1;
+  if (s > KVS_MAX_SPLITS) s = KVS_MAX_SPLITS;
+  return s;
+}
+
+WsLayout make_layout(const kvs_params_t* p, int n_max, int max_new) {
+  WsLayout L;
+  const int G = p->n_q_heads / p->n_kv_heads;
+  const int Mw = G * p->window, Md = G * max_new;
+  L.M_max = Mw > Md ? Mw : Md;
+  const int sw = splits_bound(Mw, p->n_kv_heads), sd = max_new > 0 ? splits_bound(Md, p->n_kv_heads) : 0;
+  const size_t rows_w = (size_t)sw * Mw, rows_d = (size_t)sd * Md;
+  const size_t part_rows = rows_w > rows_d ? rows_w : rows_d;
+  L.splits_max = sw > sd ? sw : sd;
+  L.U = p->batch * p->n_kv_heads;
+  L.pair_stride = n_max / 2 + 1;
+  L.tile_stride = n_max / KVS_CTILE + 2;
+  size_t o = 0;
+  L.part_ml = o; o += align_up((size_t)L.U * part_rows * sizeof(float2));
+  L.part_o = o;  o += align_up((size_t)L.U * part_rows * KVS_D * sizeof(float));
+  L.qstat = o;   o += align_up((size_t)L.U * L.M_max * sizeof(float4));
+  L.o = o;       o += align_up((size_t)L.U * L.M_max * KVS_D * sizeof(float));
+  L.score = o;   o += align_up((size_t)L.U * L.pair_stride * sizeof(float));
+  L.w = o;       o += align_up((size_t)L.U * L.pair_stride * sizeof(float));
+  L.mask = o;    o += align_up((size_t)L.U * L.pair_stride);
+  L.tile_prefix = o; o += align_up((size_t)L.U * L.tile_stride * sizeof(int32_t));
+  // tickets [KVS_MAX_ROUNDS][U] followed by flags [U][tile_stride]; zeroed once per call
+  L.sync = o;
+  L.sync_bytes = align_up(((size_t)KVS_MAX_ROUNDS * L.U + (size_t)L.U * L.tile_stride) * sizeof(uint32_t));
+  o += L.sync_bytes;
+  L.total = o;
+  return L;
+}
+
+CacheView make_view(const kvs_params_t* p, void* K, void* V, int32_t* counts, int n_max) {
+  CacheView c;
+  c.K = static_cast<__nv_bfloat16*>(K);
+  c.V = static_cast<__nv_bfloat16*>(V);
+  c.counts = counts;
+  c.ksb = p->k_stride_b; c.ksh = p->k_stride_h; c.kst = p->k_stride_t;
+  c.vsb = p->v_stride_b; c.vsh = p->v_stride_h; c.vst = p->v_stride_t;
+  c.n_max = n_max;
+  c.Hkv = p->n_kv_heads;
+  return c;
+}
+
+int choose_splits(int M, int Hkv, int nseq, int nmax_slots, int* split_len) {
+  const int nqblk = (M + 127) / 128;
+  int s = (2 * 148 + nqblk * Hkv * nseq - 1) / (nqblk * Hkv * nseq);
+  const int cap = (nmax_slots + 255) / 256;
+  if (s > cap) s = cap;
+  const int bound = splits_bound(M, Hkv);
+  if (s > bound) s = bound;
+  if (s < 1) s = 1;
+  int len = (nmax_slots + s - 1) / s;
+  len = (len + 15) / 16 * 16;
+  *split_len = len;
+  return s;
+}
+
+#define CUDA_TRY(expr)                                                                   \
+  do {                                                                                   \
+    cudaError_t e_ = (expr);                                                             \
+    if (e_ != cudaSuccess) return fail(KVS_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); \
+  } while (0)
+
+struct Common {
+  const kvs_params_t* p;
+  WsLayout L;
+  char* ws;
+  cudaStream_t st;
+  int G, Mw;
+};
+
+// The statistics of one round for the sequences in `tab` (window attention partials,
+// combine, Hessian statistics), and optionally the selection.
+kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const void* q_win,
+                                 const RoundTable& tab, int nmax_slots, bool do_select,
+                                 float* A, float* N1, float* N12, float* cosv, float* score_out,
+                                 float* w_out, uint8_t* mask_out, float* o_out, float* lse_out) {
+  const kvs_params_t* p = c.p;
+  FlashArgs fa;
+  fa.c = view;
+  fa.q = static_cast<const __nv_bfloat16*>(q_win);
+  fa.Hq = p->n_q_heads; fa.G = c.G; fa.Wq = p->window; fa.M = c.Mw;
+  fa.causal = p->causal;
+  fa.scale_log2 = p->softmax_scale * 1.4426950408889634f;
+  fa.splits = choose_splits(c.Mw, p->n_kv_heads, tab.nseq, nmax_slots, &fa.split_len);
+  fa.part_ml = reinterpret_cast<float2*>(c.ws + c.L.part_ml);
+  fa.part_o = reinterpret_cast<float*>(c.ws + c.L.part_o);
+  CUDA_TRY(launch(KVS_K_FLASH, c.st, [&] { return kvs_launch_flash_simt(fa, tab, c.st); }));
+
+  CombineArgs ca;
+  ca.M = c.Mw; ca.splits = fa.splits; ca.Hkv = p->n_kv_heads;
+  ca.part_ml = fa.part_ml; ca.part_o = fa.part_o;
+  ca.qstat = reinterpret_cast<float4*>(c.ws + c.L.qstat);
+  ca.o = reinterpret_cast<float*>(c.ws + c.L.o);
+  ca.out_bf16 = nullptr; ca.lse_out = lse_out; ca.o_out = o_out;
+  CUDA_TRY(launch(KVS_K_COMBINE, c.st, [&] { return kvs_launch_combine(ca, tab, c.st); }));
+
+  StatsArgs sa;
+  sa.c = view;
+  sa.q = fa.q; sa.Hq = fa.Hq; sa.G = fa.G; sa.Wq = fa.Wq; sa.M = fa.M;
+  sa.causal = fa.causal; sa.scale_log2 = fa.scale_log2; sa.score_mode = p->score_mode;
+  sa.qstat = ca.qstat; sa.o = ca.o;
+  sa.pair_stride = c.L.pair_stride;
+  sa.score = score_out ? score_out : reinterpret_cast<float*>(c.ws + c.L.score);
+  sa.w = w_out ? w_out : reinterpret_cast<float*>(c.ws + c.L.w);
+  sa.A = A; sa.N1 = N1; sa.N12 = N12; sa.cosv = cosv;
+  CUDA_TRY(launch(KVS_K_STATS, c.st, [&] { return kvs_launch_stats_simt(sa, tab, c.st); }));
+
+  if (do_select) {
+    SelectArgs se;
+    se.Hkv = p->n_kv_heads;
+    se.pair_stride = c.L.pair_stride; se.tile_stride = c.L.tile_stride;
+    se.score = sa.score;
+    se.mask = mask_out ? mask_out : reinterpret_cast<uint8_t*>(c.ws + c.L.mask);
+    se.tile_prefix = reinterpret_cast<int32_t*>(c.ws + c.L.tile_prefix);
+    se.from_mask = 0;
+    CUDA_TRY(launch(KVS_K_SELECT, c.st, [&] { return kvs_launch_select(se, tab, c.st); }));
+  }
+  return KVS_OK;
+}
+
+kvs_status_t check_common(const kvs_params_t* p, const void* K, const void* V, const int32_t* counts,
+                          const int32_t* seq_len, int n_max, void* ws, size_t ws_bytes, int max_new,
+                          Common* c, void* stream) {
+  kvs_status_t s = check_params(p);
+  if (s != KVS_OK) return s;
+  s = check_strides(p);
+  if (s != KVS_OK) return s;
+  if (!K || !V || !counts || !seq_len || !ws) return fail(KVS_ERR_INVALID_ARG, "NULL pointer argument");
+  if (!aligned16(K) || !aligned16(V)) return fail(KVS_ERR_INVALID_ARG, "K and V must be 16-byte aligned");
+  if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return fail(KVS_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+  if (n_max <= 0) return fail(KVS_ERR_INVALID_ARG, "n_max must be positive");
+  for (int b = 0; b < p->batch; ++b) {
+    if (seq_len[b] < 0 || seq_len[b] > n_max) return fail(KVS_ERR_INVALID_ARG, "seq_len[%d] out of range", b);
+  }
+  c->p = p;
+  c->L = make_layout(p, n_max, max_new);
+  if (ws_bytes < c->L.total) return fail(KVS_ERR_WORKSPACE, "workspace too small: %zu < %zu", ws_bytes, c->L.total);
+  c->ws = static_cast<char*>(ws);
+  c->st = static_cast<cudaStream_t>(stream);
+  c->G = p->n_q_heads / p->n_kv_heads;
+  c->Mw = c->G * p->window;
+  return KVS_OK;
+}
+
+}  // namespace
+
+// =================================================================================== C ABI
+extern "C" {
+
+int kvs_version(void) { return 100; }
+
+const char* kvs_last_error_string(void) { return g_err; }
+
+uint64_t kvs_launch_count(void) { return g_launches.load(); }
+
+kvs_status_t kvs_round_plan(const kvs_params_t* p, int32_t n, int32_t budget, int32_t max_rounds,
+                            int32_t* n_r, int32_t* off_r, int32_t* P_r, int32_t* R_r,
+                            int32_t* n_rounds) {
+  kvs_status_t s = check_params(p);
+  if (s != KVS_OK) return s;
+  if (!n_rounds) return fail(KVS_ERR_INVALID_ARG, "n_rounds is NULL");
+  if (n < 0 || budget < 1) return fail(KVS_ERR_INVALID_ARG, "n must be >= 0 and budget >= 1");
+  int r = p->first_round, cnt = 0;
+  while (n > budget) {
+    int off, P, R;
+    round_plan(p, n, budget, r, &off, &P, &R);
+    if (P == 0) { *n_rounds = cnt; return fail(KVS_ERR_BUDGET_UNREACHABLE, "round %d has no candidate pair (n=%d)", r, n); }
+    if (cnt < max_rounds) {
+      if (n_r) n_r[cnt] = n;
+      if (off_r) off_r[cnt] = off;
+      if (P_r) P_r[cnt] = P;
+      if (R_r) R_r[cnt] = R;
+    }
+    n -= R; ++r; ++cnt;
+  }
+  *n_rounds = cnt;
+  if ((n_r || off_r || P_r || R_r) && cnt > max_rounds) return fail(KVS_ERR_WORKSPACE, "plan needs %d rounds", cnt);
+  return KVS_OK;
+}
+
+kvs_status_t kvs_workspace_size(const kvs_params_t* p, int32_t max_seq_len, int32_t max_new,
+                                size_t* bytes) {
+  kvs_status_t s = check_params(p);
+  if (s != KVS_OK) return s;
+  if (!bytes || max_seq_len <= 0 || max_new < 0) return fail(KVS_ERR_INVALID_ARG, "bad size argument");
+  const int G = p->n_q_heads / p->n_kv_heads;
+  if ((int64_t)G * max_new > KVS_MAX_M) return fail(KVS_ERR_UNSUPPORTED, "group * max_new must be <= %d", KVS_MAX_M);
+  *bytes = make_layout(p, max_seq_len, max_new).total;
+  return KVS_OK;
+}
+
+kvs_status_t kvs_merge_layer(const kvs_params_t* p, void* K, void* V, int32_t* counts,
+                             const void* q_win, const int32_t* seq_len, const int32_t* budget,
+                             int32_t n_max, int32_t* new_len, void* workspace,
+                             size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+  Common c;
+  kvs_status_t s = check_common(p, K, V, counts, seq_len, n_max, workspace, workspace_bytes, 0, &c, cuda_stream);
+  if (s != KVS_OK) return s;
+  if (!q_win || !budget || !new_len) return fail(KVS_ERR_INVALID_ARG, "NULL pointer argument");
+  if (!aligned16(q_win)) return fail(KVS_ERR_INVALID_ARG, "q_win must be 16-byte aligned");
+  const int B = p->batch;
+  // plan every sequence first: nothing is enqueued if any sequence cannot reach its budget
+  std::vector<std::vector<SeqRound>> plan(B);
+  int rounds = 0;
+  for (int b = 0; b < B; ++b) {
+    if (budget[b] < 1) return fail(KVS_ERR_INVALID_ARG, "budget[%d] must be >= 1", b);
+    int n = seq_len[b], r = p->first_round;
+    if (n > budget[b] && n < p->window) return fail(KVS_ERR_INVALID_ARG, "seq_len[%d] < window", b);
+    while (n > budget[b]) {
+      int off, P, R;
+      round_plan(p, n, budget[b], r, &off, &P, &R);
+      if (P == 0) return fail(KVS_ERR_BUDGET_UNREACHABLE, "sequence %d: no candidate pair left at n=%d", b, n);
+      plan[b].push_back({n, P, R, b});
+      n -= R; ++r;
+    }
+    if ((int)plan[b].size() > rounds) rounds = (int)plan[b].size();
+  }
+  if (rounds > KVS_MAX_ROUNDS) return fail(KVS_ERR_UNSUPPORTED, "more than %d rounds", KVS_MAX_ROUNDS);
+  for (int b = 0; b < B; ++b) new_len[b] = seq_len[b] < budget[b] ? seq_len[b] : budget[b];
+  if (rounds == 0) return KVS_OK;
+
+  CUDA_TRY(cudaMemsetAsync(c.ws + c.L.sync, 0, c.L.sync_bytes, c.st));
+  uint32_t* tickets = reinterpret_cast<uint32_t*>(c.ws + c.L.sync);
+  uint32_t* flags = tickets + (size_t)KVS_MAX_ROUNDS * c.L.U;
+  const CacheView view = make_view(p, K, V, counts, n_max);
+
+  for (int i = 0; i < rounds; ++i) {
+    const int r = p->first_round + i;
+    // active sequences of this round, in chunks of KVS_SEQ_CHUNK
+    int b = 0;
+    while (b < B) {
+      RoundTable tab;
+      tab.nseq = 0;
+      tab.off = p->sink + (r & 1);
+      int nmax_slots = 0;
+      for (; b < B && tab.nseq < KVS_SEQ_CHUNK; ++b) {
+        if ((int)plan[b].size() > i) {
+          tab.s[tab.nseq++] = plan[b][i];
+          if (plan[b][i].n > nmax_slots) nmax_slots = plan[b][i].n;
+        }
+      }
+      if (tab.nseq == 0) continue;
+      s = enqueue_round_stats(c, view, q_win, tab, nmax_slots, true, nullptr, nullptr, nullptr,
+                              nullptr, nullptr, nullptr, nullptr, nullptr, nullptr);
+      if (s != KVS_OK) return s;
+      CompactArgs ka;
+      ka.c = view;
+      ka.pair_stride = c.L.pair_stride; ka.tile_stride = c.L.tile_stride;
+      ka.mask = reinterpret_cast<const uint8_t*>(c.ws + c.L.mask);
+      ka.w = reinterpret_cast<const float*>(c.ws + c.L.w);
+      ka.tile_prefix = reinterpret_cast<const int32_t*>(c.ws + c.L.tile_prefix);
+      ka.tickets = tickets + (size_t)i * c.L.U;
+      ka.flags = flags;
+      ka.epoch = (uint32_t)(i + 1);
+      ka.new_index = nullptr;
+      ka.status_dev = status_dev;
+      CUDA_TRY(launch(KVS_K_COMPACT, c.st, [&] { return kvs_launch_compact(ka, tab, c.st); }));
+    }
+  }
+  return KVS_OK;
+}
+
+kvs_status_t kvs_compact(const kvs_params_t* p, void* K, void* V, int32_t* counts,
+                         const uint8_t* merge_mask, const float* w_left, const int32_t* seq_len,
+                         const int32_t* n_merge, int32_t n_max, int32_t* new_len,
+                         int32_t* new_index, void* workspace, size_t workspace_bytes,
+                         int32_t* status_dev, void* cuda_stream) {
+  Common c;
+  kvs_status_t s = check_common(p, K, V, counts, seq_len, n_max, workspace, workspace_bytes, 0, &c, cuda_stream);
+  if (s != KVS_OK) return s;
+  if (!merge_mask || !w_left || !n_merge || !new_len) return fail(KVS_ERR_INVALID_ARG, "NULL pointer argument");
+  const int B = p->batch;
+  const int off = p->sink + (p->first_round & 1);
+  std::vector<SeqRound> act;
+  for (int b = 0; b < B; ++b) {
+    const int n = seq_len[b];
+    int P = (n - off - p->recent) / 2;
+    if (n - off - p->recent < 0 || P < 0) P = 0;
+    if (n_merge[b] < 0 || n_merge[b] > P) return fail(KVS_ERR_INVALID_ARG, "n_merge[%d] exceeds the candidate pairs", b);
+    if (n_merge[b] > 0) act.push_back({n, P, n_merge[b], b});
+  }
+  for (int b = 0; b < B; ++b) new_len[b] = seq_len[b] - n_merge[b];
+  if (act.empty() && !new_index) return KVS_OK;
+  if (new_index)   // sequences without a merge still need the identity map
+    for (int b = 0; b < B; ++b)
+      if (n_merge[b] == 0 && seq_len[b] > 0) {
+        int P = (seq_len[b] - off - p->recent) / 2;
+        if (P < 0) P = 0;
+        act.push_back({seq_len[b], P, 0, b});
+      }
+  CUDA_TRY(cudaMemsetAsync(c.ws + c.L.sync, 0, c.L.sync_bytes, c.st));
+  uint32_t* tickets = reinterpret_cast<uint32_t*>(c.ws + c.L.sync);
+  uint32_t* flags = tickets + (size_t)KVS_MAX_ROUNDS * c.L.U;
+  const CacheView view = make_view(p, K, V, counts, n_max);
+  // the caller's mask is laid out [B,Hkv,n_max/2]; the kernels use pair_stride rows, so the
+  // mask and weights are consumed in place with the caller's stride
+  const int caller_stride = n_max / 2;
+  int chunk_id = 0;
+  for (size_t k = 0; k < act.size(); k += KVS_SEQ_CHUNK, ++chunk_id) {
+    RoundTable tab;
+    tab.nseq = 0;
+    tab.off = off;
+    for (size_t u = k; u < act.size() && tab.nseq < KVS_SEQ_CHUNK; ++u) tab.s[tab.nseq++] = act[u];
+    SelectArgs se;
+    se.Hkv = p->n_kv_heads;
+    se.pair_stride = caller_stride; se.tile_stride = c.L.tile_stride;
+    se.score = nullptr;
+    se.mask = const_cast<uint8_t*>(merge_mask);
+    se.tile_prefix = reinterpret_cast<int32_t*>(c.ws + c.L.tile_prefix);
+    se.from_mask = 1;
+    CUDA_TRY(launch(KVS_K_MISC, c.st, [&] { return kvs_launch_select(se, tab, c.st); }));
+    CompactArgs ka;
+    ka.c = view;
+    ka.pair_stride = caller_stride; ka.tile_stride = c.L.tile_stride;
+    ka.mask = merge_mask; ka.w = w_left;
+    ka.tile_prefix = se.tile_prefix;
+    ka.tickets = tickets;   // distinct sequences per chunk: one ticket row serves all chunks
+    ka.flags = flags;
+    ka.epoch = 1;
+    ka.new_index = new_index;
+    ka.status_dev = status_dev;
+    CUDA_TRY(launch(KVS_K_COMPACT, c.st, [&] { return kvs_launch_compact(ka, tab, c.st); }));
+  }
+  return KVS_OK;
+}
+
+kvs_status_t kvs_decode_attn(const kvs_params_t* p, const void* q_new, int32_t n_new, const void* K,
+                             const void* V, const int32_t* counts, const int32_t* seq_len,
+                             int32_t n_max, void* out, float* lse, void* workspace,
+                             size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+  (void)status_dev;
+  if (n_new <= 0) return fail(KVS_ERR_INVALID_ARG, "n_new must be positive");
+  if (p && p->n_kv_heads > 0 && (int64_t)(p->n_q_heads / p->n_kv_heads) * n_new > KVS_MAX_M)
+    return fail(KVS_ERR_UNSUPPORTED, "group * n_new must be <= %d", KVS_MAX_M);
+  Common c;
+  kvs_status_t s = check_common(p, K, V, counts, seq_len, n_max, workspace, workspace_bytes, n_new, &c, cuda_stream);
+  if (s != KVS_OK) return s;
+  if (!q_new || !out) return fail(KVS_ERR_INVALID_ARG, "NULL pointer argument");
+  if (!aligned16(q_new) || !aligned16(out)) return fail(KVS_ERR_INVALID_ARG, "q_new/out must be 16-byte aligned");
+  const int B = p->batch;
+  const int M = c.G * n_new;
+  const CacheView view = make_view(p, const_cast<void*>(K), const_cast<void*>(V), const_cast<int32_t*>(counts), n_max);
+  for (int b0 = 0; b0 < B; b0 += KVS_SEQ_CHUNK) {
+    RoundTable tab;
+    tab.nseq = 0; tab.off = 0;
+    int nmax_slots = 0;
+    for (int b = b0; b < B && b < b0 + KVS_SEQ_CHUNK; ++b) {
+      if (seq_len[b] <= 0) continue;
+      tab.s[tab.nseq++] = {seq_len[b], 0, 0, b};
+      if (seq_len[b] > nmax_slots) nmax_slots = seq_len[b];
+    }
+    if (tab.nseq == 0) continue;
+    FlashArgs fa;
+    fa.c = view;
+    fa.q = static_cast<const __nv_bfloat16*>(q_new);
+    fa.Hq = p->n_q_heads; fa.G = c.G; fa.Wq = n_new; fa.M = M;
+    fa.causal = 0;
+    fa.scale_log2 = p->softmax_scale * 1.4426950408889634f;
+    fa.splits = choose_splits(M, p->n_kv_heads, tab.nseq, nmax_slots, &fa.split_len);
+    fa.part_ml = reinterpret_cast<float2*>(c.ws + c.L.part_ml);
+    fa.part_o = reinterpret_cast<float*>(c.ws + c.L.part_o);
+    CUDA_TRY(launch(KVS_K_FLASH, c.st, [&] { return kvs_launch_flash_simt(fa, tab, c.st); }));
+    CombineArgs ca;
+    ca.M = M; ca.splits = fa.splits; ca.Hkv = p->n_kv_heads;
+    ca.part_ml = fa.part_ml; ca.part_o = fa.part_o;
+    ca.qstat = nullptr; ca.o = nullptr;
+    ca.out_bf16 = static_cast<__nv_bfloat16*>(out);
+    ca.lse_out = lse; ca.o_out = nullptr;
+    CUDA_TRY(launch(KVS_K_COMBINE, c.st, [&] { return kvs_launch_combine(ca, tab, c.st); }));
+  }
+  return KVS_OK;
+}
+
+kvs_status_t kvs_window_stats(const kvs_params_t* p, const void* K, const void* V,
+                              const int32_t* counts, const void* q_win, const int32_t* seq_len,
+                              const int32_t* budget, int32_t n_max, float* A, float* N1, float* N12,
+                              float* cosv, float* score, float* w, uint8_t* mask, float* o_win,
+                              float* lse_win, void* workspace, size_t workspace_bytes,
+                              int32_t* status_dev, void* cuda_stream) {
+  (void)status_dev;
+  Common c;
+  kvs_status_t s = check_common(p, K, V, counts, seq_len, n_max, workspace, workspace_bytes, 0, &c, cuda_stream);
+  if (s != KVS_OK) return s;
+  if (!q_win || !budget) return fail(KVS_ERR_INVALID_ARG, "NULL pointer argument");
+  const int B = p->batch;
+  const int r = p->first_round;
+  std::vector<SeqRound> act;
+  for (int b = 0; b < B; ++b) {
+    if (seq_len[b] <= budget[b]) continue;
+    if (seq_len[b] < p->window) return fail(KVS_ERR_INVALID_ARG, "seq_len[%d] < window", b);
+    int off, P, R;
+    round_plan(p, seq_len[b], budget[b], r, &off, &P, &R);
+    if (P == 0) return fail(KVS_ERR_BUDGET_UNREACHABLE, "sequence %d: no candidate pair at n=%d", b, seq_len[b]);
+    act.push_back({seq_len[b], P, R, b});
+  }
+  // outputs use the caller's row lengths: per-slot n_max, per-pair n_max/2.  The internal
+  // pair arrays use pair_stride, so diagnostics are written with the caller's stride by
+  // running the kernels on a layout whose pair_stride is n_max/2.
+  Common cc = c;
+  cc.L.pair_stride = n_max / 2;
+  const CacheView view = make_view(p, const_cast<void*>(K), const_cast<void*>(V), const_cast<int32_t*>(counts), n_max);
+  for (size_t k = 0; k < act.size(); k += KVS_SEQ_CHUNK) {
+    RoundTable tab;
+    tab.nseq = 0;
+    tab.off = p->sink + (r & 1);
+    int nmax_slots = 0;
+    for (size_t u = k; u < act.size() && tab.nseq < KVS_SEQ_CHUNK; ++u) {
+      tab.s[tab.nseq++] = act[u];
+      if (act[u].n > nmax_slots) nmax_slots = act[u].n;
+    }
+    s = enqueue_round_stats(cc, view, q_win, tab, nmax_slots, mask != nullptr, A, N1, N12, cosv,
+                            score, w, mask, o_win, lse_win);
+    if (s != KVS_OK) return s;
+  }
+  return KVS_OK;
+}
+
+kvs_status_t kvs_profile_begin(void) {
+  g_prof.on = true;
+  g_prof.recs.clear();
+  g_prof.used = 0;
+  return KVS_OK;
+}
+
+kvs_status_t kvs_profile_end(int32_t n_kinds, float* ms, int32_t* launches) {
+  g_prof.on = false;
+  if (n_kinds < 0 || (n_kinds > 0 && (!ms || !launches))) return fail(KVS_ERR_INVALID_ARG, "bad profile buffers");
+  for (int k = 0; k < n_kinds; ++k) { ms[k] = 0.f; launches[k] = 0; }
+  for (const ProfRec& r : g_prof.recs) {
+    CUDA_TRY(cudaEventSynchronize(r.b));
+    float t = 0.f;
+    CUDA_TRY(cudaEventElapsedTime(&t, r.a, r.b));
+    if (r.kind < n_kinds) { ms[r.kind] += t; launches[r.kind] += 1; }
+  }
+  g_prof.recs.clear();
+  g_prof.used = 0;
+  return KVS_OK;
+}
+
+const char* kvs_profile_kind_name(int32_t kind) {
+  return (kind >= 0 && kind < KVS_K_COUNT) ? kKindNames[kind] : nullptr;
+}
+
+}  // extern "C"

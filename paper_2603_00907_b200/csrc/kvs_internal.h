@@ -1,0 +1,143 @@
+// Internal declarations shared by the translation units of libkvs.so.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvs.h"
+
+#define KVS_D 128                 // head dimension
+#define KVS_SEQ_CHUNK 32          // sequences handled by one launch (kernel-parameter table)
+#define KVS_MAX_M 1024            // query rows per KV head (group * window or group * n_new)
+#define KVS_MAX_SPLITS 64         // key splits of the attention partials
+#define KVS_MAX_ROUNDS 64
+#define KVS_CTILE 64              // slots per compaction tile (32 candidate pairs)
+#define KVS_SPIN_LIMIT (1 << 22)  // iterations of any device-side wait before it gives up
+
+// ----------------------------------------------------------------------------- kernel kinds
+enum KvsKernelKind {
+  KVS_K_FLASH = 0,     // window / decode attention partials
+  KVS_K_COMBINE = 1,   // partial combine
+  KVS_K_STATS = 2,     // Hessian statistics + cosine + score + weight
+  KVS_K_SELECT = 3,    // exact R-smallest selection + tile prefix
+  KVS_K_COMPACT = 4,   // merge + in-place compaction
+  KVS_K_MISC = 5,      // mask scan for kvs_compact, copies of diagnostics
+  KVS_K_COUNT = 6
+};
+
+// ----------------------------------------------------------------------------- launch tables
+struct SeqRound {
+  int32_t n;   // slots in use at the start of the round (0: sequence inactive)
+  int32_t P;   // candidate pairs
+  int32_t R;   // pairs to merge
+  int32_t b;   // sequence index in the caller's batch
+};
+
+struct RoundTable {
+  int32_t nseq;  // entries used
+  int32_t off;   // first candidate slot: sink + (round mod 2)
+  SeqRound s[KVS_SEQ_CHUNK];
+};
+
+struct CacheView {
+  __nv_bfloat16* K;
+  __nv_bfloat16* V;
+  int32_t* counts;
+  int64_t ksb, ksh, kst, vsb, vsh, vst;
+  int32_t n_max;   // slot capacity (counts row length)
+  int32_t Hkv;
+};
+
+struct FlashArgs {
+  CacheView c;
+  const __nv_bfloat16* q;  // [B, Hq, Wq, 128]
+  int32_t Hq, G, Wq, M;    // M = G * Wq rows per KV head
+  int32_t causal;
+  float scale_log2;        // softmax_scale * log2(e)
+  int32_t splits;
+  int32_t split_len;       // keys per split (multiple of the key tile)
+  float2* part_ml;         // [U, splits, M]  (running max in log2 units, sum)
+  float* part_o;           // [U, splits, M, 128]
+};
+
+struct CombineArgs {
+  int32_t M, splits, Hkv;
+  const float2* part_ml;
+  const float* part_o;
+  float4* qstat;           // [U, M]: (max log2, Z, |o|^2, lse natural)
+  float* o;                // [U, M, 128] fp32 (may be NULL)
+  __nv_bfloat16* out_bf16; // decode: [B, Hq, n_new, 128] == [U, M, 128] (may be NULL)
+  float* lse_out;          // optional [U, M]
+  float* o_out;            // optional diagnostic copy [U, M, 128]
+};
+
+struct StatsArgs {
+  CacheView c;
+  const __nv_bfloat16* q;
+  int32_t Hq, G, Wq, M;
+  int32_t causal;
+  float scale_log2;
+  int32_t score_mode;
+  const float4* qstat;
+  const float* o;
+  int32_t pair_stride;     // row length of the per-pair arrays (n_max / 2)
+  float* score;            // [U, pair_stride]
+  float* w;                // [U, pair_stride]
+  float* A;                // optional diagnostics [U, n_max]
+  float* N1;
+  float* N12;              // [U, pair_stride]
+  float* cosv;
+};
+
+struct SelectArgs {
+  int32_t Hkv;
+  int32_t pair_stride;
+  int32_t tile_stride;     // row length of tile_prefix
+  const float* score;
+  uint8_t* mask;           // [U, pair_stride]
+  int32_t* tile_prefix;    // [U, tile_stride]: merged pairs before each compaction tile
+  int32_t from_mask;       // 1: mask is an input (kvs_compact), only the prefix is built
+};
+
+struct CompactArgs {
+  CacheView c;
+  int32_t pair_stride, tile_stride;
+  const uint8_t* mask;
+  const float* w;
+  const int32_t* tile_prefix;
+  uint32_t* tickets;       // [U] zero at launch
+  uint32_t* flags;         // [U, tile_stride]; value >= epoch means "tile loaded"
+  uint32_t epoch;
+  int32_t* new_index;      // optional [U, n_max]
+  int32_t* status_dev;
+};
+
+// ----------------------------------------------------------------------------- launchers
+// Each returns the cudaError_t of its launch.  `nseq_units` = table.nseq * Hkv.
+cudaError_t kvs_launch_flash_simt(const FlashArgs& a, const RoundTable& t, cudaStream_t st);
+cudaError_t kvs_launch_combine(const CombineArgs& a, const RoundTable& t, cudaStream_t st);
+cudaError_t kvs_launch_stats_simt(const StatsArgs& a, const RoundTable& t, cudaStream_t st);
+cudaError_t kvs_launch_select(const SelectArgs& a, const RoundTable& t, cudaStream_t st);
+cudaError_t kvs_launch_compact(const CompactArgs& a, const RoundTable& t, cudaStream_t st);
+
+// ----------------------------------------------------------------------------- device helpers
+#ifdef __CUDACC__
+__device__ __forceinline__ float bf16lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_u32(uint32_t* p, uint32_t v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+#endif

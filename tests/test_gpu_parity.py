@@ -1,0 +1,333 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import kvs_oracle as oc
+from paper_2603_00907_b200 import workloads as wl
+from tests import kvs_testlib as tl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def kb():
+    from paper_2603_00907_b200 import binding, build
+    build.build()
+    binding.lib()
+    return binding
+
+
+def _setup(kb, w, data, **pkw):
+    import torch
+    dev = tl.upload_layer(data)
+    p = kb.make_params(dev["K"], dev["V"], w.n_q_heads, w.window, sink=w.sink,
+                       round_frac=w.round_frac, **pkw)
+    ws = torch.empty(kb.kvs_workspace_size(p, w.n_max, max(w.n_decode, 0)), dtype=torch.uint8,
+                     device="cuda")
+    return dev, p, ws
+
+
+def _oracle_kwargs(w, **kw):
+    d = dict(window=w.window, sink=w.sink, recent=w.window, scale=1.0 / math.sqrt(128),
+             causal=True, round_frac=w.round_frac, score_mode=0)
+    d.update(kw)
+    return d
+
+
+def _check_round_stats(kb, w, K, V, C, q_win, n_list, r, score_mode=0, causal=True):
+    """One round of statistics on caches K,V,C (numpy, [B,Hkv,Nmax,...]) vs the oracle."""
+    import torch
+    data = {"K": K, "V": V, "counts": C, "q_win": q_win, "q_new": np.zeros((0,), np.uint16)}
+    dev, p, ws = _setup(kb, w, data, first_round=r, score_mode=score_mode, causal=causal)
+    B, Hkv, Nmax = K.shape[:3]
+    G, M = w.group, w.group * w.window
+    f32 = dict(dtype=torch.float32, device="cuda")
+    A = torch.full((B, Hkv, Nmax), float("nan"), **f32)
+    N1 = torch.full((B, Hkv, Nmax), float("nan"), **f32)
+    N12, cosv, score, wgt = (torch.full((B, Hkv, Nmax // 2), float("nan"), **f32) for _ in range(4))
+    mask = torch.zeros((B, Hkv, Nmax // 2), dtype=torch.uint8, device="cuda")
+    o_win = torch.zeros((B, Hkv, M, 128), **f32)
+    lse = torch.zeros((B, Hkv, M), **f32)
+    kb.kvs_window_stats(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], n_list, list(w.budgets),
+                        ws, A=A, N1=N1, N12=N12, cosv=cosv, score=score, w=wgt, mask=mask,
+                        o_win=o_win, lse_win=lse)
+    torch.cuda.synchronize()
+    A, N1, N12, cosv, score, wgt, mask, o_win = (t.cpu().numpy() for t in
+                                                 (A, N1, N12, cosv, score, wgt, mask, o_win))
+    refs = {}
+    report = []
+    for b in range(B):
+        n = n_list[b]
+        if n <= w.budgets[b]:
+            continue
+        for h in range(Hkv):
+            st = oc.round_stats(K[b, h, :n], V[b, h, :n], C[b, h, :n].astype(np.int64),
+                                q_win[b, h * G:(h + 1) * G], w.budgets[b], r,
+                                **_oracle_kwargs(w, score_mode=score_mode, causal=causal))
+            refs[(b, h)] = st
+            off, P, R = st["off"], st["P"], st["R"]
+            sl = slice(off, off + 2 * P)
+            for name, g, ref in (("A", A[b, h, sl], st["A"][sl]), ("N1", N1[b, h, sl], st["N1"][sl]),
+                                 ("N12", N12[b, h, :P], st["N12"]), ("score", score[b, h, :P], st["score"]),
+                                 ("o", o_win[b, h], st["o"])):
+                ok, ratio, plain = tl.stat_close(g, ref)
+                report.append((b, h, name, ratio, plain))
+                assert ok, f"{name} unit {(b, h)} round {r}: err/allowed {ratio:.3g} plain rel {plain:.3g}"
+            # cosine: compared through 1 - cos (what the score uses), absolute 1e-6
+            assert np.max(np.abs(cosv[b, h, :P] - st["cos"])) < 2e-6
+            # weights: compare where the denominator is well conditioned
+            D = st["N1"][off:off + 2 * P:2] - 2 * st["N12"] + st["N1"][off + 1:off + 2 * P:2]
+            good = D > 1e-3 * (st["N1"][off:off + 2 * P:2] + st["N1"][off + 1:off + 2 * P:2])
+            assert np.max(np.abs(wgt[b, h, :P][good] - st["w"][good])) < 2e-3
+            assert np.all((wgt[b, h, :P] >= 0) & (wgt[b, h, :P] <= 1))
+            ok, nm, nout = tl.mask_band_ok(mask[b, h, :P], st["mask"], st["score"], R)
+            assert ok, f"mask unit {(b, h)} round {r}: {nm} mismatches, {nout} outside the band"
+    return refs, {"mask": mask, "w": wgt, "report": report}
+
+
+def _small(seed=1, **kw):
+    d = dict(batch=2, n_q_heads=8, n_kv_heads=2, window=8, seq_lens=(300, 517), budgets=(100, 170))
+    d.update(kw)
+    return wl.small_case(seed, **d)
+
+
+def test_window_stats_round0(kb):
+    w = _small()
+    data = wl.make_layer(w)
+    _check_round_stats(kb, w, data["K"], data["V"], data["counts"], data["q_win"], list(w.seq_lens), 0)
+
+
+def test_window_stats_modes(kb):
+    w = _small(seed=2, seq_lens=(260, 131), budgets=(90, 60))
+    data = wl.make_layer(w)
+    _check_round_stats(kb, w, data["K"], data["V"], data["counts"], data["q_win"], list(w.seq_lens), 1,
+                       score_mode=1)
+    _check_round_stats(kb, w, data["K"], data["V"], data["counts"], data["q_win"], list(w.seq_lens), 0,
+                       causal=False)
+
+
+def _oracle_round(w, K, V, C, q_win, n_list, r, w_override=None, mask_override=None):
+    """Advance every unit by one oracle round.  Returns new arrays + per-unit info."""
+    B, Hkv, Nmax = K.shape[:3]
+    G = w.group
+    Kn, Vn, Cn = np.zeros_like(K), np.zeros_like(V), np.zeros_like(C)
+    idx = np.zeros((B, Hkv, Nmax), dtype=np.int32)
+    n_new, info = [], {}
+    for b in range(B):
+        n = n_list[b]
+        if n <= w.budgets[b]:
+            Kn[b], Vn[b], Cn[b] = K[b], V[b], C[b]
+            n_new.append(n)
+            continue
+        for h in range(Hkv):
+            st = oc.round_stats(K[b, h, :n], V[b, h, :n], C[b, h, :n].astype(np.int64),
+                                q_win[b, h * G:(h + 1) * G], w.budgets[b], r, **_oracle_kwargs(w))
+            ww = st["w"] if w_override is None else w_override[b, h, :st["P"]].astype(np.float64)
+            mm = st["mask"] if mask_override is None else mask_override[b, h, :st["P"]]
+            k2, v2, c2, ix = oc.apply_merge(K[b, h, :n], V[b, h, :n], C[b, h, :n].astype(np.int64),
+                                            st["off"], mm, ww)
+            m = k2.shape[0]
+            Kn[b, h, :m], Vn[b, h, :m], Cn[b, h, :m] = k2, v2, c2
+            idx[b, h, :n] = ix
+            info[(b, h)] = st
+        n_new.append(n - info[(b, 0)]["R"])
+    return Kn, Vn, Cn, idx, n_new, info
+
+
+def test_compact_bit_exact_given_mask(kb):
+    """Same mask and fp32 weights -> indices, counts and value sums bit-exact; keys within one
+    bf16 ulp (fp32 vs float64 evaluation of the convex combination)."""
+    import torch
+    w = _small(seed=3)
+    data = wl.make_layer(w)
+    K, V, C = data["K"], data["V"], data["counts"]
+    B, Hkv, Nmax = K.shape[:3]
+    n_list = list(w.seq_lens)
+    for r in (0, 1):
+        # oracle decision, weights rounded to fp32 as the GPU stores them
+        _, _, _, _, _, info = _oracle_round(w, K, V, C, data["q_win"], n_list, r)
+        mask = np.zeros((B, Hkv, Nmax // 2), dtype=np.uint8)
+        wgt = np.zeros((B, Hkv, Nmax // 2), dtype=np.float32)
+        for (b, h), st in info.items():
+            mask[b, h, :st["P"]] = st["mask"]
+            wgt[b, h, :st["P"]] = st["w"].astype(np.float32)
+        Kn, Vn, Cn, idx, n_new, _ = _oracle_round(w, K, V, C, data["q_win"], n_list, r,
+                                                  w_override=wgt, mask_override=mask)
+        dev, p, ws = _setup(kb, w, {**data, "K": K, "V": V, "counts": C}, first_round=r)
+        new_index = torch.full((B, Hkv, Nmax), -1, dtype=torch.int32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        n_merge = [info[(b, 0)]["R"] for b in range(B)]
+        got_len = kb.kvs_compact(p, dev["K"], dev["V"], dev["counts"], torch.from_numpy(mask).cuda(),
+                                 torch.from_numpy(wgt).cuda(), n_list, n_merge, ws,
+                                 new_index=new_index, status_dev=status)
+        torch.cuda.synchronize()
+        assert status.item() == 0 and got_len == n_new
+        Kg, Vg, Cg = tl.bits_of(dev["K"]), tl.bits_of(dev["V"]), dev["counts"].cpu().numpy()
+        ig = new_index.cpu().numpy()
+        for b in range(B):
+            m, n = n_new[b], n_list[b]
+            assert np.array_equal(Cg[b, :, :m], Cn[b, :, :m])
+            assert np.array_equal(ig[b, :, :n], idx[b, :, :n])
+            assert np.array_equal(Vg[b, :, :m], Vn[b, :, :m])
+            ok, mx, nulp, worse = tl.bf16_close(Kg[b, :, :m], Kn[b, :, :m], atol=0.0)
+            assert ok, (mx, nulp, worse)
+            assert nulp <= 0.01 * Kg[b, :, :m].size
+        K, V, C, n_list = Kn, Vn, Cn, n_new
+
+
+def test_merge_layer_stagewise_and_end_to_end(kb):
+    """Round by round from the oracle's state (statistics, mask modulo the cutoff band, merge),
+    then the whole pass in one call: it must equal the composition of single-round calls bit
+    for bit, and the oracle that follows the GPU's near-cutoff choices."""
+    import torch
+    w = _small(seed=4, seq_lens=(700, 333), budgets=(128, 64))
+    data = wl.make_layer(w)
+    B, Hkv, Nmax = data["K"].shape[:3]
+    G = w.group
+    plans = [oc.full_plan(n, bud, w.sink, w.window, w.round_frac) for n, bud in zip(w.seq_lens, w.budgets)]
+    rounds = max(len(pl) for pl in plans)
+
+    # (1) full pass in one call
+    dev, p, ws = _setup(kb, w, data)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    new_len = kb.kvs_merge_layer(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], list(w.seq_lens),
+                                 list(w.budgets), ws, status_dev=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0 and new_len == list(w.budgets)
+    K_full, V_full, C_full = tl.bits_of(dev["K"]), tl.bits_of(dev["V"]), dev["counts"].cpu().numpy()
+
+    # (2) the same pass as single-round calls, recording the GPU's masks
+    dev2, _, ws2 = _setup(kb, w, data)
+    n_list = list(w.seq_lens)
+    gpu_masks = []
+    for r in range(rounds):
+        pr = kb.make_params(dev2["K"], dev2["V"], w.n_q_heads, w.window, sink=w.sink,
+                            round_frac=w.round_frac, first_round=r)
+        mask = torch.zeros((B, Hkv, Nmax // 2), dtype=torch.uint8, device="cuda")
+        kb.kvs_window_stats(pr, dev2["K"], dev2["V"], dev2["counts"], dev2["q_win"], n_list,
+                            list(w.budgets), ws2, mask=mask)
+        step_budget = [plans[b][r][0] - plans[b][r][3] if r < len(plans[b]) else w.budgets[b]
+                       for b in range(B)]
+        n_list = kb.kvs_merge_layer(pr, dev2["K"], dev2["V"], dev2["counts"], dev2["q_win"], n_list,
+                                    step_budget, ws2)
+        gpu_masks.append(mask.cpu().numpy())
+    torch.cuda.synchronize()
+    assert n_list == list(w.budgets)
+    for b in range(B):
+        m = w.budgets[b]
+        assert np.array_equal(tl.bits_of(dev2["K"])[b, :, :m], K_full[b, :, :m])
+        assert np.array_equal(tl.bits_of(dev2["V"])[b, :, :m], V_full[b, :, :m])
+        assert np.array_equal(dev2["counts"].cpu().numpy()[b, :, :m], C_full[b, :, :m])
+
+    # (3) oracle following the GPU's masks; every deviation from its own mask must be in the band
+    flips = 0
+    for b in range(B):
+        n0 = w.seq_lens[b]
+        for h in range(Hkv):
+            forced = [gpu_masks[r][b, h, :plans[b][r][2]] for r in range(len(plans[b]))]
+            trace = []
+            Ko, Vo, Co = oc.merge_unit(data["K"][b, h, :n0], data["V"][b, h, :n0],
+                                       data["counts"][b, h, :n0], data["q_win"][b, h * G:(h + 1) * G],
+                                       w.budgets[b], forced_masks=forced, trace=trace,
+                                       **_oracle_kwargs(w))
+            for r, st in enumerate(trace):
+                ok, nm, nout = tl.mask_band_ok(forced[r], st["mask"], st["score"], st["R"])
+                assert ok, f"unit {(b, h)} round {r}: {nm} mask mismatches, {nout} outside the band"
+                flips += nm
+            m = w.budgets[b]
+            assert np.array_equal(C_full[b, h, :m], Co)
+            assert Co.sum() == n0
+            okk, mxk, nulpk, _ = tl.bf16_close(K_full[b, h, :m], Ko)
+            okv, mxv, nulpv, _ = tl.bf16_close(V_full[b, h, :m], Vo)
+            assert okk and okv, (mxk, mxv)
+    print(f"band flips followed: {flips}")
+
+
+def test_decode_matches_oracle_and_is_lossless_on_identical_keys(kb):
+    import torch
+    w = _small(seed=5, seq_lens=(400, 257), budgets=(90, 60), n_decode=5)
+    data = wl.make_layer(w)
+    # plant identical neighbours so that round 0 merges them first
+    for b in range(w.batch):
+        for j in (40, 60, 100):
+            data["K"][b, :, j + 1] = data["K"][b, :, j]
+    dev, p, ws = _setup(kb, w, data)
+    B, Hq, T = w.batch, w.n_q_heads, w.n_decode
+    G, Hkv = w.group, w.n_kv_heads
+    out0 = torch.zeros((B, Hq, T, 128), dtype=torch.bfloat16, device="cuda")
+    lse0 = torch.zeros((B, Hq, T), dtype=torch.float32, device="cuda")
+    kb.kvs_decode_attn(p, dev["q_new"], dev["K"], dev["V"], dev["counts"], list(w.seq_lens), out0, ws,
+                       lse=lse0)
+    torch.cuda.synchronize()
+    o0 = tl.bits_of(out0)
+    for b in range(B):
+        n = w.seq_lens[b]
+        for h in range(Hkv):
+            ref, lse_ref = oc.decode_attention(data["q_new"][b, h * G:(h + 1) * G], data["K"][b, h, :n],
+                                               data["V"][b, h, :n], data["counts"][b, h, :n])
+            ok, mx, _, _ = tl.bf16_close(o0[b, h * G:(h + 1) * G], oc.f64_to_bf16(ref))
+            assert ok, mx
+            assert np.max(np.abs(lse0[b, h * G:(h + 1) * G].cpu().numpy() - lse_ref)) < 1e-4
+    # merge to the budget, decode again, compare with the oracle's merged cache
+    new_len = kb.kvs_merge_layer(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], list(w.seq_lens),
+                                 list(w.budgets), ws)
+    out1 = torch.zeros_like(out0)
+    kb.kvs_decode_attn(p, dev["q_new"], dev["K"], dev["V"], dev["counts"], new_len, out1, ws)
+    torch.cuda.synchronize()
+    Kg, Vg, Cg = tl.bits_of(dev["K"]), tl.bits_of(dev["V"]), dev["counts"].cpu().numpy()
+    o1 = tl.bits_of(out1)
+    for b in range(B):
+        m = new_len[b]
+        for h in range(Hkv):
+            ref, _ = oc.decode_attention(data["q_new"][b, h * G:(h + 1) * G], Kg[b, h, :m], Vg[b, h, :m],
+                                         Cg[b, h, :m])
+            ok, mx, _, _ = tl.bf16_close(o1[b, h * G:(h + 1) * G], oc.f64_to_bf16(ref))
+            assert ok, mx
+
+
+def test_identical_key_merge_is_lossless_on_gpu(kb):
+    """One round that merges only planted identical-key pairs leaves decode unchanged."""
+    import torch
+    w = _small(seed=6, batch=1, seq_lens=(200,), budgets=(197,), n_decode=4)
+    data = wl.make_layer(w)
+    for j in (50, 80, 120):          # even offsets from sink=32 -> aligned candidate pairs
+        data["K"][0, :, j + 1] = data["K"][0, :, j]
+    dev, p, ws = _setup(kb, w, data)
+    out0 = torch.zeros((1, w.n_q_heads, 4, 128), dtype=torch.bfloat16, device="cuda")
+    lse0 = torch.zeros((1, w.n_q_heads, 4), dtype=torch.float32, device="cuda")
+    kb.kvs_decode_attn(p, dev["q_new"], dev["K"], dev["V"], dev["counts"], [200], out0, ws, lse=lse0)
+    K_before = tl.bits_of(dev["K"]).copy()
+    new_len = kb.kvs_merge_layer(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], [200], [197], ws)
+    out1, lse1 = torch.zeros_like(out0), torch.zeros_like(lse0)
+    kb.kvs_decode_attn(p, dev["q_new"], dev["K"], dev["V"], dev["counts"], new_len, out1, ws, lse=lse1)
+    torch.cuda.synchronize()
+    assert new_len == [197]
+    Kg, Cg = tl.bits_of(dev["K"]), dev["counts"].cpu().numpy()
+    assert np.array_equal(Cg[0, :, 50], np.full(w.n_kv_heads, 2))
+    assert np.array_equal(Kg[0, :, 50], K_before[0, :, 50])                 # K* == K exactly
+    assert np.array_equal(Kg[0, :, 51], K_before[0, :, 52])                 # shifted by one
+    assert Cg[0, :, :197].sum() == 200 * w.n_kv_heads
+    assert torch.max(torch.abs(lse1 - lse0)).item() < 1e-5
+    assert torch.max(torch.abs(out1.float() - out0.float())).item() <= 2e-2
+
+
+def test_noop_and_error_paths_on_device(kb):
+    import torch
+    w = _small(seed=7, batch=1, seq_lens=(150,), budgets=(150,))
+    data = wl.make_layer(w)
+    dev, p, ws = _setup(kb, w, data)
+    before = tl.bits_of(dev["K"]).copy()
+    assert kb.kvs_merge_layer(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], [150], [150], ws) == [150]
+    assert kb.kvs_merge_layer(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], [100], [150], ws) == [100]
+    torch.cuda.synchronize()
+    assert np.array_equal(tl.bits_of(dev["K"]), before)
+    with pytest.raises(kb.KvsError) as e:      # sink + recent = 40 > budget 20
+        kb.kvs_merge_layer(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], [150], [20], ws)
+    assert e.value.code == 4
+    with pytest.raises(kb.KvsError) as e:
+        kb.kvs_merge_layer(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], [150], [100], ws[:1024])
+    assert e.value.code == 3
+    torch.cuda.synchronize()
+    assert np.array_equal(tl.bits_of(dev["K"]), before)
