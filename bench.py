@@ -1,0 +1,364 @@
+"""Benchmark of the KV-merge pass (one JSON line on stdout).
+
+A step is one pass of the whole hot path over the workload: for every layer, the in-place
+merge pass of all KV heads (window attention, Hessian statistics, selection, merge,
+compaction, every round down to the budget) followed by decode attention of new query
+tokens over the merged cache.  The headline `value` is context tokens consumed per second
+per layer, B * n_0 * layers / step time, with the cache resident in HBM; `e2e` repeats it
+through the same C-ABI calls with the inputs in pinned host memory (host->device copies
+and the device->host read of the merged cache inside the timed region).
+
+`--impl reference` times the float64 CPU oracle on a bounded sample of the same workload.
+"""
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2603_00907_b200 import workloads as wl  # noqa: E402
+
+METRIC = "kv_tokens_merged_per_sec_per_layer"
+UNIT = "tokens/s"
+DECODE_TOKENS = 1          # new query tokens per sequence when the config names none
+
+# algorithmic HBM bytes per cache slot and round, per kernel kind (d = 128, bf16 cache)
+ROW_BYTES = 2 * 128 * 2 + 4          # key + value sum + count
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while running."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.rows, self.proc = index, [], None
+
+    def run(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            for line in self.proc.stdout:
+                self.rows.append([c.strip() for c in line.split(",")])
+        except Exception:
+            pass
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+        self.join(timeout=2)
+        sm, mx, reasons = [], 0, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = max(mx, float(r[1]))
+                for nm, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nm)
+            except Exception:
+                continue
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx or None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def plan_rounds(w, oracle_free=True):
+    """(n_r, off, P, R) per round for each sequence, from the closed-form schedule."""
+    out = []
+    for n, bud in zip(w.seq_lens, w.budgets):
+        rounds, r = [], 0
+        while n > bud:
+            off = w.sink + (r % 2)
+            P = (n - off - w.window) // 2
+            R = min(n - bud, max(1, int(math.floor(w.round_frac * P))))
+            rounds.append((n, off, P, R))
+            n -= R
+            r += 1
+        out.append(rounds)
+    return out
+
+
+def algorithmic_bytes(w, n_layers):
+    """Algorithmic HBM bytes of one step, per kernel kind (summed over layers, heads, rounds)."""
+    plans = plan_rounds(w)
+    slots = sum(n for pl in plans for (n, _, _, _) in pl) * w.n_kv_heads * n_layers
+    kept = sum(n - R for pl in plans for (n, _, _, R) in pl) * w.n_kv_heads * n_layers
+    pairs = sum(P for pl in plans for (_, _, P, _) in pl) * w.n_kv_heads * n_layers
+    return {
+        "attn_partials": slots * ROW_BYTES,
+        "hessian_stats": slots * ROW_BYTES + pairs * 8,
+        "select": pairs * (4 + 1),
+        "merge_compact": slots * ROW_BYTES + kept * ROW_BYTES + pairs * 5,
+    }, slots
+
+
+def run_reference(args, w):
+    """The CPU oracle on one (layer, KV head) unit per step; tokens/s per layer = n_0 / (Hkv * t)."""
+    from oracle import kvs_oracle as oc
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    try:
+        import threadpoolctl
+        cores = max(i.get("num_threads", 1) for i in threadpoolctl.threadpool_info()) or 1
+    except Exception:
+        cores = os.cpu_count() or 1
+    data = wl.make_layer(w, 0)
+    n0, G = w.seq_lens[0], w.group
+
+    def one():
+        t = time.perf_counter()
+        oc.merge_unit(data["K"][0, 0, :n0], data["V"][0, 0, :n0], data["counts"][0, 0, :n0],
+                      data["q_win"][0, 0:G], w.budgets[0], window=w.window, sink=w.sink,
+                      round_frac=w.round_frac)
+        return time.perf_counter() - t
+
+    for _ in range(args.warmup):
+        one()
+    times = [one() for _ in range(args.steps)]
+    t_unit = sum(times) / len(times)
+    value = n0 / (w.n_kv_heads * t_unit)
+    sample = (f"one (layer, KV head) unit of sequence 0 per step ({n0} tokens, all rounds to budget "
+              f"{w.budgets[0]}); a layer is {w.n_kv_heads} such units per sequence, so tokens/s per "
+              f"layer = n_0 / ({w.n_kv_heads} * unit seconds)")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_unit,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_config(w, args),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def workload_config(w, args):
+    return {"workload": f"configs[{w.config_id}] {w.name}", "layers": w.layers, "batch": w.batch,
+            "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": 128,
+            "context": list(w.seq_lens), "window": w.window, "budget": list(w.budgets),
+            "sink": w.sink, "round_frac": w.round_frac,
+            "decode_new_tokens": w.n_decode or DECODE_TOKENS,
+            "l2": "inputs larger than L2 (fresh cache restored from a device master copy before "
+                  "every step, outside the timed events)",
+            "parallelism": f"dp{args.gpus} over sequences, no collective"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (debug)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    w = wl.config(args.config)
+    if args.layers:
+        w = w.scaled(layers=args.layers)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2603_00907_b200 import binding as kb, build as kbuild
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        kbuild.build()
+    if world > 1:
+        dist.barrier()
+    kb.lib()
+
+    L, B, Hq, Hkv, W, Nmax = w.layers, w.batch, w.n_q_heads, w.n_kv_heads, w.window, w.n_max
+    T = w.n_decode or DECODE_TOKENS
+    # ---- inputs: generated on the host, kept in pinned memory, master copy on the device
+    layers = wl.make_layers_parallel(w.scaled(n_decode=T), range(L), seq_offset=rank)
+    pin = lambda shape, dt: torch.empty(shape, dtype=dt, pin_memory=True)
+    hK, hV = pin((L, B, Hkv, Nmax, 128), torch.int16), pin((L, B, Hkv, Nmax, 128), torch.int16)
+    hQ, hQn = pin((L, B, Hq, W, 128), torch.int16), pin((L, B, Hq, T, 128), torch.int16)
+    hC = pin((L, B, Hkv, Nmax), torch.int32)
+    for l, d in enumerate(layers):
+        hK[l].copy_(torch.from_numpy(d["K"].view(np.int16)))
+        hV[l].copy_(torch.from_numpy(d["V"].view(np.int16)))
+        hQ[l].copy_(torch.from_numpy(d["q_win"].view(np.int16)))
+        hQn[l].copy_(torch.from_numpy(d["q_new"].view(np.int16)))
+        hC[l].copy_(torch.from_numpy(d["counts"]))
+    del layers
+    dev = torch.device("cuda", local)
+    mK, mV, mC = hK.to(dev), hV.to(dev), hC.to(dev)
+    wK, wV, wC = torch.empty_like(mK), torch.empty_like(mV), torch.empty_like(mC)
+    dQ, dQn = hQ.to(dev), hQn.to(dev)
+    out = torch.zeros((L, B, Hq, T, 128), dtype=torch.int16, device=dev)
+    bud_max = max(w.budgets)
+    hRes = pin((2, L, B, Hkv, bud_max, 128), torch.int16)
+    hResC = pin((L, B, Hkv, bud_max), torch.int32)
+    hOut = pin((L, B, Hq, T, 128), torch.int16)
+    bf = lambda t: t.view(torch.bfloat16)
+    p = kb.make_params(bf(wK[0]), bf(wV[0]), Hq, W, sink=w.sink, round_frac=w.round_frac)
+    ws = torch.empty(kb.kvs_workspace_size(p, Nmax, T), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    seq_len, budget = list(w.seq_lens), list(w.budgets)
+
+    def restore():
+        wK.copy_(mK); wV.copy_(mV); wC.copy_(mC)
+
+    def step():
+        for l in range(L):
+            new_len = kb.kvs_merge_layer(p, bf(wK[l]), bf(wV[l]), wC[l], bf(dQ[l]), seq_len, budget, ws,
+                                         status_dev=status)
+            kb.kvs_decode_attn(p, bf(dQn[l]), bf(wK[l]), bf(wV[l]), wC[l], new_len, bf(out[l]), ws)
+
+    def e2e_step():
+        wK.copy_(hK, non_blocking=True); wV.copy_(hV, non_blocking=True)
+        wC.copy_(hC, non_blocking=True)
+        dQ.copy_(hQ, non_blocking=True); dQn.copy_(hQn, non_blocking=True)
+        step()
+        hRes[0].copy_(wK[:, :, :, :bud_max], non_blocking=True)
+        hRes[1].copy_(wV[:, :, :, :bud_max], non_blocking=True)
+        hResC.copy_(wC[:, :, :, :bud_max], non_blocking=True)
+        hOut.copy_(out, non_blocking=True)
+
+    def timed(fn, steps, prepare=None):
+        total = 0.0
+        for _ in range(steps):
+            if prepare:
+                prepare()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            b.synchronize()
+            total += a.elapsed_time(b)
+        return total
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident timing
+    for _ in range(args.warmup):
+        restore(); step()
+    sync_all()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = kb.kvs_launch_count()
+    total_ms = timed(step, args.steps, prepare=restore)
+    sync_all()
+    launches = kb.kvs_launch_count() - launches0
+    clocks = sampler.stop()
+    total_ms = max_over_ranks(total_ms)
+    if status.item() != 0:
+        raise RuntimeError(f"device status {status.item()}")
+    ms_per_step = total_ms / args.steps
+    tokens_per_step = world * L * sum(w.seq_lens)
+    value = tokens_per_step / (ms_per_step * 1e-3)
+
+    # ---- per-kernel timing of the same steps (events around every launch; separate pass)
+    restore(); torch.cuda.synchronize()
+    kb.kvs_profile_begin()
+    for _ in range(min(args.steps, 2)):
+        restore(); step()
+    torch.cuda.synchronize()
+    prof = kb.kvs_profile_end()
+    n_prof = min(args.steps, 2)
+    alg, slot_rounds = algorithmic_bytes(w, L)
+    kinds = {k: v for k, v in prof.items() if v[1] > 0}
+    top = max(kinds, key=lambda k: kinds[k][0])
+    peak, peak_src = measured_peaks()
+    top_ms, top_launches = kinds[top]
+    achieved = alg.get(top, 0) * n_prof / (top_ms * 1e-3) / 1e9 if top in alg else None
+    roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": (achieved / peak) if achieved else None, "traffic": None,
+                "peak_source": f"of {peak_src}",
+                "avg_launch_us": 1e3 * top_ms / top_launches,
+                "algorithmic_bytes_per_launch": alg.get(top, 0) * n_prof / top_launches,
+                "per_kernel": {k: {"ms_per_step": v[0] / n_prof, "launches_per_step": v[1] // n_prof,
+                                   "GBps": (alg[k] * n_prof / (v[0] * 1e-3) / 1e9) if k in alg else None}
+                               for k, v in kinds.items()}}
+
+    # ---- end to end through the C ABI with host buffers
+    e2e = None
+    if not args.no_e2e:
+        e2e_step(); sync_all()
+        e2e_ms = max_over_ranks(timed(e2e_step, max(1, min(args.steps, 3)))) / max(1, min(args.steps, 3))
+        sync_all()
+        h2d = sum(t.numel() * t.element_size() for t in (hK, hV, hC, hQ, hQn))
+        d2h = sum(t.numel() * t.element_size() for t in (hRes, hResC, hOut))
+        e2e = {"value": tokens_per_step / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    # ---- CPU oracle on a bounded sample (rank 0, N = 1 only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import kvs_oracle as oc
+        d0 = wl.make_layer(w, 0)
+        n0 = w.seq_lens[0]
+        t0 = time.perf_counter()
+        oc.merge_unit(d0["K"][0, 0, :n0], d0["V"][0, 0, :n0], d0["counts"][0, 0, :n0],
+                      d0["q_win"][0, 0:w.group], w.budgets[0], window=W, sink=w.sink,
+                      round_frac=w.round_frac)
+        t_unit = time.perf_counter() - t0
+        try:
+            import threadpoolctl
+            cores = max(i.get("num_threads", 1) for i in threadpoolctl.threadpool_info()) or 1
+        except Exception:
+            cores = os.cpu_count() or 1
+        cpu = {"value": n0 / (Hkv * t_unit), "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"layer 0, sequence 0, KV head 0 only ({n0} tokens, all rounds): {t_unit:.1f} s; "
+                         f"scaled to a layer of {Hkv} heads"}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": workload_config(w, args), "clocks": clocks, "e2e": e2e,
+                "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
+                "removed_tokens_per_sec_per_layer":
+                    world * L * sum(n - b for n, b in zip(w.seq_lens, w.budgets)) / (ms_per_step * 1e-3)}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -104,19 +104,21 @@ def layer_ar_coef(w: Workload, layer: int) -> float:
 
 
 def _ar1(rng: np.random.Generator, n: int, width: int, a: float, sigma: float) -> np.ndarray:
-    """x_0 ~ N(0,1); x_t = a x_{t-1} + sigma eps_t, along axis 0."""
-    eps = rng.standard_normal((n, width), dtype=np.float32)
-    eps[1:] *= np.float32(sigma)
+    """x_0 ~ N(0,1); x_t = a x_{t-1} + sigma eps_t along the token axis.  Returns [n, width]."""
+    eps = rng.standard_normal((width, n), dtype=np.float32)      # channel-major: filter rows
+    eps[:, 1:] *= np.float32(sigma)
     # y_t = a y_{t-1} + u_t with u_0 = x_0 and zero initial state
-    return lfilter([1.0], [1.0, -a], eps.astype(np.float64), axis=0).astype(np.float32)
+    y = lfilter([1.0], [1.0, -a], eps.astype(np.float64), axis=1).astype(np.float32)
+    return np.ascontiguousarray(y.T)
 
 
-def make_layer(w: Workload, layer: int = 0) -> Dict[str, np.ndarray]:
+def make_layer(w: Workload, layer: int = 0, seq_offset: int = 0) -> Dict[str, np.ndarray]:
     """Inputs of one decoder layer.
 
     Returns uint16 (bf16 bits) arrays K, V [B,Hkv,Nmax,128], q_win [B,Hq,W,128],
     q_new [B,Hq,T,128] (T = n_decode, may be 0), int32 counts [B,Hkv,Nmax] (all 1),
     and int32 seq_len / budget [B].  Rows at or beyond seq_len[b] are zero.
+    `seq_offset` shifts the per-sequence seeds (another data-parallel rank's batch).
     """
     B, Hq, Hkv, W, d = w.batch, w.n_q_heads, w.n_kv_heads, w.window, HEAD_DIM
     nmax = w.n_max
@@ -127,7 +129,7 @@ def make_layer(w: Workload, layer: int = 0) -> Dict[str, np.ndarray]:
     q_win = np.zeros((B, Hq, W, d), dtype=np.uint16)
     q_new = np.zeros((B, Hq, w.n_decode, d), dtype=np.uint16)
     for b in range(B):
-        base = 1000 * w.config_id + 10 * layer + b
+        base = 1000 * w.config_id + 10 * layer + b + 100000 * seq_offset
         n = int(w.seq_lens[b])
         rk = np.random.default_rng([base, 1])
         rv = np.random.default_rng([base, 2])
@@ -162,3 +164,16 @@ def small_case(seed: int, batch: int = 1, n_q_heads: int = 8, n_kv_heads: int = 
     return Workload(f"small_{seed}", 100 + seed, 1, batch, n_q_heads, n_kv_heads, window,
                     tuple(seq_lens), tuple(budgets), ar_coef=ar_coef, noise_literal=None,
                     n_outlier=n_outlier, outlier_std=2.0, n_decode=n_decode)
+
+
+def make_layers_parallel(w: Workload, layers, processes: Optional[int] = None, seq_offset: int = 0) -> List[Dict[str, np.ndarray]]:
+    """make_layer for several layers on a process pool (generation is the slow part of a
+    benchmark set-up; results are identical to calling make_layer one by one)."""
+    import multiprocessing as mp
+    import os
+    layers = list(layers)
+    procs = processes or min(len(layers), max(1, (os.cpu_count() or 2) - 1), 16)
+    if procs <= 1 or len(layers) <= 1:
+        return [make_layer(w, l, seq_offset) for l in layers]
+    with mp.get_context("fork").Pool(procs) as pool:
+        return pool.starmap(make_layer, [(w, l, seq_offset) for l in layers])
