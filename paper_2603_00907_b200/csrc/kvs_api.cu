@@ -4,6 +4,7 @@
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <atomic>
@@ -52,6 +53,44 @@ cudaError_t launch(int kind, cudaStream_t st, F&& f) {
   cudaEventRecord(b, st);
   g_prof.recs.push_back({kind, a, b});
   return e;
+}
+
+// ------------------------------------------------------------------------------- tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 tensor whose innermost dimension is the 128-wide head dimension; a box is
+// [64 elements x box_rows rows] with the 128-byte swizzle that the UMMA descriptors expect.
+// dims/strides are given innermost first; strides (bytes) start at dimension 1.
+bool make_tmap(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+               int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t gd[5], gs[4];
+  cuuint32_t box[5], es[5];
+  for (int i = 0; i < rank; ++i) { gd[i] = dims[i]; box[i] = 1; es[i] = 1; }
+  for (int i = 0; i + 1 < rank; ++i) gs[i] = strides_bytes[i];
+  box[0] = 64;
+  box[1] = (cuuint32_t)box_rows;
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gd, gs, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 const char* kKindNames[KVS_K_COUNT] = {"attn_partials", "combine", "hessian_stats",
@@ -110,8 +149,9 @@ void round_plan(const kvs_params_t* p, int n, int budget, int r, int* off, int* 
 size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct WsLayout {
-  size_t part_ml, part_o, qstat, o, score, w, mask, tile_prefix, sync, total;
-  int splits_max, M_max, pair_stride, tile_stride, U;
+  size_t part_ml, part_o, qstat, o, o_hi, o_lo, score, w, mask, tile_prefix, partA, partN1, partN12, partCos,
+      sync, total;
+  int splits_max, M_max, pair_stride, tile_stride, counter_stride, nqblk_w, U;
   size_t sync_bytes;
 };
 
@@ -144,9 +184,20 @@ WsLayout make_layout(const kvs_params_t* p, int n_max, int max_new) {
   L.w = o;       o += align_up((size_t)L.U * L.pair_stride * sizeof(float));
   L.mask = o;    o += align_up((size_t)L.U * L.pair_stride);
   L.tile_prefix = o; o += align_up((size_t)L.U * L.tile_stride * sizeof(int32_t));
-  // tickets [KVS_MAX_ROUNDS][U] followed by flags [U][tile_stride]; zeroed once per call
+  L.o_hi = o;    o += align_up((size_t)L.U * L.M_max * KVS_D * sizeof(__nv_bfloat16));
+  L.o_lo = o;    o += align_up((size_t)L.U * L.M_max * KVS_D * sizeof(__nv_bfloat16));
+  L.nqblk_w = (Mw + 127) / 128;
+  L.counter_stride = n_max / 128 + 2;
+  const size_t nq = L.nqblk_w > 1 ? L.nqblk_w : 0;      // partial sums only with several query blocks
+  L.partA = o;   o += align_up((size_t)L.U * nq * n_max * sizeof(float));
+  L.partN1 = o;  o += align_up((size_t)L.U * nq * n_max * sizeof(float));
+  L.partN12 = o; o += align_up((size_t)L.U * nq * L.pair_stride * sizeof(float));
+  L.partCos = o; o += align_up((size_t)L.U * (nq ? 1 : 0) * L.pair_stride * sizeof(float));
+  // tickets [KVS_MAX_ROUNDS][U], flags [U][tile_stride], tile counters [U][counter_stride];
+  // zeroed once per call
   L.sync = o;
-  L.sync_bytes = align_up(((size_t)KVS_MAX_ROUNDS * L.U + (size_t)L.U * L.tile_stride) * sizeof(uint32_t));
+  L.sync_bytes = align_up(((size_t)KVS_MAX_ROUNDS * L.U + (size_t)L.U * L.tile_stride +
+                           (size_t)L.U * L.counter_stride) * sizeof(uint32_t));
   o += L.sync_bytes;
   L.total = o;
   return L;
@@ -190,7 +241,33 @@ struct Common {
   char* ws;
   cudaStream_t st;
   int G, Mw;
+  int32_t* status_dev;
+  bool simt_stats;           // debugging aid: statistics on the CUDA cores
+  CUtensorMap tmK, tmV, tmQ, tmOhi, tmOlo;
 };
+
+bool env_simt_stats() {
+  static int v = -1;
+  if (v < 0) { const char* e = getenv("KVS_DEBUG_SIMT_STATS"); v = (e && e[0] == '1') ? 1 : 0; }
+  return v == 1;
+}
+
+// Tensor maps of one call: K and V caches [B,Hkv,n_max,128] with the caller's strides, the
+// window queries and the two bf16 terms of the attention output as [U, M, 128].
+kvs_status_t make_call_tmaps(Common* c, const void* K, const void* V, const void* q_win, int n_max) {
+  const kvs_params_t* p = c->p;
+  const uint64_t kd[4] = {KVS_D, (uint64_t)n_max, (uint64_t)p->n_kv_heads, (uint64_t)p->batch};
+  const uint64_t ks[3] = {(uint64_t)p->k_stride_t * 2, (uint64_t)p->k_stride_h * 2, (uint64_t)p->k_stride_b * 2};
+  const uint64_t vs[3] = {(uint64_t)p->v_stride_t * 2, (uint64_t)p->v_stride_h * 2, (uint64_t)p->v_stride_b * 2};
+  const uint64_t qd[3] = {KVS_D, (uint64_t)c->Mw, (uint64_t)c->L.U};
+  const uint64_t qs[2] = {KVS_D * 2, (uint64_t)c->Mw * KVS_D * 2};
+  bool ok = make_tmap(&c->tmK, K, 4, kd, ks, 128) && make_tmap(&c->tmV, V, 4, kd, vs, 128) &&
+            make_tmap(&c->tmQ, q_win, 3, qd, qs, 128) &&
+            make_tmap(&c->tmOhi, c->ws + c->L.o_hi, 3, qd, qs, 128) &&
+            make_tmap(&c->tmOlo, c->ws + c->L.o_lo, 3, qd, qs, 128);
+  if (!ok) return fail(KVS_ERR_CUDA, "cuTensorMapEncodeTiled failed or is unavailable");
+  return KVS_OK;
+}
 
 // The statistics of one round for the sequences in `tab` (window attention partials,
 // combine, Hessian statistics), and optionally the selection.
@@ -215,6 +292,8 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
   ca.part_ml = fa.part_ml; ca.part_o = fa.part_o;
   ca.qstat = reinterpret_cast<float4*>(c.ws + c.L.qstat);
   ca.o = reinterpret_cast<float*>(c.ws + c.L.o);
+  ca.o_hi = reinterpret_cast<__nv_bfloat16*>(c.ws + c.L.o_hi);
+  ca.o_lo = reinterpret_cast<__nv_bfloat16*>(c.ws + c.L.o_lo);
   ca.out_bf16 = nullptr; ca.lse_out = lse_out; ca.o_out = o_out;
   CUDA_TRY(launch(KVS_K_COMBINE, c.st, [&] { return kvs_launch_combine(ca, tab, c.st); }));
 
@@ -227,7 +306,34 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
   sa.score = score_out ? score_out : reinterpret_cast<float*>(c.ws + c.L.score);
   sa.w = w_out ? w_out : reinterpret_cast<float*>(c.ws + c.L.w);
   sa.A = A; sa.N1 = N1; sa.N12 = N12; sa.cosv = cosv;
-  CUDA_TRY(launch(KVS_K_STATS, c.st, [&] { return kvs_launch_stats_simt(sa, tab, c.st); }));
+  if (c.simt_stats) {
+    CUDA_TRY(launch(KVS_K_STATS, c.st, [&] { return kvs_launch_stats_simt(sa, tab, c.st); }));
+  } else {
+    StatsTcArgs ta;
+    ta.Hkv = p->n_kv_heads; ta.M = c.Mw; ta.nqblk = (c.Mw + 127) / 128;
+    int pmax = 0;
+    for (int i = 0; i < tab.nseq; ++i) pmax = pmax > tab.s[i].P ? pmax : tab.s[i].P;
+    const int ntiles = (2 * pmax + 127) / 128;
+    int splits = 148 / (ta.nqblk * ta.Hkv * tab.nseq);
+    if (splits < 1) splits = 1;
+    if (splits > ntiles) splits = ntiles;
+    ta.tiles_per_split = (ntiles + splits - 1) / splits;
+    ta.splits = (ntiles + ta.tiles_per_split - 1) / ta.tiles_per_split;
+    ta.n_max = view.n_max; ta.pair_stride = c.L.pair_stride; ta.counter_stride = c.L.counter_stride;
+    ta.scale_log2 = fa.scale_log2; ta.score_mode = p->score_mode;
+    ta.counts = view.counts; ta.qstat = ca.qstat;
+    ta.score = sa.score; ta.w = sa.w; ta.A = A; ta.N1 = N1; ta.N12 = N12; ta.cosv = cosv;
+    ta.partA = reinterpret_cast<float*>(c.ws + c.L.partA);
+    ta.partN1 = reinterpret_cast<float*>(c.ws + c.L.partN1);
+    ta.partN12 = reinterpret_cast<float*>(c.ws + c.L.partN12);
+    ta.partCos = reinterpret_cast<float*>(c.ws + c.L.partCos);
+    ta.tile_counter = reinterpret_cast<uint32_t*>(c.ws + c.L.sync) + (size_t)KVS_MAX_ROUNDS * c.L.U +
+                      (size_t)c.L.U * c.L.tile_stride;
+    ta.status_dev = c.status_dev;
+    CUDA_TRY(launch(KVS_K_STATS, c.st, [&] {
+      return kvs_launch_stats_tc(ta, tab, c.tmK, c.tmV, c.tmQ, c.tmOhi, c.tmOlo, c.st);
+    }));
+  }
 
   if (do_select) {
     SelectArgs se;
@@ -263,6 +369,8 @@ kvs_status_t check_common(const kvs_params_t* p, const void* K, const void* V, c
   c->st = static_cast<cudaStream_t>(stream);
   c->G = p->n_q_heads / p->n_kv_heads;
   c->Mw = c->G * p->window;
+  c->status_dev = nullptr;
+  c->simt_stats = env_simt_stats();
   return KVS_OK;
 }
 
@@ -343,6 +451,9 @@ kvs_status_t kvs_merge_layer(const kvs_params_t* p, void* K, void* V, int32_t* c
   for (int b = 0; b < B; ++b) new_len[b] = seq_len[b] < budget[b] ? seq_len[b] : budget[b];
   if (rounds == 0) return KVS_OK;
 
+  c.status_dev = status_dev;
+  s = make_call_tmaps(&c, K, V, q_win, n_max);
+  if (s != KVS_OK) return s;
   CUDA_TRY(cudaMemsetAsync(c.ws + c.L.sync, 0, c.L.sync_bytes, c.st));
   uint32_t* tickets = reinterpret_cast<uint32_t*>(c.ws + c.L.sync);
   uint32_t* flags = tickets + (size_t)KVS_MAX_ROUNDS * c.L.U;
@@ -487,7 +598,7 @@ kvs_status_t kvs_decode_attn(const kvs_params_t* p, const void* q_new, int32_t n
     CombineArgs ca;
     ca.M = M; ca.splits = fa.splits; ca.Hkv = p->n_kv_heads;
     ca.part_ml = fa.part_ml; ca.part_o = fa.part_o;
-    ca.qstat = nullptr; ca.o = nullptr;
+    ca.qstat = nullptr; ca.o = nullptr; ca.o_hi = nullptr; ca.o_lo = nullptr;
     ca.out_bf16 = static_cast<__nv_bfloat16*>(out);
     ca.lse_out = lse; ca.o_out = nullptr;
     CUDA_TRY(launch(KVS_K_COMBINE, c.st, [&] { return kvs_launch_combine(ca, tab, c.st); }));
@@ -501,7 +612,6 @@ kvs_status_t kvs_window_stats(const kvs_params_t* p, const void* K, const void* 
                               float* cosv, float* score, float* w, uint8_t* mask, float* o_win,
                               float* lse_win, void* workspace, size_t workspace_bytes,
                               int32_t* status_dev, void* cuda_stream) {
-  (void)status_dev;
   Common c;
   kvs_status_t s = check_common(p, K, V, counts, seq_len, n_max, workspace, workspace_bytes, 0, &c, cuda_stream);
   if (s != KVS_OK) return s;
@@ -520,6 +630,11 @@ kvs_status_t kvs_window_stats(const kvs_params_t* p, const void* K, const void* 
   // outputs use the caller's row lengths: per-slot n_max, per-pair n_max/2.  The internal
   // pair arrays use pair_stride, so diagnostics are written with the caller's stride by
   // running the kernels on a layout whose pair_stride is n_max/2.
+  c.status_dev = status_dev;
+  if (act.empty()) return KVS_OK;
+  s = make_call_tmaps(&c, K, V, q_win, n_max);
+  if (s != KVS_OK) return s;
+  CUDA_TRY(cudaMemsetAsync(c.ws + c.L.sync, 0, c.L.sync_bytes, c.st));
   Common cc = c;
   cc.L.pair_stride = n_max / 2;
   const CacheView view = make_view(p, const_cast<void*>(K), const_cast<void*>(V), const_cast<int32_t*>(counts), n_max);

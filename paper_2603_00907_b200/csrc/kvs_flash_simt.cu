@@ -175,6 +175,11 @@ combine_partials(const CombineArgs a, const RoundTable tab) {
     if (a.lse_out) a.lse_out[row] = lse;
   }
   if (a.o) a.o[row * KVS_D + d] = od;
+  if (a.o_hi) {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(od);
+    a.o_hi[row * KVS_D + d] = hi;
+    a.o_lo[row * KVS_D + d] = __float2bfloat16_rn(od - __bfloat162float(hi));
+  }
   if (a.o_out) a.o_out[row * KVS_D + d] = od;
   if (a.out_bf16) a.out_bf16[row * KVS_D + d] = __float2bfloat16_rn(od);
 }

@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of libkvs.so.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -67,6 +68,8 @@ struct CombineArgs {
   const float* part_o;
   float4* qstat;           // [U, M]: (max log2, Z, |o|^2, lse natural)
   float* o;                // [U, M, 128] fp32 (may be NULL)
+  __nv_bfloat16* o_hi;     // [U, M, 128]: o = o_hi + o_lo to ~2^-17 relative (may be NULL)
+  __nv_bfloat16* o_lo;
   __nv_bfloat16* out_bf16; // decode: [B, Hq, n_new, 128] == [U, M, 128] (may be NULL)
   float* lse_out;          // optional [U, M]
   float* o_out;            // optional diagnostic copy [U, M, 128]
@@ -88,6 +91,27 @@ struct StatsArgs {
   float* N1;
   float* N12;              // [U, pair_stride]
   float* cosv;
+};
+
+struct StatsTcArgs {
+  int32_t Hkv, M, nqblk, splits, tiles_per_split;
+  int32_t n_max, pair_stride, counter_stride;
+  float scale_log2;
+  int32_t score_mode;
+  const int32_t* counts;   // [U, n_max]
+  const float4* qstat;     // [U, M]: (max log2, Z, |o|^2, lse)
+  float* score;            // [U, pair_stride]
+  float* w;
+  float* A;                // optional diagnostics [U, n_max]
+  float* N1;
+  float* N12;              // optional [U, pair_stride]
+  float* cosv;
+  float* partA;            // [U, nqblk, n_max] per-query-block partial sums
+  float* partN1;
+  float* partN12;          // [U, nqblk, pair_stride]
+  float* partCos;          // [U, pair_stride]
+  uint32_t* tile_counter;  // [U, counter_stride]; multiples of nqblk between launches
+  int32_t* status_dev;
 };
 
 struct SelectArgs {
@@ -118,6 +142,9 @@ struct CompactArgs {
 cudaError_t kvs_launch_flash_simt(const FlashArgs& a, const RoundTable& t, cudaStream_t st);
 cudaError_t kvs_launch_combine(const CombineArgs& a, const RoundTable& t, cudaStream_t st);
 cudaError_t kvs_launch_stats_simt(const StatsArgs& a, const RoundTable& t, cudaStream_t st);
+cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const CUtensorMap& tmK,
+                                const CUtensorMap& tmV, const CUtensorMap& tmQ, const CUtensorMap& tmOhi,
+                                const CUtensorMap& tmOlo, cudaStream_t st);
 cudaError_t kvs_launch_select(const SelectArgs& a, const RoundTable& t, cudaStream_t st);
 cudaError_t kvs_launch_compact(const CompactArgs& a, const RoundTable& t, cudaStream_t st);
 

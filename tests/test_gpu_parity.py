@@ -99,6 +99,16 @@ def test_window_stats_round0(kb):
     _check_round_stats(kb, w, data["K"], data["V"], data["counts"], data["q_win"], list(w.seq_lens), 0)
 
 
+def test_window_stats_several_query_blocks(kb):
+    """group * window = 160 and 288 rows: two and three query blocks, the last one partial."""
+    for seed, win, heads in ((8, 40, 8), (9, 72, 8)):
+        w = _small(seed=seed, batch=1, n_q_heads=heads, n_kv_heads=2, window=win, seq_lens=(900,),
+                   budgets=(300,))
+        data = wl.make_layer(w)
+        _check_round_stats(kb, w, data["K"], data["V"], data["counts"], data["q_win"], list(w.seq_lens), 0)
+        _check_round_stats(kb, w, data["K"], data["V"], data["counts"], data["q_win"], list(w.seq_lens), 1)
+
+
 def test_window_stats_modes(kb):
     w = _small(seed=2, seq_lens=(260, 131), budgets=(90, 60))
     data = wl.make_layer(w)
