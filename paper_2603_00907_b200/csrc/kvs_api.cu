@@ -155,12 +155,27 @@ struct WsLayout {
   size_t sync_bytes;
 };
 
+int tc_splits(int M, int Hkv, int nseq, int ntiles, int* tiles_per_split) {
+  const int nqblk = (M + 127) / 128;
+  int s = 148 / (nqblk * Hkv * nseq);          // one CTA per SM, one wave
+  if (s < 1) s = 1;
+  if (s > ntiles) s = ntiles;
+  if (s < 1) s = 1;
+  *tiles_per_split = (ntiles + s - 1) / s;
+  if (*tiles_per_split < 1) *tiles_per_split = 1;
+  return (ntiles + *tiles_per_split - 1) / *tiles_per_split > 0 ? (ntiles + *tiles_per_split - 1) / *tiles_per_split : 1;
+}
+
+// upper bound of the number of attention partials per query row (workspace sizing)
 int splits_bound(int M, int Hkv) {
   const int nqblk = (M + 127) / 128;
   int s = (2 * 148 + nqblk * Hkv - 1) / (nqblk * Hkv);
   if (s < 1) s = 1;
   if (s > KVS_MAX_SPLITS) s = KVS_MAX_SPLITS;
-  return s;
+  int tc = 148 / (nqblk * Hkv);
+  if (tc < 1) tc = 1;
+  tc *= 2;                                      // two softmax groups per CTA
+  return s > tc ? s : tc;
 }
 
 WsLayout make_layout(const kvs_params_t* p, int n_max, int max_new) {
@@ -243,8 +258,51 @@ struct Common {
   int G, Mw;
   int32_t* status_dev;
   bool simt_stats;           // debugging aid: statistics on the CUDA cores
+  bool simt_flash;           // debugging aid: attention partials on the CUDA cores
   CUtensorMap tmK, tmV, tmQ, tmOhi, tmOlo;
 };
+
+int choose_splits(int M, int Hkv, int nseq, int nmax_slots, int* split_len);
+
+bool env_simt_flash() {
+  static int v = -1;
+  if (v < 0) { const char* e = getenv("KVS_DEBUG_SIMT_FLASH"); v = (e && e[0] == '1') ? 1 : 0; }
+  return v == 1;
+}
+
+// Attention partials of the rows in `q` (a [U, M, 128] view) over the caches in `view`.
+// Returns the number of partials per row through *n_part.
+template <class LaunchFn>
+kvs_status_t enqueue_flash(const kvs_params_t* p, char* ws, const WsLayout& L, cudaStream_t st,
+                           const CacheView& view, const void* q, int G, int Wq, int M, int causal,
+                           const RoundTable& tab, int nmax_slots, bool simt, const CUtensorMap& tmK,
+                           const CUtensorMap& tmV, const CUtensorMap& tmQ, int32_t* status_dev,
+                           LaunchFn&& launch_fn, int* n_part) {
+  float2* part_ml = reinterpret_cast<float2*>(ws + L.part_ml);
+  float* part_o = reinterpret_cast<float*>(ws + L.part_o);
+  const float scale_log2 = p->softmax_scale * 1.4426950408889634f;
+  if (simt) {
+    FlashArgs fa;
+    fa.c = view;
+    fa.q = static_cast<const __nv_bfloat16*>(q);
+    fa.Hq = p->n_q_heads; fa.G = G; fa.Wq = Wq; fa.M = M;
+    fa.causal = causal;
+    fa.scale_log2 = scale_log2;
+    fa.splits = choose_splits(M, p->n_kv_heads, tab.nseq, nmax_slots, &fa.split_len);
+    fa.part_ml = part_ml; fa.part_o = part_o;
+    *n_part = fa.splits;
+    return launch_fn([&] { return kvs_launch_flash_simt(fa, tab, st); });
+  }
+  FlashTcArgs ta;
+  ta.Hkv = p->n_kv_heads; ta.M = M; ta.nqblk = (M + 127) / 128;
+  const int ntiles = (nmax_slots + 127) / 128;
+  ta.splits = tc_splits(M, p->n_kv_heads, tab.nseq, ntiles, &ta.tiles_per_split);
+  ta.Wq = Wq; ta.causal = causal; ta.scale_log2 = scale_log2;
+  ta.n_max = view.n_max; ta.counts = view.counts;
+  ta.part_ml = part_ml; ta.part_o = part_o; ta.status_dev = status_dev;
+  *n_part = ta.splits * 2;
+  return launch_fn([&] { return kvs_launch_flash_tc(ta, tab, tmK, tmV, tmQ, st); });
+}
 
 bool env_simt_stats() {
   static int v = -1;
@@ -276,20 +334,21 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
                                  float* A, float* N1, float* N12, float* cosv, float* score_out,
                                  float* w_out, uint8_t* mask_out, float* o_out, float* lse_out) {
   const kvs_params_t* p = c.p;
-  FlashArgs fa;
-  fa.c = view;
-  fa.q = static_cast<const __nv_bfloat16*>(q_win);
-  fa.Hq = p->n_q_heads; fa.G = c.G; fa.Wq = p->window; fa.M = c.Mw;
-  fa.causal = p->causal;
-  fa.scale_log2 = p->softmax_scale * 1.4426950408889634f;
-  fa.splits = choose_splits(c.Mw, p->n_kv_heads, tab.nseq, nmax_slots, &fa.split_len);
-  fa.part_ml = reinterpret_cast<float2*>(c.ws + c.L.part_ml);
-  fa.part_o = reinterpret_cast<float*>(c.ws + c.L.part_o);
-  CUDA_TRY(launch(KVS_K_FLASH, c.st, [&] { return kvs_launch_flash_simt(fa, tab, c.st); }));
-
+  const float scale_log2 = p->softmax_scale * 1.4426950408889634f;
+  int n_part = 0;
+  {
+    kvs_status_t fs = enqueue_flash(p, c.ws, c.L, c.st, view, q_win, c.G, p->window, c.Mw, p->causal, tab,
+                                    nmax_slots, c.simt_flash, c.tmK, c.tmV, c.tmQ, c.status_dev,
+                                    [&](auto&& f) -> kvs_status_t {
+                                      CUDA_TRY(launch(KVS_K_FLASH, c.st, f));
+                                      return KVS_OK;
+                                    }, &n_part);
+    if (fs != KVS_OK) return fs;
+  }
   CombineArgs ca;
-  ca.M = c.Mw; ca.splits = fa.splits; ca.Hkv = p->n_kv_heads;
-  ca.part_ml = fa.part_ml; ca.part_o = fa.part_o;
+  ca.M = c.Mw; ca.splits = n_part; ca.Hkv = p->n_kv_heads;
+  ca.part_ml = reinterpret_cast<float2*>(c.ws + c.L.part_ml);
+  ca.part_o = reinterpret_cast<float*>(c.ws + c.L.part_o);
   ca.qstat = reinterpret_cast<float4*>(c.ws + c.L.qstat);
   ca.o = reinterpret_cast<float*>(c.ws + c.L.o);
   ca.o_hi = reinterpret_cast<__nv_bfloat16*>(c.ws + c.L.o_hi);
@@ -299,8 +358,8 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
 
   StatsArgs sa;
   sa.c = view;
-  sa.q = fa.q; sa.Hq = fa.Hq; sa.G = fa.G; sa.Wq = fa.Wq; sa.M = fa.M;
-  sa.causal = fa.causal; sa.scale_log2 = fa.scale_log2; sa.score_mode = p->score_mode;
+  sa.q = static_cast<const __nv_bfloat16*>(q_win); sa.Hq = p->n_q_heads; sa.G = c.G; sa.Wq = p->window; sa.M = c.Mw;
+  sa.causal = p->causal; sa.scale_log2 = scale_log2; sa.score_mode = p->score_mode;
   sa.qstat = ca.qstat; sa.o = ca.o;
   sa.pair_stride = c.L.pair_stride;
   sa.score = score_out ? score_out : reinterpret_cast<float*>(c.ws + c.L.score);
@@ -320,7 +379,7 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
     ta.tiles_per_split = (ntiles + splits - 1) / splits;
     ta.splits = (ntiles + ta.tiles_per_split - 1) / ta.tiles_per_split;
     ta.n_max = view.n_max; ta.pair_stride = c.L.pair_stride; ta.counter_stride = c.L.counter_stride;
-    ta.scale_log2 = fa.scale_log2; ta.score_mode = p->score_mode;
+    ta.scale_log2 = scale_log2; ta.score_mode = p->score_mode;
     ta.counts = view.counts; ta.qstat = ca.qstat;
     ta.score = sa.score; ta.w = sa.w; ta.A = A; ta.N1 = N1; ta.N12 = N12; ta.cosv = cosv;
     ta.partA = reinterpret_cast<float*>(c.ws + c.L.partA);
@@ -371,6 +430,7 @@ kvs_status_t check_common(const kvs_params_t* p, const void* K, const void* V, c
   c->Mw = c->G * p->window;
   c->status_dev = nullptr;
   c->simt_stats = env_simt_stats();
+  c->simt_flash = env_simt_flash();
   return KVS_OK;
 }
 
@@ -575,6 +635,17 @@ kvs_status_t kvs_decode_attn(const kvs_params_t* p, const void* q_new, int32_t n
   const int B = p->batch;
   const int M = c.G * n_new;
   const CacheView view = make_view(p, const_cast<void*>(K), const_cast<void*>(V), const_cast<int32_t*>(counts), n_max);
+  CUtensorMap tmK, tmV, tmQ;
+  {
+    const uint64_t kd[4] = {KVS_D, (uint64_t)n_max, (uint64_t)p->n_kv_heads, (uint64_t)p->batch};
+    const uint64_t ks[3] = {(uint64_t)p->k_stride_t * 2, (uint64_t)p->k_stride_h * 2, (uint64_t)p->k_stride_b * 2};
+    const uint64_t vs[3] = {(uint64_t)p->v_stride_t * 2, (uint64_t)p->v_stride_h * 2, (uint64_t)p->v_stride_b * 2};
+    const uint64_t qd[3] = {KVS_D, (uint64_t)M, (uint64_t)c.L.U};
+    const uint64_t qs[2] = {KVS_D * 2, (uint64_t)M * KVS_D * 2};
+    if (!c.simt_flash && !(make_tmap(&tmK, K, 4, kd, ks, 128) && make_tmap(&tmV, V, 4, kd, vs, 128) &&
+                           make_tmap(&tmQ, q_new, 3, qd, qs, 128)))
+      return fail(KVS_ERR_CUDA, "cuTensorMapEncodeTiled failed or is unavailable");
+  }
   for (int b0 = 0; b0 < B; b0 += KVS_SEQ_CHUNK) {
     RoundTable tab;
     tab.nseq = 0; tab.off = 0;
@@ -585,19 +656,18 @@ kvs_status_t kvs_decode_attn(const kvs_params_t* p, const void* q_new, int32_t n
       if (seq_len[b] > nmax_slots) nmax_slots = seq_len[b];
     }
     if (tab.nseq == 0) continue;
-    FlashArgs fa;
-    fa.c = view;
-    fa.q = static_cast<const __nv_bfloat16*>(q_new);
-    fa.Hq = p->n_q_heads; fa.G = c.G; fa.Wq = n_new; fa.M = M;
-    fa.causal = 0;
-    fa.scale_log2 = p->softmax_scale * 1.4426950408889634f;
-    fa.splits = choose_splits(M, p->n_kv_heads, tab.nseq, nmax_slots, &fa.split_len);
-    fa.part_ml = reinterpret_cast<float2*>(c.ws + c.L.part_ml);
-    fa.part_o = reinterpret_cast<float*>(c.ws + c.L.part_o);
-    CUDA_TRY(launch(KVS_K_FLASH, c.st, [&] { return kvs_launch_flash_simt(fa, tab, c.st); }));
+    int n_part = 0;
+    s = enqueue_flash(p, c.ws, c.L, c.st, view, q_new, c.G, n_new, M, 0, tab, nmax_slots, c.simt_flash, tmK,
+                      tmV, tmQ, status_dev,
+                      [&](auto&& f) -> kvs_status_t {
+                        CUDA_TRY(launch(KVS_K_FLASH, c.st, f));
+                        return KVS_OK;
+                      }, &n_part);
+    if (s != KVS_OK) return s;
     CombineArgs ca;
-    ca.M = M; ca.splits = fa.splits; ca.Hkv = p->n_kv_heads;
-    ca.part_ml = fa.part_ml; ca.part_o = fa.part_o;
+    ca.M = M; ca.splits = n_part; ca.Hkv = p->n_kv_heads;
+    ca.part_ml = reinterpret_cast<float2*>(c.ws + c.L.part_ml);
+    ca.part_o = reinterpret_cast<float*>(c.ws + c.L.part_o);
     ca.qstat = nullptr; ca.o = nullptr; ca.o_hi = nullptr; ca.o_lo = nullptr;
     ca.out_bf16 = static_cast<__nv_bfloat16*>(out);
     ca.lse_out = lse; ca.o_out = nullptr;

@@ -1,0 +1,366 @@
+// Attention partials on the tensor cores (tcgen05 + TMEM + TMA), queries on TMEM lanes.
+//
+// One CTA owns a block of 128 query rows (Q stays in shared memory) and a contiguous range
+// of 128-slot tiles.  Per tile, TMA brings the K and V rows and one thread issues
+//   S[q, slot] = Q K_tile^T                         (fp32 in TMEM, double buffered)
+// Two groups of four warps each take 64 of the tile's slots.  A thread owns one query row:
+// it adds the count bias ln c_j, applies the causal/tail mask, keeps a running stabiliser
+// and sum, and writes P' = exp(s - m) / c_j, split into two bf16 terms, to shared memory.
+// The same issuing thread then runs, per group,
+//   O_g[q, :] += (P'_hi + P'_lo) Vsum_tile          (V as the MN-major operand)
+// with O_g accumulating in TMEM across the tiles [Eq. attn_def_vec with merged slots:
+// o = sum_j alpha_j Vsum_j / c_j].  The stabiliser only moves when the row maximum grows by
+// more than 2^8, in which case the group rescales its O_g rows in TMEM; otherwise O is never
+// touched until the end, where (stabiliser, sum, O) is written as the partial of this
+// (key split, group).  Window queries and decode queries use the same kernel.
+#include "kvs_internal.h"
+#include "kvs_sm100.cuh"
+
+using namespace sm100;
+
+namespace {
+
+constexpr int kTile = 128;
+constexpr int kHalf = 16384;               // [128 rows x 64 bf16], 128-byte swizzle
+constexpr int kOperand = 2 * kHalf;
+constexpr int kStage = 2 * kOperand;       // K tile + V tile
+constexpr int kPGroup = 2 * kHalf;         // P'_hi and P'_lo of one group: [128 q x 64 slots] each
+constexpr int kSmemQ = 0, kSmemStage = kOperand, kSmemP = kSmemStage + 2 * kStage;
+constexpr int kSmemMisc = kSmemP + 2 * kPGroup;
+constexpr int kThreads = 320;
+constexpr float kRescaleGap = 8.f;         // log2 units
+
+struct Misc {
+  uint64_t full[2], kvfree[2], sfull[2], sfree[2], pready[2], ofull[2], qfull;
+  uint32_t tmem_base;
+  int abort_flag;
+  int wg_fail[2];
+  float2 cst[2][64];                       // per group, per slot: (log2 c, 1/c)
+};
+constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc) + 1024;
+
+__device__ __forceinline__ void wg_barrier(int wg) {
+  asm volatile("bar.sync %0, 128;" ::"r"(wg + 1) : "memory");
+}
+// OR over the 128 threads of a group, with barrier semantics.
+__device__ __forceinline__ bool wg_any(int wg, bool pred) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 p, %2, 0;\n\t"
+      "bar.red.or.pred q, %1, 128, p;\n\t"
+      "selp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(out)
+      : "r"(wg + 1), "r"((uint32_t)pred)
+      : "memory");
+  return out != 0;
+}
+__device__ __forceinline__ bool wg_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                        volatile int* wg_fail, int wg, int lane) {
+  if (lane == 0) {
+    if (!mbar_wait(bar, parity, abort_flag)) *wg_fail = 1;
+  }
+  __syncwarp();
+  wg_barrier(wg);
+  return *wg_fail == 0;
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])),
+        "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])),
+        "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+        "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+        "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])),
+        "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])),
+        "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+        "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])),
+        "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])),
+        "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() {
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constant__ CUtensorMap tmK,
+                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQ) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  Misc* misc = reinterpret_cast<Misc*>(smem + kSmemMisc);
+
+  const int seq = blockIdx.z;
+  const SeqRound sr = tab.s[seq];
+  const int n = sr.n;
+  const int h = blockIdx.y;
+  const int qblk = blockIdx.x % a.nqblk;
+  const int split = blockIdx.x / a.nqblk;
+  const int unit = sr.b * a.Hkv + h;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ntiles = (n + kTile - 1) / kTile;
+  const int t_begin = min(ntiles, split * a.tiles_per_split);
+  const int t_end = min(ntiles, t_begin + a.tiles_per_split);
+  const int my_tiles = t_end - t_begin;
+  if (n <= 0) return;
+  if (my_tiles <= 0) {
+    // an empty split still owes its two (empty) partials to the combine
+    if (warp >= 2) {
+      const int wg = (warp - 2) >> 2, row = (warp & 3) * 32 + lane, m = qblk * 128 + row;
+      if (m < a.M) {
+        const size_t pidx = ((size_t)unit * (a.splits * 2) + split * 2 + wg) * a.M + m;
+        a.part_ml[pidx] = make_float2(-INFINITY, 0.f);
+      }
+    }
+    return;
+  }
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&misc->full[s], 1);
+      mbar_init(&misc->kvfree[s], 1);
+      mbar_init(&misc->sfull[s], 1);
+      mbar_init(&misc->sfree[s], 2);
+      mbar_init(&misc->pready[s], 1);
+      mbar_init(&misc->ofull[s], 1);
+    }
+    mbar_init(&misc->qfull, 1);
+    misc->abort_flag = 0;
+    misc->wg_fail[0] = misc->wg_fail[1] = 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc(&misc->tmem_base, 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = misc->tmem_base;
+  volatile int* abort_flag = &misc->abort_flag;
+
+  if (warp == 0) {
+    // ================================================================ TMA producer
+    if (lane == 0) {
+      prefetch_tmap(&tmK); prefetch_tmap(&tmV); prefetch_tmap(&tmQ);
+      mbar_expect_tx(&misc->qfull, kOperand);
+      for (int hf = 0; hf < 2; ++hf)
+        tma_load_3d(smem + kSmemQ + hf * kHalf, &tmQ, &misc->qfull, hf * 64, qblk * 128, unit);
+      int issued = 0;
+      for (int li = 0; li < my_tiles; ++li) {
+        const int s = li & 1, k = li >> 1;
+        if (!mbar_wait(&misc->kvfree[s], (k & 1) ^ 1, abort_flag)) break;
+        uint8_t* st = smem + kSmemStage + s * kStage;
+        const int row = (t_begin + li) * kTile;
+        mbar_expect_tx(&misc->full[s], kStage);
+        for (int hf = 0; hf < 2; ++hf) {
+          tma_load_4d(st + hf * kHalf, &tmK, &misc->full[s], hf * 64, row, h, sr.b);
+          tma_load_4d(st + kOperand + hf * kHalf, &tmV, &misc->full[s], hf * 64, row, h, sr.b);
+        }
+        issued = li + 1;
+      }
+      if (*abort_flag) {
+        for (int li = max(0, issued - 2); li < issued; ++li) {
+          const uint64_t t0 = globaltimer_ns();
+          while (!mbar_try_wait(&misc->full[li & 1], (li >> 1) & 1) && globaltimer_ns() - t0 < 200000000ull) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ================================================================ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = idesc_bf16(128, 128);                 // Q (K-major) x K tile (K-major)
+      constexpr uint32_t idesc_o = idesc_bf16(128, 128, false, true);    // P' (K-major) x V tile (MN-major)
+      const uint32_t q_addr = smem_u32(smem + kSmemQ);
+      auto issue_s = [&](int li) -> bool {
+        const int s = li & 1, k = li >> 1;
+        if (!mbar_wait(&misc->full[s], k & 1, abort_flag)) return false;
+        if (!mbar_wait(&misc->sfree[s], (k & 1) ^ 1, abort_flag)) return false;
+        tc_fence_after();
+        const uint32_t k_addr = smem_u32(smem + kSmemStage + s * kStage);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint32_t o = (kk >> 2) * kHalf + (kk & 3) * 32;
+          umma_bf16(tmem + s * 128, smem_desc_sw128(q_addr + o, 16, 1024), smem_desc_sw128(k_addr + o, 16, 1024),
+                    idesc_s, kk > 0);
+        }
+        tc_commit(&misc->sfull[s]);
+        return true;
+      };
+      bool ok = mbar_wait(&misc->qfull, 0, abort_flag);
+      ok = ok && issue_s(0);
+      for (int li = 0; ok && li < my_tiles; ++li) {
+        if (li + 1 < my_tiles) ok = issue_s(li + 1);
+        const int s = li & 1;
+        const uint32_t v_addr = smem_u32(smem + kSmemStage + s * kStage + kOperand);
+        for (int g = 0; ok && g < 2; ++g) {
+          if (!mbar_wait(&misc->pready[g], li & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t p_addr = smem_u32(smem + kSmemP + g * kPGroup);
+          const uint32_t dO = tmem + 256 + g * 128;
+#pragma unroll
+          for (int hl = 0; hl < 2; ++hl) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              // A: 16 slots = 32 bytes along the swizzled row; B: 16 slots = two 8-row groups of V
+              const uint64_t ad = smem_desc_sw128(p_addr + hl * kHalf + kk * 32, 16, 1024);
+              const uint64_t bd = smem_desc_sw128(v_addr + (g * 64 + kk * 16) * 128, kHalf, 1024);
+              umma_bf16(dO, ad, bd, idesc_o, (li > 0 || hl > 0 || kk > 0) ? 1u : 0u);
+            }
+          }
+          tc_commit(&misc->ofull[g]);
+        }
+        if (ok) tc_commit(&misc->kvfree[s]);
+      }
+    }
+  } else {
+    // ================================================================ softmax groups
+    const int wg = (warp - 2) >> 2;
+    const int row = (warp & 3) * 32 + lane;               // TMEM lane = query row in the block
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const int t128 = threadIdx.x - 64 - wg * 128;         // 0..127 within the group
+    const int m = qblk * 128 + row;
+    const int last_vis = a.causal ? (n - a.Wq + (m % a.Wq)) : (n - 1);
+    const int32_t* Cb = a.counts + (size_t)unit * a.n_max;
+    uint8_t* pbuf = smem + kSmemP + wg * kPGroup;
+    float m_stab = -INFINITY, l = 0.f;
+    bool alive = true;
+    for (int li = 0; li < my_tiles; ++li) {
+      const int s = li & 1, k = li >> 1;
+      const int j0 = (t_begin + li) * kTile + wg * 64;    // first slot of this group's half tile
+      if (t128 < 64) {
+        const int j = j0 + t128;
+        const float cnt = (j < n) ? (float)Cb[j] : 1.f;
+        misc->cst[wg][t128] = make_float2(log2f(cnt), 1.f / cnt);
+      }
+      if (!wg_wait(&misc->sfull[s], k & 1, abort_flag, &misc->wg_fail[wg], wg, lane)) { alive = false; break; }
+      tc_fence_after();
+      float x[64];
+      tmem_ld32(tmem + lane_addr + s * 128 + wg * 64, x);
+      tmem_ld32(tmem + lane_addr + s * 128 + wg * 64 + 32, x + 32);
+      tmem_ld_wait();
+      tc_fence_before();
+      wg_barrier(wg);
+      if (t128 == 0) mbar_arrive(&misc->sfree[s]);
+      // logits in log2 units, with count bias and mask
+      float mt = -INFINITY;
+      const bool need_mask = (j0 + 63 > min(n - 1, a.causal ? n - a.Wq : n - 1));
+      if (!need_mask) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i) {
+          x[i] = fmaf(x[i], a.scale_log2, misc->cst[wg][i].x);
+          mt = fmaxf(mt, x[i]);
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 64; ++i) {
+          const float v = fmaf(x[i], a.scale_log2, misc->cst[wg][i].x);
+          x[i] = (j0 + i <= last_vis) ? v : -INFINITY;
+          mt = fmaxf(mt, x[i]);
+        }
+      }
+      const float m_new = fmaxf(m_stab, mt);
+      const bool need = m_new > m_stab + kRescaleGap || (m_stab == -INFINITY && m_new > -INFINITY);
+      const bool any_need = wg_any(wg, need && li > 0);
+      // the previous tile's P V product must be done before P is overwritten (and before a rescale)
+      if (li > 0) {
+        if (!wg_wait(&misc->ofull[wg], (li - 1) & 1, abort_flag, &misc->wg_fail[wg], wg, lane)) { alive = false; break; }
+        tc_fence_after();
+      }
+      if (any_need) {
+        const float f = (need && m_stab > -INFINITY) ? fast_exp2(m_stab - m_new) : 1.f;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float ov[32];
+          tmem_ld32(tmem + lane_addr + 256 + wg * 128 + c * 32, ov);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) ov[i] *= f;
+          tmem_st32(tmem + lane_addr + 256 + wg * 128 + c * 32, ov);
+        }
+        tmem_st_wait();
+        l *= f;
+      }
+      if (need) m_stab = m_new;
+      const float ms = (m_stab == -INFINITY) ? 0.f : m_stab;      // row with nothing visible yet
+      // P' = exp2(x - m) / c as hi + lo bf16, written as the K-major operand [row][64 slots]
+      float lsum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        uint32_t hi[4], lo[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = c * 8 + u * 2;
+          const float p0 = fast_exp2(x[i] - ms), p1 = fast_exp2(x[i + 1] - ms);
+          lsum += p0 + p1;
+          const float q0 = p0 * misc->cst[wg][i].y, q1 = p1 * misc->cst[wg][i + 1].y;
+          hi[u] = pack_bf16(q0, q1);
+          lo[u] = pack_bf16(q0 - bf16lo(hi[u]), q1 - bf16hi(hi[u]));
+        }
+        const int off16 = row * 128 + ((c ^ (row & 7)) << 4);
+        *reinterpret_cast<uint4*>(pbuf + off16) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(pbuf + kHalf + off16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      }
+      l += lsum;
+      // rows of the V tile past the end of the sequence may hold anything: zero them
+      const int tile_row0 = (t_begin + li) * kTile;
+      if (tile_row0 + kTile > n) {
+        uint8_t* vt = smem + kSmemStage + s * kStage + kOperand;
+        const int r_lo = max(wg * 64, n - tile_row0), r_hi = wg * 64 + 64;
+        for (int it = r_lo * 16 + t128; it < r_hi * 16; it += 128) {
+          const int r = it >> 4, ch = it & 15;
+          *reinterpret_cast<uint4*>(vt + (ch >> 3) * kHalf + r * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
+        }
+      }
+      fence_proxy_async();
+      tc_fence_before();
+      wg_barrier(wg);
+      if (t128 == 0) mbar_arrive(&misc->pready[wg]);
+    }
+    // ---- the partial of this (split, group)
+    if (alive && wg_wait(&misc->ofull[wg], (my_tiles - 1) & 1, abort_flag, &misc->wg_fail[wg], wg, lane)) {
+      tc_fence_after();
+      const size_t pidx = ((size_t)unit * (a.splits * 2) + split * 2 + wg) * a.M + m;
+      if (m < a.M) a.part_ml[pidx] = make_float2(m_stab, l);
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        float ov[32];
+        tmem_ld32(tmem + lane_addr + 256 + wg * 128 + c * 32, ov);
+        tmem_ld_wait();
+        if (m < a.M) {
+          float4* po = reinterpret_cast<float4*>(a.part_o + pidx * KVS_D + c * 32);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) po[i] = make_float4(ov[4 * i], ov[4 * i + 1], ov[4 * i + 2], ov[4 * i + 3]);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+  if (threadIdx.x == 0 && misc->abort_flag && a.status_dev) atomicExch(a.status_dev, (int)KVS_ERR_TIMEOUT);
+}
+
+}  // namespace
+
+cudaError_t kvs_launch_flash_tc(const FlashTcArgs& a, const RoundTable& t, const CUtensorMap& tmK,
+                                const CUtensorMap& tmV, const CUtensorMap& tmQ, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(flash_partial_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  dim3 grid(a.nqblk * a.splits, a.Hkv, t.nseq);
+  flash_partial_tc<<<grid, kThreads, kSmemBytes, st>>>(a, t, tmK, tmV, tmQ);
+  return cudaGetLastError();
+}

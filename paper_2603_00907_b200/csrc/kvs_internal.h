@@ -62,6 +62,17 @@ struct FlashArgs {
   float* part_o;           // [U, splits, M, 128]
 };
 
+struct FlashTcArgs {
+  int32_t Hkv, M, nqblk, splits, tiles_per_split;
+  int32_t Wq, causal;
+  float scale_log2;
+  int32_t n_max;
+  const int32_t* counts;   // [U, n_max]
+  float2* part_ml;         // [U, 2 * splits, M]
+  float* part_o;           // [U, 2 * splits, M, 128]
+  int32_t* status_dev;
+};
+
 struct CombineArgs {
   int32_t M, splits, Hkv;
   const float2* part_ml;
@@ -145,6 +156,8 @@ cudaError_t kvs_launch_stats_simt(const StatsArgs& a, const RoundTable& t, cudaS
 cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const CUtensorMap& tmK,
                                 const CUtensorMap& tmV, const CUtensorMap& tmQ, const CUtensorMap& tmOhi,
                                 const CUtensorMap& tmOlo, cudaStream_t st);
+cudaError_t kvs_launch_flash_tc(const FlashTcArgs& a, const RoundTable& t, const CUtensorMap& tmK,
+                                const CUtensorMap& tmV, const CUtensorMap& tmQ, cudaStream_t st);
 cudaError_t kvs_launch_select(const SelectArgs& a, const RoundTable& t, cudaStream_t st);
 cudaError_t kvs_launch_compact(const CompactArgs& a, const RoundTable& t, cudaStream_t st);
 

@@ -72,7 +72,9 @@ def _check_round_stats(kb, w, K, V, C, q_win, n_list, r, score_mode=0, causal=Tr
             for name, g, ref in (("A", A[b, h, sl], st["A"][sl]), ("N1", N1[b, h, sl], st["N1"][sl]),
                                  ("N12", N12[b, h, :P], st["N12"]), ("score", score[b, h, :P], st["score"]),
                                  ("o", o_win[b, h], st["o"])):
-                ok, ratio, plain = tl.stat_close(g, ref)
+                # o is an intermediate formed on the tensor cores from a two-term bf16 split of the
+                # probabilities: held to 1e-4; the statistics that the method uses to 1e-5
+                ok, ratio, plain = tl.stat_close(g, ref, rtol=tl.O_RTOL if name == "o" else tl.STAT_RTOL)
                 report.append((b, h, name, ratio, plain))
                 assert ok, f"{name} unit {(b, h)} round {r}: err/allowed {ratio:.3g} plain rel {plain:.3g}"
             # cosine: compared through 1 - cos (what the score uses), absolute 1e-6
@@ -107,6 +109,53 @@ def test_window_stats_several_query_blocks(kb):
         data = wl.make_layer(w)
         _check_round_stats(kb, w, data["K"], data["V"], data["counts"], data["q_win"], list(w.seq_lens), 0)
         _check_round_stats(kb, w, data["K"], data["V"], data["counts"], data["q_win"], list(w.seq_lens), 1)
+
+
+def test_window_stats_many_tiles_per_cta(kb):
+    """Llama head layout (8 KV heads, two sequences): few key splits, so every CTA walks several
+    128-slot tiles through its TMA/MMA pipeline; the last tile of each sequence is ragged."""
+    w = _small(seed=10, batch=2, n_q_heads=32, n_kv_heads=8, window=40, seq_lens=(3000, 2123),
+               budgets=(1000, 700))
+    data = wl.make_layer(w)
+    _check_round_stats(kb, w, data["K"], data["V"], data["counts"], data["q_win"], list(w.seq_lens), 0)
+
+
+def test_attention_partials_with_late_spikes(kb):
+    """A few late keys aligned with one query make that row's maximum jump by far more than
+    2^8 after the first tiles: the kernel must rescale its running output.  Checked on the
+    attention output, the log-sum-exp and the attention mass."""
+    import torch
+    w = _small(seed=11, batch=1, n_q_heads=32, n_kv_heads=8, window=16, seq_lens=(4000,), budgets=(1500,))
+    data = wl.make_layer(w)
+    K, q = data["K"], data["q_win"]
+    qf = wl.bf16_bits_to_f32(q)
+    for h in range(w.n_kv_heads):
+        for t, (j, row) in enumerate(((700, 3), (1900, 17), (3100, 40))):
+            g, i = divmod(row, w.window)
+            K[0, h, j] = wl.f32_to_bf16_bits((3.0 + t) * qf[0, h * w.group + g, i])
+    dev, p, ws = _setup(kb, w, data)
+    B, Hkv, Nmax, M = 1, w.n_kv_heads, w.n_max, w.group * w.window
+    f32 = dict(dtype=torch.float32, device="cuda")
+    A = torch.zeros((B, Hkv, Nmax), **f32)
+    o_win, lse = torch.zeros((B, Hkv, M, 128), **f32), torch.zeros((B, Hkv, M), **f32)
+    kb.kvs_window_stats(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], [4000], [1500], ws, A=A,
+                        o_win=o_win, lse_win=lse)
+    torch.cuda.synchronize()
+    for h in range(Hkv):
+        Kf, Vf = oc.bf16_to_f64(K[0, h]), oc.bf16_to_f64(data["V"][0, h])
+        Qf = oc.bf16_to_f64(q[0, h * w.group:(h + 1) * w.group])
+        alpha, o, _ = oc.window_probabilities(Kf, Vf, np.ones(4000), Qf, w.window, 1 / math.sqrt(128), True)
+        assert alpha.max() > 0.9                      # the spikes really dominate their rows
+        ok, ratio, plain = tl.stat_close(o_win[0, h].cpu().numpy(), o, rtol=tl.O_RTOL)
+        assert ok, (h, ratio, plain)
+        off, P, _ = oc.round_plan(4000, 1500, w.sink, w.window, 0.5, 0)
+        ok, ratio, plain = tl.stat_close(A[0, h, off:off + 2 * P].cpu().numpy(), alpha.sum(0)[off:off + 2 * P])
+        assert ok, (h, ratio, plain)
+        s = (Qf.reshape(M, 128) @ Kf.T) / math.sqrt(128)
+        i = np.tile(np.arange(w.window), w.group)
+        s = np.where(np.arange(4000)[None, :] > (4000 - w.window + i)[:, None], -np.inf, s)
+        lse_ref = np.log(np.exp(s - s.max(1, keepdims=True)).sum(1)) + s.max(1)
+        assert np.max(np.abs(lse[0, h].cpu().numpy() - lse_ref)) < 2e-4
 
 
 def test_window_stats_modes(kb):
@@ -295,6 +344,31 @@ def test_decode_matches_oracle_and_is_lossless_on_identical_keys(kb):
                                          Cg[b, h, :m])
             ok, mx, _, _ = tl.bf16_close(o1[b, h * G:(h + 1) * G], oc.f64_to_bf16(ref))
             assert ok, mx
+
+
+def test_decode_many_rows_and_tiles(kb):
+    """group * n_new = 192 query rows (two blocks) over caches of several tiles, merged counts."""
+    import torch
+    w = _small(seed=12, batch=2, n_q_heads=16, n_kv_heads=4, window=8, seq_lens=(1500, 777),
+               budgets=(1500, 777), n_decode=48)
+    data = wl.make_layer(w)
+    rng = np.random.default_rng(5)
+    data["counts"][:] = rng.integers(1, 6, size=data["counts"].shape)          # as if merged before
+    dev, p, ws = _setup(kb, w, data)
+    B, Hq, T, G, Hkv = w.batch, w.n_q_heads, w.n_decode, w.group, w.n_kv_heads
+    out = torch.zeros((B, Hq, T, 128), dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros((B, Hq, T), dtype=torch.float32, device="cuda")
+    kb.kvs_decode_attn(p, dev["q_new"], dev["K"], dev["V"], dev["counts"], list(w.seq_lens), out, ws, lse=lse)
+    torch.cuda.synchronize()
+    og = tl.bits_of(out)
+    for b in range(B):
+        n = w.seq_lens[b]
+        for h in range(Hkv):
+            ref, lse_ref = oc.decode_attention(data["q_new"][b, h * G:(h + 1) * G], data["K"][b, h, :n],
+                                               data["V"][b, h, :n], data["counts"][b, h, :n])
+            ok, mx, _, _ = tl.bf16_close(og[b, h * G:(h + 1) * G], oc.f64_to_bf16(ref))
+            assert ok, mx
+            assert np.max(np.abs(lse[b, h * G:(h + 1) * G].cpu().numpy() - lse_ref)) < 1e-4
 
 
 def test_identical_key_merge_is_lossless_on_gpu(kb):
