@@ -46,6 +46,7 @@ class ClockSampler(threading.Thread):
     def __init__(self, index: int):
         super().__init__(daemon=True)
         self.index, self.rows, self.proc = index, [], None
+        self.t_begin = self.t_end = None            # timed region (perf_counter)
 
     def run(self):
         try:
@@ -54,7 +55,7 @@ class ClockSampler(threading.Thread):
                  "--format=csv,noheader,nounits", "-lms", "100"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             for line in self.proc.stdout:
-                self.rows.append([c.strip() for c in line.split(",")])
+                self.rows.append((time.perf_counter(), [c.strip() for c in line.split(",")]))
         except Exception:
             pass
 
@@ -64,7 +65,12 @@ class ClockSampler(threading.Thread):
         self.join(timeout=2)
         sm, mx, reasons = [], 0, set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        inside = [r for t, r in self.rows
+                  if self.t_begin is not None and self.t_begin <= t <= (self.t_end or t)]
+        # a short timed region may fall between two samples: then the samples taken while the
+        # same steps ran as warm-up stand in, and the record says so
+        scope = "timed region" if len(inside) >= 3 else "warm-up and timed region"
+        for r in (inside if len(inside) >= 3 else [r for _, r in self.rows]):
             try:
                 sm.append(float(r[0]))
                 mx = max(mx, float(r[1]))
@@ -74,7 +80,7 @@ class ClockSampler(threading.Thread):
             except Exception:
                 continue
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx or None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "scope": scope}
 
 
 def measured_peaks():
@@ -155,6 +161,23 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
+def max_over_ranks(ms, world, device):
+    """Slowest rank's time: what a multi-GPU step takes."""
+    if world == 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def rank_tokens_per_step(w, n_layers):
+    """Context tokens one rank consumes per step; every rank holds its own batch of sequences
+    (seeds shifted by the rank), so the job total is world times this."""
+    return n_layers * sum(w.seq_lens)
+
+
 def workload_config(w, args):
     return {"workload": f"configs[{w.config_id}] {w.name}", "layers": w.layers, "batch": w.batch,
             "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": 128,
@@ -163,17 +186,23 @@ def workload_config(w, args):
             "decode_new_tokens": w.n_decode or DECODE_TOKENS,
             "l2": "inputs larger than L2 (fresh cache restored from a device master copy before "
                   "every step, outside the timed events)",
+            "calls_per_step": ("one kvs_merge_layer + one kvs_decode_attn per layer"
+                               if args.per_layer_calls else
+                               "one kvs_merge_layer + one kvs_decode_attn over all layers "
+                               "(layers folded into the batch dimension)"),
             "parallelism": f"dp{args.gpus} over sequences, no collective"}
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=1)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (debug)")
+    ap.add_argument("--per-layer-calls", action="store_true",
+                    help="one kvs_merge_layer call per layer instead of one call over all layers")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -225,15 +254,30 @@ def main():
     hResC = pin((L, B, Hkv, bud_max), torch.int32)
     hOut = pin((L, B, Hq, T, 128), torch.int16)
     bf = lambda t: t.view(torch.bfloat16)
-    p = kb.make_params(bf(wK[0]), bf(wV[0]), Hq, W, sink=w.sink, round_frac=w.round_frac)
-    ws = torch.empty(kb.kvs_workspace_size(p, Nmax, T), dtype=torch.uint8, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    seq_len, budget = list(w.seq_lens), list(w.budgets)
+    # Every (layer, sequence) is an independent problem: unless --per-layer-calls is given the
+    # layers are folded into the batch dimension ([L, B, ...] is [L*B, ...] in memory) and one
+    # call per step merges all of them, so that every launch fills the GPU.
+    fold = not args.per_layer_calls
+    if fold:
+        fK, fV, fC = (t.view(L * B, *t.shape[2:]) for t in (wK, wV, wC))
+        fQ, fQn, fOut = (t.view(L * B, *t.shape[2:]) for t in (dQ, dQn, out))
+        p = kb.make_params(bf(fK), bf(fV), Hq, W, sink=w.sink, round_frac=w.round_frac)
+        seq_len, budget = list(w.seq_lens) * L, list(w.budgets) * L
+    else:
+        p = kb.make_params(bf(wK[0]), bf(wV[0]), Hq, W, sink=w.sink, round_frac=w.round_frac)
+        seq_len, budget = list(w.seq_lens), list(w.budgets)
+    ws = torch.empty(kb.kvs_workspace_size(p, Nmax, T), dtype=torch.uint8, device=dev)
 
     def restore():
         wK.copy_(mK); wV.copy_(mV); wC.copy_(mC)
 
     def step():
+        if fold:
+            new_len = kb.kvs_merge_layer(p, bf(fK), bf(fV), fC, bf(fQ), seq_len, budget, ws,
+                                         status_dev=status)
+            kb.kvs_decode_attn(p, bf(fQn), bf(fK), bf(fV), fC, new_len, bf(fOut), ws)
+            return
         for l in range(L):
             new_len = kb.kvs_merge_layer(p, bf(wK[l]), bf(wV[l]), wC[l], bf(dQ[l]), seq_len, budget, ws,
                                          status_dev=status)
@@ -268,29 +312,24 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
-    def max_over_ranks(ms):
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
     # ---- device-resident timing
+    sampler = ClockSampler(local)
+    sampler.start()
     for _ in range(args.warmup):
         restore(); step()
     sync_all()
-    sampler = ClockSampler(local)
-    sampler.start()
     launches0 = kb.kvs_launch_count()
+    sampler.t_begin = time.perf_counter()
     total_ms = timed(step, args.steps, prepare=restore)
     sync_all()
+    sampler.t_end = time.perf_counter()
     launches = kb.kvs_launch_count() - launches0
     clocks = sampler.stop()
-    total_ms = max_over_ranks(total_ms)
+    total_ms = max_over_ranks(total_ms, world, dev)
     if status.item() != 0:
         raise RuntimeError(f"device status {status.item()}")
     ms_per_step = total_ms / args.steps
-    tokens_per_step = world * L * sum(w.seq_lens)
+    tokens_per_step = world * rank_tokens_per_step(w, L)
     value = tokens_per_step / (ms_per_step * 1e-3)
 
     # ---- per-kernel timing of the same steps (events around every launch; separate pass)
@@ -320,7 +359,7 @@ def main():
     e2e = None
     if not args.no_e2e:
         e2e_step(); sync_all()
-        e2e_ms = max_over_ranks(timed(e2e_step, max(1, min(args.steps, 3)))) / max(1, min(args.steps, 3))
+        e2e_ms = max_over_ranks(timed(e2e_step, max(1, min(args.steps, 3))), world, dev) / max(1, min(args.steps, 3))
         sync_all()
         h2d = sum(t.numel() * t.element_size() for t in (hK, hV, hC, hQ, hQn))
         d2h = sum(t.numel() * t.element_size() for t in (hRes, hResC, hOut))
