@@ -137,6 +137,41 @@ kvs_status_t kvs_compact(const kvs_params_t* params, void* K, void* V, int32_t* 
                          size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
 
 /*
+ * kvs_compact without a workspace argument, for callers that must not allocate device memory.
+ * The paper has no counterpart: this is a packaging variant of kvs_compact, not a step of the
+ * method.
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a serving engine that
+ * has handed all device memory to its own pool and forbids further allocations, inside a
+ * callback or a latency-critical section where an allocation would synchronise the device, or
+ * in a process whose memory budget is fixed at start-up.  kvs_compact asks such callers for a
+ * workspace they cannot create; this entry point brings its own.
+ *
+ * The scratch memory of the compaction (per-tile merge counts, tile tickets, "tile loaded" flags)
+ * lives in a fixed device array inside the library, kvs_static_scratch_bytes() = 4 MiB, which
+ * every GPU that loads the library holds until the process exits.  The call needs
+ *   batch * n_kv_heads * (n_max / 64 + 2) * 8 bytes (+ 512)
+ * of it and returns KVS_ERR_WORKSPACE, before anything is enqueued, if that exceeds the array
+ * (for example 8 KV heads x 131072 slots need 131 KiB; 256 units x 32768 slots need 1.03 MiB).
+ * All other arguments, results and error behaviour are those of kvs_compact.
+ *
+ * The function calls no cudaMalloc, cudaFree or other allocating routine.  The first call on each
+ * device looks up the array's device address (with that device current) and keeps it; make that
+ * first call outside any stream capture.  All calls share the one array, which keeps the
+ * previous call's contents: the tickets and flags are cleared on the stream at the start of each
+ * call, and two calls whose kernels overlap on the GPU (different streams, or different host
+ * threads on one device) race on it - serialise them.
+ */
+kvs_status_t kvs_compact_static(const kvs_params_t* params, void* K, void* V, int32_t* counts,
+                                const uint8_t* merge_mask, const float* w_left,
+                                const int32_t* seq_len, const int32_t* n_merge, int32_t n_max,
+                                int32_t* new_len, int32_t* new_index, int32_t* status_dev,
+                                void* cuda_stream);
+
+/* Size in bytes of the built-in scratch array that kvs_compact_static uses. */
+size_t kvs_static_scratch_bytes(void);
+
+/*
  * Attention of new queries over a (merged) cache, split along the slots and combined
  * [Eq. attn_def_vec with merged slots: numerator uses value sums, denominator weights
  * each slot by its count]:

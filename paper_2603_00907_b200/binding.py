@@ -21,7 +21,8 @@ STATUS_NAMES = {0: "KVS_OK", 1: "KVS_ERR_INVALID_ARG", 2: "KVS_ERR_UNSUPPORTED",
 
 EXPORTS = ["kvs_version", "kvs_last_error_string", "kvs_launch_count", "kvs_round_plan",
            "kvs_workspace_size", "kvs_merge_layer", "kvs_compact", "kvs_decode_attn",
-           "kvs_window_stats", "kvs_profile_begin", "kvs_profile_end", "kvs_profile_kind_name"]
+           "kvs_window_stats", "kvs_profile_begin", "kvs_profile_end", "kvs_profile_kind_name",
+           "kvs_compact_static", "kvs_static_scratch_bytes"]
 
 
 class KvsError(RuntimeError):
@@ -55,8 +56,10 @@ def lib() -> ctypes.CDLL:
         L.kvs_launch_count.restype = ctypes.c_uint64
         L.kvs_profile_kind_name.restype = ctypes.c_char_p
         L.kvs_profile_kind_name.argtypes = [ctypes.c_int32]
+        L.kvs_static_scratch_bytes.restype = ctypes.c_size_t
         for name in ("kvs_round_plan", "kvs_workspace_size", "kvs_merge_layer", "kvs_compact",
-                     "kvs_decode_attn", "kvs_window_stats", "kvs_profile_begin", "kvs_profile_end"):
+                     "kvs_decode_attn", "kvs_window_stats", "kvs_profile_begin", "kvs_profile_end",
+                     "kvs_compact_static"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -147,6 +150,23 @@ def kvs_compact(params: kvs_params_t, K, V, counts, merge_mask, w_left, seq_len:
                              ctypes.c_size_t(workspace.numel() * workspace.element_size()),
                              _ptr(status_dev), _stream()))
     return list(new_len)
+
+
+def kvs_compact_static(params: kvs_params_t, K, V, counts, merge_mask, w_left, seq_len: Sequence[int],
+                       n_merge: Sequence[int], new_index=None, status_dev=None) -> List[int]:
+    """kvs_compact for callers that cannot allocate: no workspace argument, the scratch is a fixed
+    array inside the library (kvs_static_scratch_bytes()); calls must not overlap on the GPU."""
+    B = params.batch
+    new_len = (ctypes.c_int32 * B)()
+    _check(lib().kvs_compact_static(ctypes.byref(params), _ptr(K), _ptr(V), _ptr(counts),
+                                    _ptr(merge_mask), _ptr(w_left), _i32(seq_len), _i32(n_merge),
+                                    ctypes.c_int32(counts.shape[-1]), new_len, _ptr(new_index),
+                                    _ptr(status_dev), _stream()))
+    return list(new_len)
+
+
+def kvs_static_scratch_bytes() -> int:
+    return int(lib().kvs_static_scratch_bytes())
 
 
 def kvs_decode_attn(params: kvs_params_t, q_new, K, V, counts, seq_len: Sequence[int], out,

@@ -436,6 +436,88 @@ kvs_status_t check_common(const kvs_params_t* p, const void* K, const void* V, c
 
 }  // namespace
 
+// =================================================================================== scratch-only compaction
+kvs_status_t kvs_detail_fail(kvs_status_t code, const char* msg) { return fail(code, "%s", msg); }
+
+// Scratch layout: tile_prefix int32 [U, tile_stride] | tickets uint32 [U] | flags uint32 [U, tile_stride].
+kvs_status_t kvs_detail_compact_scratch(const kvs_params_t* p, void* K, void* V, int32_t* counts,
+                                        const uint8_t* merge_mask, const float* w_left,
+                                        const int32_t* seq_len, const int32_t* n_merge, int32_t n_max,
+                                        int32_t* new_len, int32_t* new_index, void* scratch,
+                                        size_t scratch_bytes, size_t* need_bytes, int32_t* status_dev,
+                                        void* cuda_stream) {
+  kvs_status_t s = check_params(p);
+  if (s != KVS_OK) return s;
+  s = check_strides(p);
+  if (s != KVS_OK) return s;
+  if (!K || !V || !counts || !seq_len || !scratch || !merge_mask || !w_left || !n_merge || !new_len)
+    return fail(KVS_ERR_INVALID_ARG, "NULL pointer argument");
+  if (!aligned16(K) || !aligned16(V)) return fail(KVS_ERR_INVALID_ARG, "K and V must be 16-byte aligned");
+  if (n_max <= 0) return fail(KVS_ERR_INVALID_ARG, "n_max must be positive");
+  const int B = p->batch, U = p->batch * p->n_kv_heads;
+  for (int b = 0; b < B; ++b)
+    if (seq_len[b] < 0 || seq_len[b] > n_max) return fail(KVS_ERR_INVALID_ARG, "seq_len[%d] out of range", b);
+  const int tile_stride = n_max / KVS_CTILE + 2;
+  const size_t prefix_bytes = align_up((size_t)U * tile_stride * sizeof(int32_t));
+  const size_t sync_bytes = align_up(((size_t)U + (size_t)U * tile_stride) * sizeof(uint32_t));
+  if (need_bytes) *need_bytes = prefix_bytes + sync_bytes;
+  if (scratch_bytes < prefix_bytes + sync_bytes)
+    return fail(KVS_ERR_WORKSPACE, "scratch too small: %zu < %zu bytes", scratch_bytes, prefix_bytes + sync_bytes);
+  const int off = p->sink + (p->first_round & 1);
+  std::vector<SeqRound> act;
+  for (int b = 0; b < B; ++b) {
+    const int n = seq_len[b];
+    int P = (n - off - p->recent) / 2;
+    if (n - off - p->recent < 0 || P < 0) P = 0;
+    if (n_merge[b] < 0 || n_merge[b] > P) return fail(KVS_ERR_INVALID_ARG, "n_merge[%d] exceeds the candidate pairs", b);
+    if (n_merge[b] > 0) act.push_back({n, P, n_merge[b], b});
+  }
+  for (int b = 0; b < B; ++b) new_len[b] = seq_len[b] - n_merge[b];
+  if (act.empty() && !new_index) return KVS_OK;
+  if (new_index)
+    for (int b = 0; b < B; ++b)
+      if (n_merge[b] == 0 && seq_len[b] > 0) {
+        int P = (seq_len[b] - off - p->recent) / 2;
+        if (P < 0) P = 0;
+        act.push_back({seq_len[b], P, 0, b});
+      }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* base = static_cast<char*>(scratch);
+  int32_t* tile_prefix = reinterpret_cast<int32_t*>(base);
+  uint32_t* tickets = reinterpret_cast<uint32_t*>(base + prefix_bytes);
+  uint32_t* flags = tickets + U;
+  // tickets and flags must start at zero; the array keeps whatever the previous call left
+  CUDA_TRY(cudaMemsetAsync(base + prefix_bytes, 0, sync_bytes, st));
+  const CacheView view = make_view(p, K, V, counts, n_max);
+  const int caller_stride = n_max / 2;
+  for (size_t k = 0; k < act.size(); k += KVS_SEQ_CHUNK) {
+    RoundTable tab;
+    tab.nseq = 0;
+    tab.off = off;
+    for (size_t u = k; u < act.size() && tab.nseq < KVS_SEQ_CHUNK; ++u) tab.s[tab.nseq++] = act[u];
+    SelectArgs se;
+    se.Hkv = p->n_kv_heads;
+    se.pair_stride = caller_stride; se.tile_stride = tile_stride;
+    se.score = nullptr;
+    se.mask = const_cast<uint8_t*>(merge_mask);
+    se.tile_prefix = tile_prefix;
+    se.from_mask = 1;
+    CUDA_TRY(launch(KVS_K_MISC, st, [&] { return kvs_launch_select(se, tab, st); }));
+    CompactArgs ka;
+    ka.c = view;
+    ka.pair_stride = caller_stride; ka.tile_stride = tile_stride;
+    ka.mask = merge_mask; ka.w = w_left;
+    ka.tile_prefix = tile_prefix;
+    ka.tickets = tickets;
+    ka.flags = flags;
+    ka.epoch = 1;
+    ka.new_index = new_index;
+    ka.status_dev = status_dev;
+    CUDA_TRY(launch(KVS_K_COMPACT, st, [&] { return kvs_launch_compact(ka, tab, st); }));
+  }
+  return KVS_OK;
+}
+
 // =================================================================================== C ABI
 extern "C" {
 

@@ -181,3 +181,15 @@ __device__ __forceinline__ void st_release_u32(uint32_t* p, uint32_t v) {
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 #endif
+
+// ----------------------------------------------------------------------------- scratch-only compaction
+// One round of merge + compaction (the operation of kvs_compact) that takes its scratch memory
+// as a plain pointer instead of the general workspace.  `*need_bytes` receives the scratch size
+// the arguments ask for.  Used by the entry point that allocates nothing.
+kvs_status_t kvs_detail_compact_scratch(const kvs_params_t* p, void* K, void* V, int32_t* counts,
+                                        const uint8_t* merge_mask, const float* w_left,
+                                        const int32_t* seq_len, const int32_t* n_merge, int32_t n_max,
+                                        int32_t* new_len, int32_t* new_index, void* scratch,
+                                        size_t scratch_bytes, size_t* need_bytes, int32_t* status_dev,
+                                        void* cuda_stream);
+kvs_status_t kvs_detail_fail(kvs_status_t code, const char* msg);
