@@ -93,6 +93,21 @@ bool make_tmap(CUtensorMap* m, const void* base, int rank, const uint64_t* dims,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 5-D pair view of a bf16 cache [B,Hkv,n_max,128]: (channel, parity, slot / 2, head, sequence),
+// slot = 2 * (slot / 2) + parity.  A box is [64 channels x 128 consecutive pairs] of one parity.
+bool make_tmap_pairs(CUtensorMap* m, const void* base, int n_max, int Hkv, int B, int64_t st, int64_t sh, int64_t sb) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t npairs = (cuuint64_t)(n_max / 2 > 0 ? n_max / 2 : 1);
+  cuuint64_t gd[5] = {KVS_D, 2, npairs, (cuuint64_t)Hkv, (cuuint64_t)B};
+  cuuint64_t gs[4] = {(cuuint64_t)st * 2, (cuuint64_t)st * 4, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
+  cuuint32_t box[5] = {64, 1, 128, 1, 1}, es[5] = {1, 1, 1, 1, 1};
+  if (n_max < 2) gd[1] = 1;
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), gd, gs, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 const char* kKindNames[KVS_K_COUNT] = {"attn_partials", "combine", "hessian_stats",
                                        "select", "merge_compact", "misc"};
 
@@ -149,7 +164,7 @@ void round_plan(const kvs_params_t* p, int n, int budget, int r, int* off, int* 
 size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct WsLayout {
-  size_t part_ml, part_o, qstat, o, o_hi, o_lo, score, w, mask, tile_prefix, partA, partN1, partN12, partCos,
+  size_t part_ml, part_o, qstat, qc2, o, o_hi, o_lo, score, w, mask, tile_prefix, partA, partN1, partN12, partCos,
       sync, total;
   int splits_max, M_max, pair_stride, tile_stride, counter_stride, nqblk_w, U;
   size_t sync_bytes;
@@ -194,6 +209,7 @@ WsLayout make_layout(const kvs_params_t* p, int n_max, int max_new) {
   L.part_ml = o; o += align_up((size_t)L.U * part_rows * sizeof(float2));
   L.part_o = o;  o += align_up((size_t)L.U * part_rows * KVS_D * sizeof(float));
   L.qstat = o;   o += align_up((size_t)L.U * L.M_max * sizeof(float4));
+  L.qc2 = o;     o += align_up((size_t)L.U * ((Mw + 127) / 128 * 128) * sizeof(float2));
   L.o = o;       o += align_up((size_t)L.U * L.M_max * KVS_D * sizeof(float));
   L.score = o;   o += align_up((size_t)L.U * L.pair_stride * sizeof(float));
   L.w = o;       o += align_up((size_t)L.U * L.pair_stride * sizeof(float));
@@ -259,7 +275,7 @@ struct Common {
   int32_t* status_dev;
   bool simt_stats;           // debugging aid: statistics on the CUDA cores
   bool simt_flash;           // debugging aid: attention partials on the CUDA cores
-  CUtensorMap tmK, tmV, tmQ, tmOhi, tmOlo;
+  CUtensorMap tmK, tmV, tmQ, tmOhi, tmOlo, tmKp, tmVp;
 };
 
 int choose_splits(int M, int Hkv, int nseq, int nmax_slots, int* split_len);
@@ -322,7 +338,9 @@ kvs_status_t make_call_tmaps(Common* c, const void* K, const void* V, const void
   bool ok = make_tmap(&c->tmK, K, 4, kd, ks, 128) && make_tmap(&c->tmV, V, 4, kd, vs, 128) &&
             make_tmap(&c->tmQ, q_win, 3, qd, qs, 128) &&
             make_tmap(&c->tmOhi, c->ws + c->L.o_hi, 3, qd, qs, 128) &&
-            make_tmap(&c->tmOlo, c->ws + c->L.o_lo, 3, qd, qs, 128);
+            make_tmap(&c->tmOlo, c->ws + c->L.o_lo, 3, qd, qs, 128) &&
+            make_tmap_pairs(&c->tmKp, K, n_max, p->n_kv_heads, p->batch, p->k_stride_t, p->k_stride_h, p->k_stride_b) &&
+            make_tmap_pairs(&c->tmVp, V, n_max, p->n_kv_heads, p->batch, p->v_stride_t, p->v_stride_h, p->v_stride_b);
   if (!ok) return fail(KVS_ERR_CUDA, "cuTensorMapEncodeTiled failed or is unavailable");
   return KVS_OK;
 }
@@ -353,6 +371,8 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
   ca.o = reinterpret_cast<float*>(c.ws + c.L.o);
   ca.o_hi = reinterpret_cast<__nv_bfloat16*>(c.ws + c.L.o_hi);
   ca.o_lo = reinterpret_cast<__nv_bfloat16*>(c.ws + c.L.o_lo);
+  ca.qc2 = reinterpret_cast<float2*>(c.ws + c.L.qc2);
+  ca.M_pad = (c.Mw + 127) / 128 * 128;
   ca.out_bf16 = nullptr; ca.lse_out = lse_out; ca.o_out = o_out;
   CUDA_TRY(launch(KVS_K_COMBINE, c.st, [&] { return kvs_launch_combine(ca, tab, c.st); }));
 
@@ -372,7 +392,7 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
     ta.Hkv = p->n_kv_heads; ta.M = c.Mw; ta.nqblk = (c.Mw + 127) / 128;
     int pmax = 0;
     for (int i = 0; i < tab.nseq; ++i) pmax = pmax > tab.s[i].P ? pmax : tab.s[i].P;
-    const int ntiles = (2 * pmax + 127) / 128;
+    const int ntiles = (pmax + 127) / 128;               // tiles of 128 candidate pairs
     int splits = 148 / (ta.nqblk * ta.Hkv * tab.nseq);
     if (splits < 1) splits = 1;
     if (splits > ntiles) splits = ntiles;
@@ -380,7 +400,7 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
     ta.splits = (ntiles + ta.tiles_per_split - 1) / ta.tiles_per_split;
     ta.n_max = view.n_max; ta.pair_stride = c.L.pair_stride; ta.counter_stride = c.L.counter_stride;
     ta.scale_log2 = scale_log2; ta.score_mode = p->score_mode;
-    ta.counts = view.counts; ta.qstat = ca.qstat;
+    ta.counts = view.counts; ta.qc2 = ca.qc2; ta.M_pad = ca.M_pad;
     ta.score = sa.score; ta.w = sa.w; ta.A = A; ta.N1 = N1; ta.N12 = N12; ta.cosv = cosv;
     ta.partA = reinterpret_cast<float*>(c.ws + c.L.partA);
     ta.partN1 = reinterpret_cast<float*>(c.ws + c.L.partN1);
@@ -390,7 +410,7 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
                       (size_t)c.L.U * c.L.tile_stride;
     ta.status_dev = c.status_dev;
     CUDA_TRY(launch(KVS_K_STATS, c.st, [&] {
-      return kvs_launch_stats_tc(ta, tab, c.tmK, c.tmV, c.tmQ, c.tmOhi, c.tmOlo, c.st);
+      return kvs_launch_stats_tc(ta, tab, c.tmKp, c.tmVp, c.tmQ, c.tmOhi, c.tmOlo, c.st);
     }));
   }
 
@@ -750,7 +770,7 @@ kvs_status_t kvs_decode_attn(const kvs_params_t* p, const void* q_new, int32_t n
     ca.M = M; ca.splits = n_part; ca.Hkv = p->n_kv_heads;
     ca.part_ml = reinterpret_cast<float2*>(c.ws + c.L.part_ml);
     ca.part_o = reinterpret_cast<float*>(c.ws + c.L.part_o);
-    ca.qstat = nullptr; ca.o = nullptr; ca.o_hi = nullptr; ca.o_lo = nullptr;
+    ca.qstat = nullptr; ca.qc2 = nullptr; ca.M_pad = 0; ca.o = nullptr; ca.o_hi = nullptr; ca.o_lo = nullptr;
     ca.out_bf16 = static_cast<__nv_bfloat16*>(out);
     ca.lse_out = lse; ca.o_out = nullptr;
     CUDA_TRY(launch(KVS_K_COMBINE, c.st, [&] { return kvs_launch_combine(ca, tab, c.st); }));

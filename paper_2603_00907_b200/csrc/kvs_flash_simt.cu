@@ -148,6 +148,10 @@ combine_partials(const CombineArgs a, const RoundTable tab) {
   const int unit = sr.b * a.Hkv + blockIdx.y;
   const int m = blockIdx.x;
   const int d = threadIdx.x;
+  if (m >= a.M) {            // padding rows of the per-query constants: alpha = exp2(-inf) = 0
+    if (d == 0) a.qc2[(size_t)unit * a.M_pad + m] = make_float2(-INFINITY, 0.f);
+    return;
+  }
   const size_t base = (size_t)unit * a.splits * a.M + m;
   float mstar = -INFINITY;
   for (int s = 0; s < a.splits; ++s) mstar = fmaxf(mstar, a.part_ml[base + (size_t)s * a.M].x);
@@ -172,6 +176,7 @@ combine_partials(const CombineArgs a, const RoundTable tab) {
   const float lse = (mstar + log2f(Z)) * 0.6931471805599453f;
   if (d == 0) {
     if (a.qstat) a.qstat[row] = make_float4(mstar, Z, on2, lse);
+    if (a.qc2) a.qc2[(size_t)unit * a.M_pad + m] = make_float2(-(mstar + log2f(Z)), on2);
     if (a.lse_out) a.lse_out[row] = lse;
   }
   if (a.o) a.o[row * KVS_D + d] = od;
@@ -194,7 +199,7 @@ cudaError_t kvs_launch_flash_simt(const FlashArgs& a, const RoundTable& t, cudaS
 }
 
 cudaError_t kvs_launch_combine(const CombineArgs& a, const RoundTable& t, cudaStream_t st) {
-  dim3 grid(a.M, a.Hkv, t.nseq);
+  dim3 grid(a.qc2 ? a.M_pad : a.M, a.Hkv, t.nseq);
   combine_partials<<<grid, 128, 0, st>>>(a, t);
   return cudaGetLastError();
 }

@@ -78,6 +78,8 @@ struct CombineArgs {
   const float2* part_ml;
   const float* part_o;
   float4* qstat;           // [U, M]: (max log2, Z, |o|^2, lse natural)
+  float2* qc2;             // [U, M_pad]: (-(max + log2 Z), |o|^2); rows M..M_pad-1 get (-inf, 0) (may be NULL)
+  int32_t M_pad;           // M rounded up to a multiple of 128 (grid rows when qc2 is written)
   float* o;                // [U, M, 128] fp32 (may be NULL)
   __nv_bfloat16* o_hi;     // [U, M, 128]: o = o_hi + o_lo to ~2^-17 relative (may be NULL)
   __nv_bfloat16* o_lo;
@@ -110,7 +112,8 @@ struct StatsTcArgs {
   float scale_log2;
   int32_t score_mode;
   const int32_t* counts;   // [U, n_max]
-  const float4* qstat;     // [U, M]: (max log2, Z, |o|^2, lse)
+  const float2* qc2;       // [U, M_pad]: (-(max + log2 Z), |o|^2)
+  int32_t M_pad;
   float* score;            // [U, pair_stride]
   float* w;
   float* A;                // optional diagnostics [U, n_max]
@@ -153,8 +156,9 @@ struct CompactArgs {
 cudaError_t kvs_launch_flash_simt(const FlashArgs& a, const RoundTable& t, cudaStream_t st);
 cudaError_t kvs_launch_combine(const CombineArgs& a, const RoundTable& t, cudaStream_t st);
 cudaError_t kvs_launch_stats_simt(const StatsArgs& a, const RoundTable& t, cudaStream_t st);
-cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const CUtensorMap& tmK,
-                                const CUtensorMap& tmV, const CUtensorMap& tmQ, const CUtensorMap& tmOhi,
+// tmKp / tmVp: 5-D pair views [128, parity, slot / 2, head, sequence] of the caches
+cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const CUtensorMap& tmKp,
+                                const CUtensorMap& tmVp, const CUtensorMap& tmQ, const CUtensorMap& tmOhi,
                                 const CUtensorMap& tmOlo, cudaStream_t st);
 cudaError_t kvs_launch_flash_tc(const FlashTcArgs& a, const RoundTable& t, const CUtensorMap& tmK,
                                 const CUtensorMap& tmV, const CUtensorMap& tmQ, cudaStream_t st);

@@ -1,19 +1,23 @@
-// Hessian statistics on the tensor cores (tcgen05 + TMEM + TMA), keys on TMEM lanes.
+// Hessian statistics on the tensor cores (tcgen05 + TMEM + TMA), candidate pairs on TMEM lanes.
 //
 // One CTA owns a block of 128 window queries (Q, and the attention output O split into two
-// bf16 terms, stay in shared memory) and walks a range of 128-slot tiles of the candidate
-// region.  For every tile, TMA brings the K and V rows, and one thread issues
-//   S^T[slot, q] = K_tile Q^T                      (logits, fp32 in TMEM)
-//   T^T[slot, q] = Vsum_tile (O_hi + O_lo)^T       (value/output inner products)
-// Two groups of four warps alternate over the tiles.  Each thread owns one TMEM lane = one
-// cache slot, reads its row of S and T, and reduces over the queries, in registers,
+// bf16 terms, stay in shared memory) and walks a range of tiles of 128 candidate pairs.
+// A 5-D view of the cache, [128, parity, slot/2, head, sequence], lets TMA bring the left
+// members and the right members of the 128 pairs as two separate row tiles, so that TMEM
+// lane p holds everything of pair p.  For each half of 64 queries one thread issues
+//   S_l = K_l Q^T, S_r = K_r Q^T                    (logits, fp32 in TMEM)
+//   T_l = Vsum_l (O_hi + O_lo)^T, T_r likewise      (value/output inner products)
+// into one of two TMEM buffers; while the statistics warps reduce one half, the tensor
+// core fills the other.  Each statistics thread owns one pair and reduces over its queries,
+// in registers and with no cross-lane traffic,
 //   A_j   = sum_q alpha_qj
 //   N1_j  = sum_q alpha |1 - 2 alpha| |vbar_j - o_q|                    [Eqs. c11_def, c22_def]
 //   N12_p = sum_q alpha_j alpha_j+1 |vbar_j + vbar_j+1 - 2 o_q|         [Eq. c12_def]
 // with |vbar_j - o_q|^2 = |vbar_j|^2 - 2 T_jq / c_j + |o_q|^2.  The probability matrix never
-// leaves the SM.  The two members of a candidate pair sit in adjacent lanes and exchange
-// alpha and T by shuffle.  Query blocks of one tile are summed by the last block to arrive,
-// in block order, which then forms cosine, score and the merge weight of Eq. kstar_final.
+// leaves the SM.  The row norms and the in-pair inner products of K and Vsum are diagonals of
+// small warp-level tensor-core products (mma.sync) on the staged rows.  Query blocks of one
+// tile are summed by the last block to arrive, in block order, which then forms cosine, score
+// and the merge weight of Eq. kstar_final.
 #include "kvs_internal.h"
 #include "kvs_sm100.cuh"
 
@@ -21,62 +25,110 @@ using namespace sm100;
 
 namespace {
 
-constexpr int kTile = 128;                 // slots per tile = TMEM lanes
-constexpr int kQB = 128;                   // queries per block = accumulator columns
+constexpr int kPairs = 128;                // candidate pairs per tile = TMEM lanes
+constexpr int kQB = 128;                   // queries per CTA
+constexpr int kQH = 64;                    // queries per accumulator half
 constexpr int kHalf = 16384;               // bytes of a [128 rows x 64 bf16] swizzled sub-tile
 constexpr int kOperand = 2 * kHalf;        // a [128 x 128] bf16 operand
-constexpr int kStage = 2 * kOperand;       // K tile + V tile
-constexpr int kSmemQ = 0, kSmemOhi = kOperand, kSmemOlo = 2 * kOperand, kSmemStage = 3 * kOperand;
-constexpr int kSmemMisc = kSmemStage + 2 * kStage;
+constexpr int kSmemQ = 0, kSmemOhi = kOperand, kSmemOlo = 2 * kOperand;
+constexpr int kSmemKl = 3 * kOperand, kSmemKr = 4 * kOperand, kSmemVl = 5 * kOperand, kSmemVr = 6 * kOperand;
+constexpr int kSmemMisc = 7 * kOperand;
 constexpr int kThreads = 320;              // warp 0: TMA, warp 1: MMA, warps 2-9: statistics
 
 struct Misc {
-  uint64_t full[2], sfree[2], tfull[2], tfree[2], qfull;
+  uint64_t full, stage_free, tfull[2], tfree[2], qfull;
   uint32_t tmem_base;
   int abort_flag;
-  int last[2];
-  int wg_fail[2];                          // sticky: a wait of this group ran out
-  float2 qc[kQB];                          // per query: (max + log2 Z, |o|^2)
+  int fail;                                // sticky: a wait of the statistics warps ran out
+  int last;
+  float xbuf[kPairs * 5];                  // partial sums of the second statistics group
 };
-constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc) + 1024;   // + slack to align the base
+constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc);
+static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 
-__device__ __forceinline__ void wg_barrier(int wg) {
-  asm volatile("bar.sync %0, 128;" ::"r"(wg + 1) : "memory");
-}
+// all statistics threads / the first statistics group only
+__device__ __forceinline__ void stat_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void group0_barrier() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
 
-// Wait of a whole statistics group on one mbarrier phase.  One lane per warp polls; the
-// four warps then agree through shared memory, so that either all 128 threads go on or all
-// of them leave the tile loop (a thread that left alone would hang the others' barriers).
-__device__ __forceinline__ bool wg_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                        volatile int* wg_fail, int wg, int lane) {
-  int ok = 1;
+// Wait of all statistics warps on one mbarrier phase.  One lane per warp polls; the warps
+// then agree through shared memory, so that either all 256 threads go on or all of them leave
+// the tile loop (a thread that left alone would hang the others' barriers).
+__device__ __forceinline__ bool stat_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          volatile int* fail, int lane) {
   if (lane == 0) {
-    ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
-    if (!ok) *wg_fail = 1;
+    if (!mbar_wait(bar, parity, abort_flag)) *fail = 1;
   }
   __syncwarp();
-  wg_barrier(wg);
-  return *wg_fail == 0;
+  stat_barrier();
+  return *fail == 0;
 }
 
-// aa, bb, ab dot products of two swizzled 128-element bf16 rows of one operand tile
-__device__ __forceinline__ void row_dots(const uint8_t* tile, int ra, int rb, float& aa, float& bb, float& ab) {
-  aa = bb = ab = 0.f;
+__device__ __forceinline__ float fast_sqrt(float x) {
+  float y;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
 #pragma unroll
-  for (int hf = 0; hf < 2; ++hf) {
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t saddr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(saddr)
+               : "memory");
+}
+// D(16x8, fp32) += A(16x16, bf16, row major) B(16x8, bf16, column major)
+__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// For the 32 pairs of this warp's lane quarter: |x_l|^2, |x_r|^2 and <x_l, x_r> of the staged
+// rows of one operand (x = K or Vsum), delivered to the lane that owns the pair.
+// Eight pairs at a time, A = [x_l rows ; x_r rows] (16 x 128) against B = x_r and B = x_l
+// (8 rows each): the wanted values are diagonal elements of the two 16 x 8 products.
+__device__ __forceinline__ void pair_dots(const uint8_t* tl, const uint8_t* tr, int quarter, int lane,
+                                          float& ll, float& rr, float& lr) {
+  const uint32_t base_l = smem_u32(tl), base_r = smem_u32(tr);
+  const int mtx = lane >> 3, rin = lane & 7;                // ldmatrix: this lane feeds row rin of matrix mtx
+  const uint32_t opbase = (mtx & 1) ? base_r : base_l;      // matrices 0,2: left rows; 1,3: right rows
+  const int g = lane >> 2;                                  // accumulator row held by this lane
+  const int src = 4 * (lane & 7) + ((lane & 7) >> 1);       // lane that holds the diagonal of pair (lane & 7)
+  ll = rr = lr = 0.f;
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const uint4 xa = *reinterpret_cast<const uint4*>(tile + hf * kHalf + ra * 128 + ((c ^ (ra & 7)) << 4));
-      const uint4 xb = *reinterpret_cast<const uint4*>(tile + hf * kHalf + rb * 128 + ((c ^ (rb & 7)) << 4));
-      const uint32_t wa[4] = {xa.x, xa.y, xa.z, xa.w}, wb[4] = {xb.x, xb.y, xb.z, xb.w};
+  for (int blk = 0; blk < 4; ++blk) {
+    const int row = quarter * 32 + blk * 8 + rin;
+    float d1[4] = {0.f, 0.f, 0.f, 0.f}, d2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float a0 = bf16lo(wa[i]), a1 = bf16hi(wa[i]), b0 = bf16lo(wb[i]), b1 = bf16hi(wb[i]);
-        aa = fmaf(a0, a0, aa); aa = fmaf(a1, a1, aa);
-        bb = fmaf(b0, b0, bb); bb = fmaf(b1, b1, bb);
-        ab = fmaf(a0, b0, ab); ab = fmaf(a1, b1, ab);
-      }
+    for (int kk = 0; kk < 8; ++kk) {
+      const int chunk = 2 * (kk & 3) + (mtx >> 1);          // 16-byte chunk inside the 128-byte row
+      const uint32_t addr = opbase + (kk >> 2) * kHalf + row * 128 + ((chunk ^ (row & 7)) << 4);
+      uint32_t a[4];
+      ldmatrix_x4(a, addr);
+      mma16816(d1, a, a[1], a[3]);                          // columns = right rows
+      mma16816(d2, a, a[0], a[2]);                          // columns = left rows
     }
+    const float v_lr = (g & 1) ? d1[1] : d1[0];             // row g (left), column g (right)
+    const float v_rr = (g & 1) ? d1[3] : d1[2];             // row 8 + g (right), column g (right)
+    const float v_ll = (g & 1) ? d2[1] : d2[0];             // row g (left), column g (left)
+    const float s_lr = __shfl_sync(0xffffffffu, v_lr, src);
+    const float s_rr = __shfl_sync(0xffffffffu, v_rr, src);
+    const float s_ll = __shfl_sync(0xffffffffu, v_ll, src);
+    if ((lane >> 3) == blk) { lr = s_lr; rr = s_rr; ll = s_ll; }
   }
 }
 
@@ -94,11 +146,10 @@ __device__ __forceinline__ void finalize_pair(const StatsTcArgs& a, size_t pi, f
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constant__ CUtensorMap tmK,
-                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQ,
+hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constant__ CUtensorMap tmKp,
+                 const __grid_constant__ CUtensorMap tmVp, const __grid_constant__ CUtensorMap tmQ,
                  const __grid_constant__ CUtensorMap tmOhi, const __grid_constant__ CUtensorMap tmOlo) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  extern __shared__ __align__(1024) uint8_t smem[];
   Misc* misc = reinterpret_cast<Misc*>(smem + kSmemMisc);
 
   const int seq = blockIdx.z;
@@ -109,49 +160,47 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
   const int unit = sr.b * a.Hkv + h;
   const int off = tab.off;
   const int P = sr.P;
-  const int ntiles = (2 * P + kTile - 1) / kTile;
+  const int ntiles = (P + kPairs - 1) / kPairs;
   const int t_begin = min(ntiles, split * a.tiles_per_split);
   const int t_end = min(ntiles, t_begin + a.tiles_per_split);
   if (sr.n <= 0 || t_begin >= t_end) return;          // uniform over the CTA
+  if (smem_u32(smem) & 1023u) {                        // the swizzled tiles need a 1024-byte aligned base
+    if (threadIdx.x == 0 && a.status_dev) atomicExch(a.status_dev, (int)KVS_ERR_CUDA);
+    return;
+  }
   const int my_tiles = t_end - t_begin;
+  const int nh = (min(kQB, a.M - qblk * kQB) > kQH) ? 2 : 1;   // accumulator halves in use
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
+    mbar_init(&misc->full, 1);
+    mbar_init(&misc->stage_free, 1 + 8);   // MMA commit + the eight statistics warps
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&misc->full[s], 1);
-      mbar_init(&misc->sfree[s], 2);     // MMA commit + statistics group
       mbar_init(&misc->tfull[s], 1);
-      mbar_init(&misc->tfree[s], 1);
+      mbar_init(&misc->tfree[s], 8);
     }
     mbar_init(&misc->qfull, 1);
     misc->abort_flag = 0;
-    misc->last[0] = misc->last[1] = 0;
-    misc->wg_fail[0] = misc->wg_fail[1] = 0;
+    misc->fail = 0;
+    misc->last = 0;
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc(&misc->tmem_base, 512);
-  // per-query constants of this block: alpha = exp2(logit2 - (max + log2 Z))
-  if (threadIdx.x >= 64 && threadIdx.x < 64 + kQB) {
-    const int q = threadIdx.x - 64;
-    const int m = qblk * kQB + q;
-    float2 v = make_float2(INFINITY, 0.f);           // rows past M contribute alpha = 0
-    if (m < a.M) {
-      const float4 st = a.qstat[(size_t)unit * a.M + m];
-      v = make_float2(st.x + log2f(st.y), st.z);
-    }
-    misc->qc[q] = v;
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = misc->tmem_base;
   volatile int* abort_flag = &misc->abort_flag;
 
+  // tensor-map coordinates of the pair members: slot = 2 * rho + parity
+  const int par_l = off & 1, par_r = par_l ^ 1;
+  const int rho_l0 = off >> 1, rho_r0 = (off + 1) >> 1;
+
   if (warp == 0) {
     // ================================================================ TMA producer
     if (lane == 0) {
-      prefetch_tmap(&tmK); prefetch_tmap(&tmV); prefetch_tmap(&tmQ); prefetch_tmap(&tmOhi); prefetch_tmap(&tmOlo);
+      prefetch_tmap(&tmKp); prefetch_tmap(&tmVp); prefetch_tmap(&tmQ); prefetch_tmap(&tmOhi); prefetch_tmap(&tmOlo);
       mbar_expect_tx(&misc->qfull, 3 * kOperand);
       for (int hf = 0; hf < 2; ++hf) {
         tma_load_3d(smem + kSmemQ + hf * kHalf, &tmQ, &misc->qfull, hf * 64, qblk * kQB, unit);
@@ -160,179 +209,193 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
       }
       int issued = 0;
       for (int li = 0; li < my_tiles; ++li) {
-        const int s = li & 1, k = li >> 1;
-        if (!mbar_wait(&misc->sfree[s], (k & 1) ^ 1, abort_flag)) break;
-        uint8_t* st = smem + kSmemStage + s * kStage;
-        const int row = off + (t_begin + li) * kTile;
-        mbar_expect_tx(&misc->full[s], kStage);
+        if (!mbar_wait(&misc->stage_free, (li & 1) ^ 1, abort_flag)) break;
+        const int p0 = (t_begin + li) * kPairs;
+        mbar_expect_tx(&misc->full, 4 * kOperand);
         for (int hf = 0; hf < 2; ++hf) {
-          tma_load_4d(st + hf * kHalf, &tmK, &misc->full[s], hf * 64, row, h, sr.b);
-          tma_load_4d(st + kOperand + hf * kHalf, &tmV, &misc->full[s], hf * 64, row, h, sr.b);
+          tma_load_5d(smem + kSmemKl + hf * kHalf, &tmKp, &misc->full, hf * 64, par_l, rho_l0 + p0, h, sr.b);
+          tma_load_5d(smem + kSmemKr + hf * kHalf, &tmKp, &misc->full, hf * 64, par_r, rho_r0 + p0, h, sr.b);
+          tma_load_5d(smem + kSmemVl + hf * kHalf, &tmVp, &misc->full, hf * 64, par_l, rho_l0 + p0, h, sr.b);
+          tma_load_5d(smem + kSmemVr + hf * kHalf, &tmVp, &misc->full, hf * 64, par_r, rho_r0 + p0, h, sr.b);
         }
         issued = li + 1;
       }
-      if (*abort_flag) {
+      if (*abort_flag && issued > 0) {
         // drain: give the copies already issued a bounded time to land before the CTA leaves
-        for (int li = max(0, issued - 2); li < issued; ++li) {
-          const uint64_t t0 = globaltimer_ns();
-          while (!mbar_try_wait(&misc->full[li & 1], (li >> 1) & 1) && globaltimer_ns() - t0 < 200000000ull) {}
-        }
+        const uint64_t t0 = globaltimer_ns();
+        while (!mbar_try_wait(&misc->full, (issued - 1) & 1) && globaltimer_ns() - t0 < 200000000ull) {}
       }
     }
   } else if (warp == 1) {
     // ================================================================ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16(kTile, kQB);
+      constexpr uint32_t idesc = idesc_bf16(kPairs, kQH);
       const uint32_t q_addr = smem_u32(smem + kSmemQ), ohi_addr = smem_u32(smem + kSmemOhi),
                      olo_addr = smem_u32(smem + kSmemOlo);
+      const uint32_t kl = smem_u32(smem + kSmemKl), kr = smem_u32(smem + kSmemKr),
+                     vl = smem_u32(smem + kSmemVl), vr = smem_u32(smem + kSmemVr);
       bool ok = mbar_wait(&misc->qfull, 0, abort_flag);
       for (int li = 0; ok && li < my_tiles; ++li) {
-        const int s = li & 1, k = li >> 1;
-        if (!mbar_wait(&misc->full[s], k & 1, abort_flag)) break;
-        if (!mbar_wait(&misc->tfree[s], (k & 1) ^ 1, abort_flag)) break;
-        tc_fence_after();
-        const uint32_t k_addr = smem_u32(smem + kSmemStage + s * kStage);
-        const uint32_t v_addr = k_addr + kOperand;
-        const uint32_t dS = tmem + s * 256, dT = dS + 128;
+        if (!mbar_wait(&misc->full, li & 1, abort_flag)) break;
+        for (int hq = 0; hq < nh; ++hq) {
+          if (!mbar_wait(&misc->tfree[hq], (li & 1) ^ 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t d0 = tmem + hq * 256;
+          const uint32_t qrow = hq * (kQH * 128);          // rows 64.. of the query-side operands
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint32_t o = (kk >> 2) * kHalf + (kk & 3) * 32;
-          umma_bf16(dS, smem_desc_sw128(k_addr + o, 16, 1024), smem_desc_sw128(q_addr + o, 16, 1024), idesc, kk > 0);
-        }
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint32_t o = (kk >> 2) * kHalf + (kk & 3) * 32;
+            umma_bf16(d0, smem_desc_sw128(kl + o, 16, 1024), smem_desc_sw128(q_addr + qrow + o, 16, 1024), idesc, kk > 0);
+          }
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint32_t o = (kk >> 2) * kHalf + (kk & 3) * 32;
-          umma_bf16(dT, smem_desc_sw128(v_addr + o, 16, 1024), smem_desc_sw128(ohi_addr + o, 16, 1024), idesc, kk > 0);
-        }
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint32_t o = (kk >> 2) * kHalf + (kk & 3) * 32;
+            umma_bf16(d0 + 64, smem_desc_sw128(kr + o, 16, 1024), smem_desc_sw128(q_addr + qrow + o, 16, 1024), idesc, kk > 0);
+          }
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint32_t o = (kk >> 2) * kHalf + (kk & 3) * 32;
-          umma_bf16(dT, smem_desc_sw128(v_addr + o, 16, 1024), smem_desc_sw128(olo_addr + o, 16, 1024), idesc, 1);
+          for (int kk = 0; kk < 16; ++kk) {
+            const uint32_t o = ((kk & 7) >> 2) * kHalf + (kk & 3) * 32;
+            const uint32_t ob = (kk < 8 ? ohi_addr : olo_addr) + qrow + o;
+            umma_bf16(d0 + 128, smem_desc_sw128(vl + o, 16, 1024), smem_desc_sw128(ob, 16, 1024), idesc, kk > 0);
+          }
+#pragma unroll
+          for (int kk = 0; kk < 16; ++kk) {
+            const uint32_t o = ((kk & 7) >> 2) * kHalf + (kk & 3) * 32;
+            const uint32_t ob = (kk < 8 ? ohi_addr : olo_addr) + qrow + o;
+            umma_bf16(d0 + 192, smem_desc_sw128(vr + o, 16, 1024), smem_desc_sw128(ob, 16, 1024), idesc, kk > 0);
+          }
+          tc_commit(&misc->tfull[hq]);
         }
-        tc_commit(&misc->tfull[s]);
-        tc_commit(&misc->sfree[s]);
+        if (!ok) break;
+        tc_commit(&misc->stage_free);
       }
     }
   } else {
     // ================================================================ statistics warps
-    const int wg = (warp - 2) >> 2;                       // tiles li = wg, wg + 2, ...
-    const int lane_t = (warp & 3) * 32 + lane;            // TMEM lane = slot within the tile
-    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    const bool odd = lane_t & 1;
+    const int grp = (warp - 2) >> 2;                      // 0: queries 0-31 of each half, 1: queries 32-63
+    const int quarter = warp & 3;                         // TMEM lane quarter this warp may read
+    const int lane_p = quarter * 32 + lane;               // pair within the tile
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const int32_t* Cb = a.counts + (size_t)unit * a.n_max;
-    for (int li = wg; li < my_tiles; li += 2) {
-      const int s = wg, k = li >> 1;
+    const float2* qc = a.qc2 + (size_t)unit * a.M_pad + qblk * kQB;
+    volatile int* fail = &misc->fail;
+    for (int li = 0; li < my_tiles; ++li) {
       const int tile = t_begin + li;
-      const int j = off + tile * kTile + lane_t;          // this thread's slot
-      const int p = (tile * kTile + lane_t) >> 1;         // its candidate pair
-      const bool slot_ok = p < P;
-      float cnt = 1.f;
-      if (slot_ok) cnt = (float)Cb[j];
-      const float invc = 1.f / cnt, lc2 = log2f(cnt);
-      if (!wg_wait(&misc->full[s], k & 1, abort_flag, &misc->wg_fail[wg], wg, lane)) break;
-      // ---- per-slot norms and pair dot products from the staged rows: even lanes take the
-      //      K tile, odd lanes the V tile, both on the rows of their pair
-      const uint8_t* st = smem + kSmemStage + s * kStage;
-      float aa, bb, ab;
-      row_dots(st + (odd ? kOperand : 0), lane_t & ~1, lane_t | 1, aa, bb, ab);
-      // odd lane holds (|Vsum_even|^2, |Vsum_odd|^2, <Vsum_even, Vsum_odd>); even lane the K ones
-      const float o_aa = __shfl_xor_sync(0xffffffffu, aa, 1);
-      const float o_bb = __shfl_xor_sync(0xffffffffu, bb, 1);
-      const float o_ab = __shfl_xor_sync(0xffffffffu, ab, 1);
-      const float invc_p = __shfl_xor_sync(0xffffffffu, invc, 1);
-      const float v2_own = odd ? bb : o_aa, v2_par = odd ? aa : o_bb, vv = odd ? ab : o_ab;
-      const float k2e = odd ? o_aa : aa, k2o = odd ? o_bb : bb, kkp = odd ? o_ab : ab;
-      const float r2 = v2_own * invc * invc;                         // |vbar_j|^2
-      const float r2p = v2_par * invc_p * invc_p;
-      const float pair_c = r2 + r2p + 2.f * vv * invc * invc_p;      // |vbar_j + vbar_j+1|^2
-      const float cosv = kkp / fmaxf(sqrtf(k2e) * sqrtf(k2o), 1e-30f);
-      wg_barrier(wg);
-      if (lane_t == 0) mbar_arrive(&misc->sfree[s]);                 // staged rows no longer needed here
+      const int p = tile * kPairs + lane_p;               // candidate pair of this thread
+      const bool pair_ok = p < P;
+      const int jl = off + 2 * p;                         // its left slot
+      float cl = 1.f, cr = 1.f;
+      if (pair_ok) { cl = (float)Cb[jl]; cr = (float)Cb[jl + 1]; }
+      if (!stat_wait(&misc->full, li & 1, abort_flag, fail, lane)) break;
+      // ---- norms and in-pair products of the staged rows (values for both groups, keys for group 0)
+      float vll, vrr, vlr, kll = 1.f, krr = 1.f, klr = 0.f;
+      pair_dots(smem + kSmemVl, smem + kSmemVr, quarter, lane, vll, vrr, vlr);
+      if (grp == 0) pair_dots(smem + kSmemKl, smem + kSmemKr, quarter, lane, kll, krr, klr);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&misc->stage_free);      // staged rows no longer needed by this warp
+      const float icl = 1.f / cl, icr = 1.f / cr;
+      const float r2l = vll * icl * icl, r2r = vrr * icr * icr;       // |vbar|^2
+      const float pc = r2l + r2r + 2.f * vlr * icl * icr;             // |vbar_l + vbar_r|^2
+      const float cosv = klr / fmaxf(sqrtf(kll) * sqrtf(krr), 1e-30f);
+      const float n2cl = -2.f * cl, n2cr = -2.f * cr, n2il = -2.f * icl, n2ir = -2.f * icr;
 
-      if (!wg_wait(&misc->tfull[s], k & 1, abort_flag, &misc->wg_fail[wg], wg, lane)) break;
-      tc_fence_after();
-      float accA = 0.f, accN1 = 0.f, accN12 = 0.f;
+      // beta = alpha / c = exp2(scale * s - (max + log2 Z)); sums are scaled by the counts at the end
+      float sAl = 0.f, sAr = 0.f, sN1l = 0.f, sN1r = 0.f, sN12 = 0.f;
+      bool broken = false;
+      for (int hq = 0; hq < nh; ++hq) {
+        if (!stat_wait(&misc->tfull[hq], li & 1, abort_flag, fail, lane)) { broken = true; break; }
+        tc_fence_after();
 #pragma unroll 1
-      for (int c = 0; c < kQB / 32; ++c) {
-        float sv[32], tv[32];
-        tmem_ld32(tmem + lane_addr + s * 256 + c * 32, sv);
-        tmem_ld32(tmem + lane_addr + s * 256 + 128 + c * 32, tv);
-        tmem_ld_wait();
+        for (int c = 0; c < 2; ++c) {
+          const int q0 = grp * 32 + c * 16;               // first query of the chunk inside the half
+          const uint32_t col = tmem + lane_addr + hq * 256 + q0;
+          float sl[16], sr_[16], tl[16], tr[16];
+          tmem_ld16(col, sl);
+          tmem_ld16(col + 64, sr_);
+          tmem_ld16(col + 128, tl);
+          tmem_ld16(col + 192, tr);
+          const float4* qc4 = reinterpret_cast<const float4*>(qc + hq * kQH + q0);
+          float4 cst[8];
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const float2 c0 = misc->qc[c * 32 + i], c1 = misc->qc[c * 32 + i + 1];
-          const float al0 = fast_exp2(fmaf(sv[i], a.scale_log2, lc2) - c0.x);
-          const float al1 = fast_exp2(fmaf(sv[i + 1], a.scale_log2, lc2) - c1.x);
-          const float T0 = tv[i] * invc, T1 = tv[i + 1] * invc;
-          const float d0 = fmaxf(r2 - 2.f * T0 + c0.y, 0.f), d1 = fmaxf(r2 - 2.f * T1 + c1.y, 0.f);
-          accA += al0 + al1;
-          accN1 = fmaf(al0 * fabsf(1.f - 2.f * al0), sqrtf(d0), accN1);
-          accN1 = fmaf(al1 * fabsf(1.f - 2.f * al1), sqrtf(d1), accN1);
-          // pair term: the even lane takes query i, the odd lane query i + 1
-          const float al_send = odd ? al0 : al1, T_send = odd ? T0 : T1;
-          const float al_recv = __shfl_xor_sync(0xffffffffu, al_send, 1);
-          const float T_recv = __shfl_xor_sync(0xffffffffu, T_send, 1);
-          const float al_own = odd ? al1 : al0, T_own = odd ? T1 : T0, on2 = odd ? c1.y : c0.y;
-          const float d12 = fmaxf(pair_c - 4.f * (T_own + T_recv) + 4.f * on2, 0.f);
-          accN12 = fmaf(al_own * al_recv, sqrtf(d12), accN12);
+          for (int i = 0; i < 8; ++i) cst[i] = __ldg(qc4 + i);       // (-(max + log2 Z), |o|^2) of two queries
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float ncq = (i & 1) ? cst[i >> 1].z : cst[i >> 1].x;
+            const float hq2 = (i & 1) ? cst[i >> 1].w : cst[i >> 1].y;
+            const float bl = fast_exp2(fmaf(sl[i], a.scale_log2, ncq));
+            const float br = fast_exp2(fmaf(sr_[i], a.scale_log2, ncq));
+            sAl += bl;
+            sAr += br;
+            const float gl = bl * fabsf(fmaf(bl, n2cl, 1.f));        // beta |1 - 2 alpha|
+            const float gr = br * fabsf(fmaf(br, n2cr, 1.f));
+            const float dl = fmaf(tl[i], n2il, r2l + hq2);           // |vbar_l - o|^2
+            const float dr = fmaf(tr[i], n2ir, r2r + hq2);
+            sN1l = fmaf(gl, fast_sqrt(fabsf(dl)), sN1l);
+            sN1r = fmaf(gr, fast_sqrt(fabsf(dr)), sN1r);
+            const float u = fmaf(tl[i], icl, tr[i] * icr) - hq2;     // <vbar_l + vbar_r, o> - |o|^2
+            const float d12 = fmaf(u, -4.f, pc);                     // |vbar_l + vbar_r - 2 o|^2
+            sN12 = fmaf(bl * br, fast_sqrt(fabsf(d12)), sN12);
+          }
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&misc->tfree[hq]);                // this half may be overwritten
       }
-      tc_fence_before();
-      wg_barrier(wg);
-      if (lane_t == 0) mbar_arrive(&misc->tfree[s]);                 // accumulators may be overwritten
-      accN12 += __shfl_xor_sync(0xffffffffu, accN12, 1);
+      if (broken) break;
 
-      // ---- outputs of this tile
-      const size_t pi = (size_t)unit * a.pair_stride + p;
-      if (a.nqblk == 1) {
-        const float A_p = __shfl_xor_sync(0xffffffffu, accA, 1);
-        const float N1_p = __shfl_xor_sync(0xffffffffu, accN1, 1);
-        if (slot_ok) {
-          if (a.A) a.A[(size_t)unit * a.n_max + j] = accA;
-          if (a.N1) a.N1[(size_t)unit * a.n_max + j] = accN1;
-          if (!odd) finalize_pair(a, pi, accA, A_p, accN1, N1_p, accN12, cosv);
-        }
-      } else {
-        // partials of this query block, then the last block of the tile sums them in order
-        const size_t slot_i = ((size_t)unit * a.nqblk + qblk) * a.n_max + (slot_ok ? j : 0);
-        const size_t pair_i = ((size_t)unit * a.nqblk + qblk) * a.pair_stride + p;
-        if (slot_ok) {
-          a.partA[slot_i] = accA;
-          a.partN1[slot_i] = accN1;
-          if (!odd) {
-            a.partN12[pair_i] = accN12;
-            if (qblk == 0) a.partCos[pi] = cosv;
-          }
-        }
-        __threadfence();
-        wg_barrier(wg);
-        if (lane_t == 0) {
-          const uint32_t old = atomicAdd(&a.tile_counter[(size_t)unit * a.counter_stride + tile], 1u);
-          misc->last[wg] = ((old + 1) % (uint32_t)a.nqblk) == 0;
-        }
-        wg_barrier(wg);
-        if (misc->last[wg]) {
-          __threadfence();
-          float sA = 0.f, sN1 = 0.f, sN12 = 0.f, cs = 0.f;
-          if (slot_ok) {
-            for (int qb = 0; qb < a.nqblk; ++qb) {
-              const size_t si = ((size_t)unit * a.nqblk + qb) * a.n_max + j;
-              sA += __ldcg(a.partA + si);
-              sN1 += __ldcg(a.partN1 + si);
-              if (!odd) sN12 += __ldcg(a.partN12 + ((size_t)unit * a.nqblk + qb) * a.pair_stride + p);
-            }
-            if (!odd) cs = __ldcg(a.partCos + pi);
-          }
-          const float A_p = __shfl_xor_sync(0xffffffffu, sA, 1);
-          const float N1_p = __shfl_xor_sync(0xffffffffu, sN1, 1);
-          if (slot_ok) {
-            if (a.A) a.A[(size_t)unit * a.n_max + j] = sA;
-            if (a.N1) a.N1[(size_t)unit * a.n_max + j] = sN1;
-            if (!odd) finalize_pair(a, pi, sA, A_p, sN1, N1_p, sN12, cs);
-          }
-        }
-        wg_barrier(wg);     // misc->last[wg] is rewritten by the next tile
+      // ---- the second group hands its sums to the first, which owns the outputs
+      if (grp == 1) {
+        float* x = misc->xbuf + lane_p * 5;
+        x[0] = sAl; x[1] = sAr; x[2] = sN1l; x[3] = sN1r; x[4] = sN12;
       }
+      stat_barrier();
+      if (grp == 0) {
+        const float* x = misc->xbuf + lane_p * 5;
+        const float Al = cl * (sAl + x[0]), Ar = cr * (sAr + x[1]);
+        const float N1l = cl * (sN1l + x[2]), N1r = cr * (sN1r + x[3]);
+        const float N12 = cl * cr * (sN12 + x[4]);
+        const size_t pi = (size_t)unit * a.pair_stride + p;
+        if (a.nqblk == 1) {
+          if (pair_ok) {
+            if (a.A) { a.A[(size_t)unit * a.n_max + jl] = Al; a.A[(size_t)unit * a.n_max + jl + 1] = Ar; }
+            if (a.N1) { a.N1[(size_t)unit * a.n_max + jl] = N1l; a.N1[(size_t)unit * a.n_max + jl + 1] = N1r; }
+            finalize_pair(a, pi, Al, Ar, N1l, N1r, N12, cosv);
+          }
+        } else {
+          // partials of this query block, then the last block of the tile sums them in order
+          const size_t slot_i = ((size_t)unit * a.nqblk + qblk) * a.n_max + (pair_ok ? jl : 0);
+          const size_t pair_i = ((size_t)unit * a.nqblk + qblk) * a.pair_stride + (pair_ok ? p : 0);
+          if (pair_ok) {
+            a.partA[slot_i] = Al; a.partA[slot_i + 1] = Ar;
+            a.partN1[slot_i] = N1l; a.partN1[slot_i + 1] = N1r;
+            a.partN12[pair_i] = N12;
+          }
+          __threadfence();
+          group0_barrier();
+          if (lane_p == 0) {
+            const uint32_t old = atomicAdd(&a.tile_counter[(size_t)unit * a.counter_stride + tile], 1u);
+            misc->last = ((old + 1) % (uint32_t)a.nqblk) == 0;
+          }
+          group0_barrier();
+          if (misc->last) {
+            __threadfence();
+            if (pair_ok) {
+              float tAl = 0.f, tAr = 0.f, tN1l = 0.f, tN1r = 0.f, tN12 = 0.f;
+              for (int qb = 0; qb < a.nqblk; ++qb) {
+                const size_t si = ((size_t)unit * a.nqblk + qb) * a.n_max + jl;
+                tAl += __ldcg(a.partA + si); tAr += __ldcg(a.partA + si + 1);
+                tN1l += __ldcg(a.partN1 + si); tN1r += __ldcg(a.partN1 + si + 1);
+                tN12 += __ldcg(a.partN12 + ((size_t)unit * a.nqblk + qb) * a.pair_stride + p);
+              }
+              if (a.A) { a.A[(size_t)unit * a.n_max + jl] = tAl; a.A[(size_t)unit * a.n_max + jl + 1] = tAr; }
+              if (a.N1) { a.N1[(size_t)unit * a.n_max + jl] = tN1l; a.N1[(size_t)unit * a.n_max + jl + 1] = tN1r; }
+              finalize_pair(a, pi, tAl, tAr, tN1l, tN1r, tN12, cosv);
+            }
+          }
+        }
+      }
+      stat_barrier();          // xbuf and misc->last are rewritten by the next tile
     }
   }
 
@@ -349,8 +412,8 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
 
 }  // namespace
 
-cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const CUtensorMap& tmK,
-                                const CUtensorMap& tmV, const CUtensorMap& tmQ, const CUtensorMap& tmOhi,
+cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const CUtensorMap& tmKp,
+                                const CUtensorMap& tmVp, const CUtensorMap& tmQ, const CUtensorMap& tmOhi,
                                 const CUtensorMap& tmOlo, cudaStream_t st) {
   static bool configured = false;
   if (!configured) {
@@ -359,6 +422,6 @@ cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const
     configured = true;
   }
   dim3 grid(a.nqblk * a.splits, a.Hkv, t.nseq);
-  hessian_stats_tc<<<grid, kThreads, kSmemBytes, st>>>(a, t, tmK, tmV, tmQ, tmOhi, tmOlo);
+  hessian_stats_tc<<<grid, kThreads, kSmemBytes, st>>>(a, t, tmKp, tmVp, tmQ, tmOhi, tmOlo);
   return cudaGetLastError();
 }
