@@ -1,16 +1,24 @@
 // Merge of the selected adjacent pairs and stable in-place compaction of the cache.
 //
 // A tile is 64 consecutive slots starting at the first candidate slot (32 candidate pairs;
-// tiles past the last pair only shift the protected tail).  Each CTA takes a tile by ticket,
-// loads its rows into registers, forms the merged rows
+// tiles past the last pair only shift the protected tail).  CTAs are persistent: within one
+// (sequence, KV head) they take tiles by ticket.  A producer warp takes the ticket, streams
+// the tile's K and Vsum rows into a three-stage shared-memory ring with bulk asynchronous
+// copies, and stages the tile's decision (mask bits, weights, counts, merged pairs before the
+// tile).  Eight consumer warps read the rows into registers, free the stage, form the merged
+// rows
 //   K*    = bf16( K_right + w (K_left - K_right) )        [Eq. kstar_final, weight form]
 //   Vsum* = bf16( Vsum_left + Vsum_right ),  c* = c_left + c_right   [v* = v_m + v_{m+1}]
-// publishes "tile loaded", waits (bounded) until every earlier tile whose source rows it is
-// about to overwrite has loaded too, and stores the surviving rows at
+// publish "tile loaded", wait (bounded) until every earlier tile whose source rows they are
+// about to overwrite has loaded too, and store the surviving rows at
 //   new slot = old slot - (merged pairs before it).
-// Tickets make the wait safe: a tile only waits for tiles that took their ticket earlier,
-// and those never wait for later ones.
+// Tickets make the wait safe: a tile only waits for tiles with smaller tickets, whose owners
+// are running and handle their own tiles in ticket order, so the smallest unpublished tile
+// never waits.
 #include "kvs_internal.h"
+#include "kvs_sm100.cuh"
+
+using namespace sm100;
 
 namespace {
 
@@ -32,8 +40,52 @@ __device__ __forceinline__ uint4 add_v8(uint4 l, uint4 r) {
   return make_uint4(add_v2(l.x, r.x), add_v2(l.y, r.y), add_v2(l.z, r.z), add_v2(l.w, r.w));
 }
 
-__global__ void __launch_bounds__(256)
+constexpr int kStages = 3;
+constexpr int kRowBytes = KVS_D * 2;                       // one bf16 row
+constexpr int kOperandBytes = KVS_CTILE * kRowBytes;       // 16 KB: the K (or Vsum) rows of a tile
+constexpr int kStageBytes = 2 * kOperandBytes;
+constexpr int kConsumers = 256;
+constexpr int kThreads = kConsumers + 32;                  // + the producer warp
+
+struct TileMeta {
+  int32_t tile;                  // -1: no more tiles
+  int32_t E0;                    // merged pairs before the tile
+  uint32_t selbits;              // bit i: pair i of the tile is merged
+  int32_t pad;
+  float w[32];
+  int32_t cnt[KVS_CTILE];
+};
+struct Shared {
+  uint64_t full[kStages], meta_full[kStages], empty[kStages];
+  int abort_flag;
+  int fail;
+  TileMeta meta[kStages];
+};
+constexpr int kSmemBytes = kStages * kStageBytes + (int)sizeof(Shared);
+
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// Wait of all consumer warps on two mbarrier phases; either all 256 threads go on or all leave.
+__device__ __forceinline__ bool consumer_wait(uint64_t* b0, uint64_t* b1, uint32_t parity, volatile int* abort_flag,
+                                              volatile int* fail, int lane) {
+  if (lane == 0) {
+    if (!mbar_wait(b0, parity, abort_flag) || (b1 && !mbar_wait(b1, parity, abort_flag))) *fail = 1;
+  }
+  __syncwarp();
+  consumer_barrier();
+  return *fail == 0;
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
 merge_compact_kernel(const CompactArgs a, const RoundTable tab) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  Shared* sh = reinterpret_cast<Shared*>(smem + kStages * kStageBytes);
+
   const int seq = blockIdx.z;
   const SeqRound sr = tab.s[seq];
   const int n = sr.n;
@@ -42,136 +94,194 @@ merge_compact_kernel(const CompactArgs a, const RoundTable tab) {
   const int unit = sr.b * a.c.Hkv + h;
   const int off = tab.off;
   const int ntiles = (n - off + KVS_CTILE - 1) / KVS_CTILE;
-  const int tid = threadIdx.x;
-
-  __shared__ int s_tile;
-  __shared__ uint32_t s_selbits;
-  __shared__ int s_abort;
-  if (tid == 0) {
-    s_tile = (int)atomicAdd(&a.tickets[unit], 1u);
-    s_abort = 0;
-  }
-  __syncthreads();
-  const int t = s_tile;
-  if (t >= ntiles) return;
-
+  if ((int)blockIdx.x >= ntiles) return;                   // more CTAs than tiles: nothing to take
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int P = sr.P;
-  const uint8_t* mask = a.mask + (size_t)unit * a.pair_stride;
-  const float* wl = a.w + (size_t)unit * a.pair_stride;
-  if (tid < 32) {
-    const int p = 32 * t + tid;
-    const bool sel = p < P && mask[p] != 0;
-    const uint32_t bits = __ballot_sync(0xffffffffu, sel);
-    if (tid == 0) s_selbits = bits;
+
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sh->full[s], 1);
+      mbar_init(&sh->meta_full[s], 1);
+      mbar_init(&sh->empty[s], kConsumers / 32);
+    }
+    sh->abort_flag = 0;
+    sh->fail = 0;
+    mbar_fence_init();
   }
   __syncthreads();
-  const uint32_t selbits = s_selbits;
-  const int E0 = a.tile_prefix[(size_t)unit * a.tile_stride + t];
-  const int j0 = off + KVS_CTILE * t;
-
-  const int i = tid >> 3;          // pair in tile
-  const int c0 = tid & 7;          // chunks c0 and c0 + 8 (16 bytes each)
-  const int p = 32 * t + i;
-  const bool sel = (selbits >> i) & 1u;
-  const int e = __popc(selbits & ((1u << i) - 1u));
-  const int jl = j0 + 2 * i, jr = jl + 1;
-  const bool okl = jl < n, okr = jr < n;
-  const int dl = jl - E0 - e;
-  const int dr = jr - E0 - e;      // used only when !sel
+  volatile int* abort_flag = &sh->abort_flag;
 
   __nv_bfloat16* Kb = a.c.K + sr.b * a.c.ksb + h * a.c.ksh;
   __nv_bfloat16* Vb = a.c.V + sr.b * a.c.vsb + h * a.c.vsh;
   int32_t* Cb = a.c.counts + (size_t)unit * a.c.n_max;
 
-  uint4 kl[2], kr[2], vl[2], vr[2];
-  int32_t cl = 0, cr = 0;
-#pragma unroll
-  for (int u = 0; u < 2; ++u) {
-    const int ch = (c0 + 8 * u) * 8;
-    kl[u] = kr[u] = vl[u] = vr[u] = make_uint4(0, 0, 0, 0);
-    if (okl) {
-      kl[u] = *reinterpret_cast<const uint4*>(Kb + (int64_t)jl * a.c.kst + ch);
-      vl[u] = *reinterpret_cast<const uint4*>(Vb + (int64_t)jl * a.c.vst + ch);
-    }
-    if (okr) {
-      kr[u] = *reinterpret_cast<const uint4*>(Kb + (int64_t)jr * a.c.kst + ch);
-      vr[u] = *reinterpret_cast<const uint4*>(Vb + (int64_t)jr * a.c.vst + ch);
-    }
-  }
-  if (c0 == 0) {
-    if (okl) cl = Cb[jl];
-    if (okr) cr = Cb[jr];
-  }
-  if (sel) {
-    const float w = wl[p];
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      kl[u] = merge_k8(kl[u], kr[u], w);
-      vl[u] = add_v8(vl[u], vr[u]);
-    }
-    cl += cr;
-  }
-  __syncthreads();   // every load of this tile has returned (its values were just used)
-
-  const int moved = E0 + __popc(selbits);
-  if (moved != 0) {
-    if (tid == 0) st_release_u32(&a.flags[(size_t)unit * a.tile_stride + t], a.epoch);
-    // earlier tiles whose source rows overlap [j0 - E0, j0)
-    if (E0 > 0) {
-      const int first = (j0 - E0 - off) / KVS_CTILE;
-      for (int tt = t - 1 - tid; tt >= first; tt -= 256) {
-        const uint32_t* f = &a.flags[(size_t)unit * a.tile_stride + tt];
-        int spins = 0;
-        while (ld_acquire_u32(f) < a.epoch) {
-          if (++spins > KVS_SPIN_LIMIT) { s_abort = 1; break; }
-          __nanosleep(20);
+  if (warp == kConsumers / 32) {
+    // ================================================================ producer warp
+    const uint8_t* mask = a.mask + (size_t)unit * a.pair_stride;
+    const float* wl = a.w + (size_t)unit * a.pair_stride;
+    uint32_t next_ticket = 0;
+    if (lane == 0) next_ticket = atomicAdd(&a.tickets[unit], 1u);
+    for (int k = 0;; ++k) {
+      const int s = k % kStages;
+      const uint32_t ph = (uint32_t)(k / kStages) & 1u;
+      int ok = 1;
+      if (lane == 0) ok = mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      const int t = (int)__shfl_sync(0xffffffffu, next_ticket, 0);
+      TileMeta* m = &sh->meta[s];
+      if (t >= ntiles) {
+        if (lane == 0) { m->tile = -1; mbar_arrive(&sh->meta_full[s]); }
+        break;
+      }
+      if (lane == 0) next_ticket = atomicAdd(&a.tickets[unit], 1u);   // its latency hides behind this tile
+      const int j0 = off + KVS_CTILE * t;
+      const int rows = min(KVS_CTILE, n - j0);
+      uint8_t* sk = smem + s * kStageBytes;
+      uint8_t* sv = sk + kOperandBytes;
+      if (lane == 0) mbar_expect_tx(&sh->full[s], (uint32_t)rows * 2u * kRowBytes);
+      __syncwarp();
+      if (a.c.kst == KVS_D && a.c.vst == KVS_D) {
+        if (lane == 0) bulk_load(sk, Kb + (int64_t)j0 * KVS_D, (uint32_t)rows * kRowBytes, &sh->full[s]);
+        if (lane == 1) bulk_load(sv, Vb + (int64_t)j0 * KVS_D, (uint32_t)rows * kRowBytes, &sh->full[s]);
+      } else {
+        for (int r = lane; r < rows; r += 32) {
+          bulk_load(sk + r * kRowBytes, Kb + (int64_t)(j0 + r) * a.c.kst, kRowBytes, &sh->full[s]);
+          bulk_load(sv + r * kRowBytes, Vb + (int64_t)(j0 + r) * a.c.vst, kRowBytes, &sh->full[s]);
         }
       }
+      // the tile's decision
+      const int pp = 32 * t + lane;
+      const bool in_range = pp < P;
+      const bool sel = in_range && mask[pp] != 0;
+      m->w[lane] = in_range ? wl[pp] : 0.5f;
+      m->cnt[lane] = (lane < rows) ? Cb[j0 + lane] : 0;
+      m->cnt[lane + 32] = (lane + 32 < rows) ? Cb[j0 + lane + 32] : 0;
+      const uint32_t bits = __ballot_sync(0xffffffffu, sel);
+      if (lane == 0) {
+        m->selbits = bits;
+        m->E0 = a.tile_prefix[(size_t)unit * a.tile_stride + t];
+        m->tile = t;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->meta_full[s]);
     }
-    __syncthreads();
-    if (s_abort) {
-      if (tid == 0 && a.status_dev) atomicExch(a.status_dev, (int)KVS_ERR_TIMEOUT);
-      return;
-    }
+  } else {
+    // ================================================================ consumer warps
+    const int i = tid >> 3;          // pair in tile
+    const int c0 = tid & 7;          // chunks c0 and c0 + 8 (16 bytes each)
+    volatile int* fail = &sh->fail;
+    for (int k = 0;; ++k) {
+      const int s = k % kStages;
+      const uint32_t ph = (uint32_t)(k / kStages) & 1u;
+      if (!consumer_wait(&sh->meta_full[s], nullptr, ph, abort_flag, fail, lane)) break;
+      const TileMeta* m = &sh->meta[s];
+      const int t = m->tile;
+      if (t < 0) break;
+      if (!consumer_wait(&sh->full[s], nullptr, ph, abort_flag, fail, lane)) break;
+      const int j0 = off + KVS_CTILE * t;
+      const int jl = j0 + 2 * i, jr = jl + 1;
+      const bool okl = jl < n, okr = jr < n;
+      const uint8_t* sk = smem + s * kStageBytes;
+      const uint8_t* sv = sk + kOperandBytes;
+      uint4 kl[2], kr[2], vl[2], vr[2];
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const int ch = (c0 + 8 * u) * 8;
-      if (okl && (sel || dl != jl)) {
-        *reinterpret_cast<uint4*>(Kb + (int64_t)dl * a.c.kst + ch) = kl[u];
-        *reinterpret_cast<uint4*>(Vb + (int64_t)dl * a.c.vst + ch) = vl[u];
+      for (int u = 0; u < 2; ++u) {
+        const int ob = (c0 + 8 * u) * 16;
+        kl[u] = *reinterpret_cast<const uint4*>(sk + (2 * i) * kRowBytes + ob);
+        kr[u] = *reinterpret_cast<const uint4*>(sk + (2 * i + 1) * kRowBytes + ob);
+        vl[u] = *reinterpret_cast<const uint4*>(sv + (2 * i) * kRowBytes + ob);
+        vr[u] = *reinterpret_cast<const uint4*>(sv + (2 * i + 1) * kRowBytes + ob);
       }
-      if (okr && !sel && dr != jr) {
-        *reinterpret_cast<uint4*>(Kb + (int64_t)dr * a.c.kst + ch) = kr[u];
-        *reinterpret_cast<uint4*>(Vb + (int64_t)dr * a.c.vst + ch) = vr[u];
+      const uint32_t selbits = m->selbits;
+      const int E0 = m->E0;
+      const float w = m->w[i];
+      int32_t cl = m->cnt[2 * i], cr = m->cnt[2 * i + 1];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->empty[s]);          // the stage may be refilled
+
+      const bool sel = (selbits >> i) & 1u;
+      const int e = __popc(selbits & ((1u << i) - 1u));
+      const int dl = jl - E0 - e;
+      const int dr = jr - E0 - e;      // used only when !sel
+      if (sel) {
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          kl[u] = merge_k8(kl[u], kr[u], w);
+          vl[u] = add_v8(vl[u], vr[u]);
+        }
+        cl += cr;
+      }
+      // the tile's source rows are out of global memory: later tiles may overwrite them
+      if (tid == 0) st_release_u32(&a.flags[(size_t)unit * a.tile_stride + t], a.epoch);
+      const int moved = E0 + __popc(selbits);
+      if (E0 > 0 && gridDim.x > 1) {
+        // earlier tiles whose source rows overlap [j0 - E0, j0); a CTA that owns the whole unit
+        // has read them itself, in order, before it gets here
+        const int first = (j0 - E0 - off) / KVS_CTILE;
+        for (int tt = t - 1 - tid; tt >= first; tt -= kConsumers) {
+          const uint32_t* f = &a.flags[(size_t)unit * a.tile_stride + tt];
+          int spins = 0;
+          while (ld_acquire_u32(f) < a.epoch) {
+            if (++spins > KVS_SPIN_LIMIT || *abort_flag) { *fail = 1; *abort_flag = 1; break; }
+            __nanosleep(20);
+          }
+        }
+        consumer_barrier();
+        if (*fail) break;
+      }
+      if (moved != 0) {
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int ch = (c0 + 8 * u) * 8;
+          if (okl && (sel || dl != jl)) {
+            *reinterpret_cast<uint4*>(Kb + (int64_t)dl * a.c.kst + ch) = kl[u];
+            *reinterpret_cast<uint4*>(Vb + (int64_t)dl * a.c.vst + ch) = vl[u];
+          }
+          if (okr && !sel && dr != jr) {
+            *reinterpret_cast<uint4*>(Kb + (int64_t)dr * a.c.kst + ch) = kr[u];
+            *reinterpret_cast<uint4*>(Vb + (int64_t)dr * a.c.vst + ch) = vr[u];
+          }
+        }
+        if (c0 == 0) {
+          if (okl) Cb[dl] = cl;
+          if (okr && !sel) Cb[dr] = cr;
+        }
+      }
+      if (a.new_index && c0 == 0) {
+        int32_t* ni = a.new_index + (size_t)unit * a.c.n_max;
+        if (okl) ni[jl] = dl;
+        if (okr) ni[jr] = sel ? dl : dr;
+      }
+      if (a.new_index && t == 0) {
+        int32_t* ni = a.new_index + (size_t)unit * a.c.n_max;
+        for (int j = tid; j < off && j < n; j += kConsumers) ni[j] = j;
       }
     }
-    if (c0 == 0) {
-      if (okl) Cb[dl] = cl;
-      if (okr && !sel) Cb[dr] = cr;
-    }
-  } else if (tid == 0) {
-    // nothing moves, but later tiles may still wait on this flag
-    st_release_u32(&a.flags[(size_t)unit * a.tile_stride + t], a.epoch);
   }
-  if (a.new_index && c0 == 0) {
-    int32_t* ni = a.new_index + (size_t)unit * a.c.n_max;
-    if (okl) ni[jl] = dl;
-    if (okr) ni[jr] = sel ? dl : dr;
-  }
-  if (a.new_index && t == 0) {
-    int32_t* ni = a.new_index + (size_t)unit * a.c.n_max;
-    for (int j = tid; j < off && j < n; j += 256) ni[j] = j;
-  }
+  __syncthreads();
+  if (tid == 0 && sh->abort_flag && a.status_dev) atomicExch(a.status_dev, (int)KVS_ERR_TIMEOUT);
 }
 
 }  // namespace
 
 cudaError_t kvs_launch_compact(const CompactArgs& a, const RoundTable& t, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(merge_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
   int nmax = 0;
   for (int i = 0; i < t.nseq; ++i) nmax = nmax > t.s[i].n ? nmax : t.s[i].n;
   const int ntiles = (nmax - t.off + KVS_CTILE - 1) / KVS_CTILE;
   if (ntiles <= 0) return cudaSuccess;
-  dim3 grid(ntiles, a.c.Hkv, t.nseq);
-  merge_compact_kernel<<<grid, 256, 0, st>>>(a, t);
+  // persistent CTAs: two per SM over all units of the launch, at most one per tile
+  const int units = a.c.Hkv * t.nseq;
+  int per_unit = (2 * 148) / units;
+  if (per_unit > ntiles) per_unit = ntiles;
+  if (per_unit < 1) per_unit = 1;
+  dim3 grid(per_unit, a.c.Hkv, t.nseq);
+  merge_compact_kernel<<<grid, kThreads, kSmemBytes, st>>>(a, t);
   return cudaGetLastError();
 }

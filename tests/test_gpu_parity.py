@@ -236,6 +236,65 @@ def test_compact_bit_exact_given_mask(kb):
         K, V, C, n_list = Kn, Vn, Cn, n_new
 
 
+def test_compact_one_cta_per_unit_and_strided_rows(kb):
+    """256 (sequence, KV head) units in one launch: every unit is compacted by a single persistent
+    CTA that owns all of its tiles (no cross-CTA flags).  The cache is also given a slot stride of
+    160 elements, so rows are fetched one by one.  Random valid decisions; oracle bookkeeping."""
+    import torch
+    w = _small(seed=13, batch=32, n_q_heads=8, n_kv_heads=8, window=8,
+               seq_lens=tuple(200 + 37 * (i % 7) for i in range(32)), budgets=(64,) * 32)
+    data = wl.make_layer(w)
+    rng = np.random.default_rng(11)
+    B, Hkv, Nmax = w.batch, w.n_kv_heads, w.n_max
+    for strided in (False, True):
+        K, V, C = data["K"].copy(), data["V"].copy(), data["counts"].copy()
+        if strided:
+            Kd = torch.zeros((B, Hkv, Nmax, 160), dtype=torch.bfloat16, device="cuda")[..., :128]
+            Vd = torch.zeros((B, Hkv, Nmax, 160), dtype=torch.bfloat16, device="cuda")[..., :128]
+            Kd.copy_(tl.to_dev_bf16(K)); Vd.copy_(tl.to_dev_bf16(V))
+        else:
+            Kd, Vd = tl.to_dev_bf16(K), tl.to_dev_bf16(V)
+        Cd = torch.from_numpy(C).cuda()
+        n_list = list(w.seq_lens)
+        for r in (0, 1):
+            off = w.sink + (r % 2)
+            mask = np.zeros((B, Hkv, Nmax // 2), dtype=np.uint8)
+            wgt = rng.random((B, Hkv, Nmax // 2), dtype=np.float32)
+            n_merge = []
+            for b in range(B):
+                P = (n_list[b] - off - w.window) // 2
+                R = int(rng.integers(1, P // 2))
+                for h in range(Hkv):
+                    mask[b, h, rng.choice(P, size=R, replace=False)] = 1
+                n_merge.append(R)
+            p = kb.make_params(Kd, Vd, w.n_q_heads, w.window, sink=w.sink, first_round=r)
+            assert p.k_stride_t == (160 if strided else 128)
+            ws = torch.empty(kb.kvs_workspace_size(p, Nmax, 0), dtype=torch.uint8, device="cuda")
+            status = torch.zeros(1, dtype=torch.int32, device="cuda")
+            new_index = torch.full((B, Hkv, Nmax), -1, dtype=torch.int32, device="cuda")
+            got = kb.kvs_compact(p, Kd, Vd, Cd, torch.from_numpy(mask).cuda(), torch.from_numpy(wgt).cuda(),
+                                 n_list, n_merge, ws, new_index=new_index, status_dev=status)
+            torch.cuda.synchronize()
+            assert status.item() == 0
+            Kg, Vg, Cg, ig = tl.bits_of(Kd), tl.bits_of(Vd), Cd.cpu().numpy(), new_index.cpu().numpy()
+            Kn, Vn, Cn = np.zeros_like(K), np.zeros_like(V), np.zeros_like(C)
+            for b in range(B):
+                n, m = n_list[b], n_list[b] - n_merge[b]
+                assert got[b] == m
+                for h in range(Hkv):
+                    P = (n - off - w.window) // 2
+                    k2, v2, c2, ix = oc.apply_merge(K[b, h, :n], V[b, h, :n], C[b, h, :n].astype(np.int64), off,
+                                                    mask[b, h, :P], wgt[b, h, :P].astype(np.float64))
+                    Kn[b, h, :m], Vn[b, h, :m], Cn[b, h, :m] = k2, v2, c2
+                    assert np.array_equal(Cg[b, h, :m], c2)
+                    assert np.array_equal(ig[b, h, :n], ix)
+                    assert np.array_equal(Vg[b, h, :m], v2)
+                    ok, mx, nulp, worse = tl.bf16_close(Kg[b, h, :m], k2, atol=0.0)
+                    assert ok, (mx, nulp, worse)
+            K, V, C = Kn, Vn, Cn
+            n_list = got
+
+
 def test_merge_layer_stagewise_and_end_to_end(kb):
     """Round by round from the oracle's state (statistics, mask modulo the cutoff band, merge),
     then the whole pass in one call: it must equal the composition of single-round calls bit
