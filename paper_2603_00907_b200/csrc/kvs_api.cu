@@ -164,7 +164,7 @@ void round_plan(const kvs_params_t* p, int n, int budget, int r, int* off, int* 
 size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct WsLayout {
-  size_t part_ml, part_o, qstat, qc2, o, o_hi, o_lo, score, w, mask, tile_prefix, partA, partN1, partN12, partCos,
+  size_t part_ml, part_o, qstat, qc2, norms, o, o_hi, o_lo, score, w, mask, tile_prefix, partA, partN1, partN12, partCos,
       sync, total;
   int splits_max, M_max, pair_stride, tile_stride, counter_stride, nqblk_w, U;
   size_t sync_bytes;
@@ -211,6 +211,7 @@ WsLayout make_layout(const kvs_params_t* p, int n_max, int max_new) {
   L.qstat = o;   o += align_up((size_t)L.U * L.M_max * sizeof(float4));
   L.qc2 = o;     o += align_up((size_t)L.U * ((Mw + 127) / 128 * 128) * sizeof(float2));
   L.o = o;       o += align_up((size_t)L.U * L.M_max * KVS_D * sizeof(float));
+  L.norms = o;   o += align_up((size_t)L.U * L.pair_stride * sizeof(float4));
   L.score = o;   o += align_up((size_t)L.U * L.pair_stride * sizeof(float));
   L.w = o;       o += align_up((size_t)L.U * L.pair_stride * sizeof(float));
   L.mask = o;    o += align_up((size_t)L.U * L.pair_stride);
@@ -293,7 +294,7 @@ kvs_status_t enqueue_flash(const kvs_params_t* p, char* ws, const WsLayout& L, c
                            const CacheView& view, const void* q, int G, int Wq, int M, int causal,
                            const RoundTable& tab, int nmax_slots, bool simt, const CUtensorMap& tmK,
                            const CUtensorMap& tmV, const CUtensorMap& tmQ, int32_t* status_dev,
-                           LaunchFn&& launch_fn, int* n_part) {
+                           bool pair_norms, LaunchFn&& launch_fn, int* n_part) {
   float2* part_ml = reinterpret_cast<float2*>(ws + L.part_ml);
   float* part_o = reinterpret_cast<float*>(ws + L.part_o);
   const float scale_log2 = p->softmax_scale * 1.4426950408889634f;
@@ -311,7 +312,10 @@ kvs_status_t enqueue_flash(const kvs_params_t* p, char* ws, const WsLayout& L, c
   }
   FlashTcArgs ta;
   ta.Hkv = p->n_kv_heads; ta.M = M; ta.nqblk = (M + 127) / 128;
-  const int ntiles = (nmax_slots + 127) / 128;
+  // with pair norms the tiles start at -(off & 1), so that candidate pairs never straddle a tile
+  const int ntiles = (nmax_slots + (pair_norms ? (tab.off & 1) : 0) + 127) / 128;
+  ta.pair_norms = pair_norms ? reinterpret_cast<float4*>(ws + L.norms) : nullptr;
+  ta.pair_stride = L.pair_stride;
   ta.splits = tc_splits(M, p->n_kv_heads, tab.nseq, ntiles, &ta.tiles_per_split);
   ta.Wq = Wq; ta.causal = causal; ta.scale_log2 = scale_log2;
   ta.n_max = view.n_max; ta.counts = view.counts;
@@ -356,7 +360,7 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
   int n_part = 0;
   {
     kvs_status_t fs = enqueue_flash(p, c.ws, c.L, c.st, view, q_win, c.G, p->window, c.Mw, p->causal, tab,
-                                    nmax_slots, c.simt_flash, c.tmK, c.tmV, c.tmQ, c.status_dev,
+                                    nmax_slots, c.simt_flash, c.tmK, c.tmV, c.tmQ, c.status_dev, !c.simt_stats,
                                     [&](auto&& f) -> kvs_status_t {
                                       CUDA_TRY(launch(KVS_K_FLASH, c.st, f));
                                       return KVS_OK;
@@ -398,16 +402,14 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
     if (splits > ntiles) splits = ntiles;
     ta.tiles_per_split = (ntiles + splits - 1) / splits;
     ta.splits = (ntiles + ta.tiles_per_split - 1) / ta.tiles_per_split;
-    ta.n_max = view.n_max; ta.pair_stride = c.L.pair_stride; ta.counter_stride = c.L.counter_stride;
+    ta.n_max = view.n_max; ta.pair_stride = c.L.pair_stride;
     ta.scale_log2 = scale_log2; ta.score_mode = p->score_mode;
     ta.counts = view.counts; ta.qc2 = ca.qc2; ta.M_pad = ca.M_pad;
+    ta.pair_norms = reinterpret_cast<const float4*>(c.ws + c.L.norms); ta.norm_stride = c.L.pair_stride;
     ta.score = sa.score; ta.w = sa.w; ta.A = A; ta.N1 = N1; ta.N12 = N12; ta.cosv = cosv;
     ta.partA = reinterpret_cast<float*>(c.ws + c.L.partA);
     ta.partN1 = reinterpret_cast<float*>(c.ws + c.L.partN1);
     ta.partN12 = reinterpret_cast<float*>(c.ws + c.L.partN12);
-    ta.partCos = reinterpret_cast<float*>(c.ws + c.L.partCos);
-    ta.tile_counter = reinterpret_cast<uint32_t*>(c.ws + c.L.sync) + (size_t)KVS_MAX_ROUNDS * c.L.U +
-                      (size_t)c.L.U * c.L.tile_stride;
     ta.status_dev = c.status_dev;
     CUDA_TRY(launch(KVS_K_STATS, c.st, [&] {
       return kvs_launch_stats_tc(ta, tab, c.tmKp, c.tmVp, c.tmQ, c.tmOhi, c.tmOlo, c.st);
@@ -449,8 +451,9 @@ kvs_status_t check_common(const kvs_params_t* p, const void* K, const void* V, c
   c->G = p->n_q_heads / p->n_kv_heads;
   c->Mw = c->G * p->window;
   c->status_dev = nullptr;
-  c->simt_stats = env_simt_stats();
   c->simt_flash = env_simt_flash();
+  // the tensor-core statistics need the pair norms that the tensor-core attention pass writes
+  c->simt_stats = env_simt_stats() || c->simt_flash;
   return KVS_OK;
 }
 
@@ -760,7 +763,7 @@ kvs_status_t kvs_decode_attn(const kvs_params_t* p, const void* q_new, int32_t n
     if (tab.nseq == 0) continue;
     int n_part = 0;
     s = enqueue_flash(p, c.ws, c.L, c.st, view, q_new, c.G, n_new, M, 0, tab, nmax_slots, c.simt_flash, tmK,
-                      tmV, tmQ, status_dev,
+                      tmV, tmQ, status_dev, false,
                       [&](auto&& f) -> kvs_status_t {
                         CUDA_TRY(launch(KVS_K_FLASH, c.st, f));
                         return KVS_OK;

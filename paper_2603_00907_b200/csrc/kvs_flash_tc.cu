@@ -13,6 +13,11 @@
 // more than 2^8, in which case the group rescales its O_g rows in TMEM; otherwise O is never
 // touched until the end, where (stabiliser, sum, O) is written as the partial of this
 // (key split, group).  Window queries and decode queries use the same kernel.
+//
+// Two more warps serve the statistics pass that follows the window attention: tiles are then
+// aligned with the round's candidate pairs, and for every pair they form |vbar_l|^2, |vbar_r|^2,
+// |vbar_l + vbar_r|^2 and the adjacent-key cosine from the staged rows (diagonals of small
+// mma.sync products), so that the statistics kernel does not have to touch the rows for it.
 #include "kvs_internal.h"
 #include "kvs_sm100.cuh"
 
@@ -27,7 +32,7 @@ constexpr int kStage = 2 * kOperand;       // K tile + V tile
 constexpr int kPGroup = 2 * kHalf;         // P'_hi and P'_lo of one group: [128 q x 64 slots] each
 constexpr int kSmemQ = 0, kSmemStage = kOperand, kSmemP = kSmemStage + 2 * kStage;
 constexpr int kSmemMisc = kSmemP + 2 * kPGroup;
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;              // warp 0: TMA, 1: MMA, 2-9: softmax, 10-11: pair norms
 constexpr float kRescaleGap = 8.f;         // log2 units
 
 struct Misc {
@@ -90,6 +95,54 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t saddr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(saddr)
+               : "memory");
+}
+// D(16x8, fp32) += A(16x16, bf16, row major) B(16x8, bf16, column major)
+__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// For the 32 pairs (rows 2i, 2i+1) of rows [64 * half, 64 * half + 64) of one staged operand:
+// |x_l|^2, |x_r|^2 and <x_l, x_r>, delivered to lane i.  Eight pairs at a time,
+// A = [x_l rows ; x_r rows] (16 x 128) against B = x_r and B = x_l (8 rows each): the wanted
+// values are diagonal elements of the two 16 x 8 products.
+__device__ __forceinline__ void pair_dots(const uint8_t* tile, int half, int lane, float& ll, float& rr, float& lr) {
+  const uint32_t base = smem_u32(tile);
+  const int mtx = lane >> 3, rin = lane & 7;                // ldmatrix: this lane feeds row rin of matrix mtx
+  const int g = lane >> 2;                                  // accumulator row held by this lane
+  const int src = 4 * (lane & 7) + ((lane & 7) >> 1);       // lane that holds the diagonal of pair (lane & 7)
+  ll = rr = lr = 0.f;
+#pragma unroll
+  for (int blk = 0; blk < 4; ++blk) {
+    const int row = half * 64 + blk * 16 + 2 * rin + (mtx & 1);   // matrices 0,2: left rows; 1,3: right rows
+    float d1[4] = {0.f, 0.f, 0.f, 0.f}, d2[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {
+      const int chunk = 2 * (kk & 3) + (mtx >> 1);          // 16-byte chunk inside the 128-byte row
+      const uint32_t addr = base + (kk >> 2) * kHalf + row * 128 + ((chunk ^ (row & 7)) << 4);
+      uint32_t a[4];
+      ldmatrix_x4(a, addr);
+      mma16816(d1, a, a[1], a[3]);                          // columns = right rows
+      mma16816(d2, a, a[0], a[2]);                          // columns = left rows
+    }
+    const float v_lr = (g & 1) ? d1[1] : d1[0];             // row g (left), column g (right)
+    const float v_rr = (g & 1) ? d1[3] : d1[2];             // row 8 + g (right), column g (right)
+    const float v_ll = (g & 1) ? d2[1] : d2[0];             // row g (left), column g (left)
+    const float s_lr = __shfl_sync(0xffffffffu, v_lr, src);
+    const float s_rr = __shfl_sync(0xffffffffu, v_rr, src);
+    const float s_ll = __shfl_sync(0xffffffffu, v_ll, src);
+    if ((lane >> 3) == blk) { lr = s_lr; rr = s_rr; ll = s_ll; }
+  }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQ) {
@@ -105,14 +158,16 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
   const int split = blockIdx.x / a.nqblk;
   const int unit = sr.b * a.Hkv + h;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int ntiles = (n + kTile - 1) / kTile;
+  // with pair norms, tile t covers slots [128 t - shift, 128 t - shift + 128): aligned with the pairs
+  const int shift = a.pair_norms ? (tab.off & 1) : 0;
+  const int ntiles = (n + shift + kTile - 1) / kTile;
   const int t_begin = min(ntiles, split * a.tiles_per_split);
   const int t_end = min(ntiles, t_begin + a.tiles_per_split);
   const int my_tiles = t_end - t_begin;
   if (n <= 0) return;
   if (my_tiles <= 0) {
     // an empty split still owes its two (empty) partials to the combine
-    if (warp >= 2) {
+    if (warp >= 2 && warp < 10) {
       const int wg = (warp - 2) >> 2, row = (warp & 3) * 32 + lane, m = qblk * 128 + row;
       if (m < a.M) {
         const size_t pidx = ((size_t)unit * (a.splits * 2) + split * 2 + wg) * a.M + m;
@@ -121,11 +176,12 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     }
     return;
   }
+  const bool do_norms = a.pair_norms != nullptr && qblk == 0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2; ++s) {
       mbar_init(&misc->full[s], 1);
-      mbar_init(&misc->kvfree[s], 1);
+      mbar_init(&misc->kvfree[s], do_norms ? 3 : 1);    // MMA commit (+ the two pair-norm warps)
       mbar_init(&misc->sfull[s], 1);
       mbar_init(&misc->sfree[s], 2);
       mbar_init(&misc->pready[s], 1);
@@ -155,7 +211,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         const int s = li & 1, k = li >> 1;
         if (!mbar_wait(&misc->kvfree[s], (k & 1) ^ 1, abort_flag)) break;
         uint8_t* st = smem + kSmemStage + s * kStage;
-        const int row = (t_begin + li) * kTile;
+        const int row = (t_begin + li) * kTile - shift;
         mbar_expect_tx(&misc->full[s], kStage);
         for (int hf = 0; hf < 2; ++hf) {
           tma_load_4d(st + hf * kHalf, &tmK, &misc->full[s], hf * 64, row, h, sr.b);
@@ -217,6 +273,36 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         if (ok) tc_commit(&misc->kvfree[s]);
       }
     }
+  } else if (warp >= 10) {
+    // ================================================================ pair-norm warps
+    if (do_norms) {
+      const int hw = warp - 10;                                  // rows [64 hw, 64 hw + 64) of every tile
+      const int off = tab.off;
+      const int32_t* Cn = a.counts + (size_t)unit * a.n_max;
+      for (int li = 0; li < my_tiles; ++li) {
+        const int s = li & 1, k = li >> 1;
+        const int slot_l = (t_begin + li) * kTile - shift + hw * 64 + 2 * lane;   // left slot of this lane's pair
+        const int p = (slot_l - off) >> 1;
+        const bool pair_ok = slot_l >= off && p < sr.P;
+        float cl = 1.f, cr = 1.f;
+        if (pair_ok) { cl = (float)Cn[slot_l]; cr = (float)Cn[slot_l + 1]; }
+        int ok = 1;
+        if (lane == 0) ok = mbar_wait(&misc->full[s], k & 1, abort_flag) ? 1 : 0;
+        if (!__shfl_sync(0xffffffffu, ok, 0)) break;
+        const uint8_t* st = smem + kSmemStage + s * kStage;
+        float kll, krr, klr, vll, vrr, vlr;
+        pair_dots(st, hw, lane, kll, krr, klr);
+        pair_dots(st + kOperand, hw, lane, vll, vrr, vlr);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&misc->kvfree[s]);            // staged rows no longer needed here
+        if (pair_ok) {
+          const float icl = 1.f / cl, icr = 1.f / cr;
+          const float r2l = vll * icl * icl, r2r = vrr * icr * icr;
+          a.pair_norms[(size_t)unit * a.pair_stride + p] =
+              make_float4(r2l, r2r, r2l + r2r + 2.f * vlr * icl * icr, klr / fmaxf(sqrtf(kll) * sqrtf(krr), 1e-30f));
+        }
+      }
+    }
   } else {
     // ================================================================ softmax groups
     const int wg = (warp - 2) >> 2;
@@ -231,10 +317,10 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     bool alive = true;
     for (int li = 0; li < my_tiles; ++li) {
       const int s = li & 1, k = li >> 1;
-      const int j0 = (t_begin + li) * kTile + wg * 64;    // first slot of this group's half tile
+      const int j0 = (t_begin + li) * kTile - shift + wg * 64;    // first slot of this group's half tile
       if (t128 < 64) {
         const int j = j0 + t128;
-        const float cnt = (j < n) ? (float)Cb[j] : 1.f;
+        const float cnt = (j >= 0 && j < n) ? (float)Cb[j] : 1.f;
         misc->cst[wg][t128] = make_float2(log2f(cnt), 1.f / cnt);
       }
       if (!wg_wait(&misc->sfull[s], k & 1, abort_flag, &misc->wg_fail[wg], wg, lane)) { alive = false; break; }
@@ -248,7 +334,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       if (t128 == 0) mbar_arrive(&misc->sfree[s]);
       // logits in log2 units, with count bias and mask
       float mt = -INFINITY;
-      const bool need_mask = (j0 + 63 > min(n - 1, a.causal ? n - a.Wq : n - 1));
+      const bool need_mask = (j0 < 0) || (j0 + 63 > min(n - 1, a.causal ? n - a.Wq : n - 1));
       if (!need_mask) {
 #pragma unroll
         for (int i = 0; i < 64; ++i) {
@@ -259,7 +345,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
 #pragma unroll
         for (int i = 0; i < 64; ++i) {
           const float v = fmaf(x[i], a.scale_log2, misc->cst[wg][i].x);
-          x[i] = (j0 + i <= last_vis) ? v : -INFINITY;
+          x[i] = (j0 + i >= 0 && j0 + i <= last_vis) ? v : -INFINITY;
           mt = fmaxf(mt, x[i]);
         }
       }
@@ -306,14 +392,14 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         *reinterpret_cast<uint4*>(pbuf + kHalf + off16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
       }
       l += lsum;
-      // rows of the V tile past the end of the sequence may hold anything: zero them
-      const int tile_row0 = (t_begin + li) * kTile;
-      if (tile_row0 + kTile > n) {
+      // rows of the V tile outside the sequence may hold anything: zero them
+      const int tile_row0 = (t_begin + li) * kTile - shift;
+      if (tile_row0 < 0 || tile_row0 + kTile > n) {
         uint8_t* vt = smem + kSmemStage + s * kStage + kOperand;
-        const int r_lo = max(wg * 64, n - tile_row0), r_hi = wg * 64 + 64;
-        for (int it = r_lo * 16 + t128; it < r_hi * 16; it += 128) {
+        for (int it = wg * 64 * 16 + t128; it < (wg * 64 + 64) * 16; it += 128) {
           const int r = it >> 4, ch = it & 15;
-          *reinterpret_cast<uint4*>(vt + (ch >> 3) * kHalf + r * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
+          if (tile_row0 + r < 0 || tile_row0 + r >= n)
+            *reinterpret_cast<uint4*>(vt + (ch >> 3) * kHalf + r * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
         }
       }
       fence_proxy_async();

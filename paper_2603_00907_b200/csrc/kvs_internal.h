@@ -70,6 +70,8 @@ struct FlashTcArgs {
   const int32_t* counts;   // [U, n_max]
   float2* part_ml;         // [U, 2 * splits, M]
   float* part_o;           // [U, 2 * splits, M, 128]
+  float4* pair_norms;      // optional [U, pair_stride]: (|vbar_l|^2, |vbar_r|^2, |vbar_l + vbar_r|^2, cos(K_l, K_r))
+  int32_t pair_stride;     //   of the round's candidate pairs; tiles are then aligned with the pairs
   int32_t* status_dev;
 };
 
@@ -108,7 +110,7 @@ struct StatsArgs {
 
 struct StatsTcArgs {
   int32_t Hkv, M, nqblk, splits, tiles_per_split;
-  int32_t n_max, pair_stride, counter_stride;
+  int32_t n_max, pair_stride;
   float scale_log2;
   int32_t score_mode;
   const int32_t* counts;   // [U, n_max]
@@ -123,8 +125,8 @@ struct StatsTcArgs {
   float* partA;            // [U, nqblk, n_max] per-query-block partial sums
   float* partN1;
   float* partN12;          // [U, nqblk, pair_stride]
-  float* partCos;          // [U, pair_stride]
-  uint32_t* tile_counter;  // [U, counter_stride]; multiples of nqblk between launches
+  const float4* pair_norms; // [U, norm_stride] from the attention pass
+  int32_t norm_stride;
   int32_t* status_dev;
 };
 

@@ -14,10 +14,12 @@
 //   N1_j  = sum_q alpha |1 - 2 alpha| |vbar_j - o_q|                    [Eqs. c11_def, c22_def]
 //   N12_p = sum_q alpha_j alpha_j+1 |vbar_j + vbar_j+1 - 2 o_q|         [Eq. c12_def]
 // with |vbar_j - o_q|^2 = |vbar_j|^2 - 2 T_jq / c_j + |o_q|^2.  The probability matrix never
-// leaves the SM.  The row norms and the in-pair inner products of K and Vsum are diagonals of
-// small warp-level tensor-core products (mma.sync) on the staged rows.  Query blocks of one
-// tile are summed by the last block to arrive, in block order, which then forms cosine, score
-// and the merge weight of Eq. kstar_final.
+// leaves the SM.  The row norms |vbar|^2, |vbar_l + vbar_r|^2 and the adjacent-key cosine of
+// every pair come from the attention pass that precedes this kernel (it streams the same rows).
+// With one query block the kernel forms score and the merge weight of Eq. kstar_final itself;
+// with several, each block writes its partial sums and a small kernel adds them in block order.
+// Every synchronisation is an mbarrier with a bounded wait, so a warp that gives up can never
+// leave another one stuck.
 #include "kvs_internal.h"
 #include "kvs_sm100.cuh"
 
@@ -36,31 +38,23 @@ constexpr int kSmemMisc = 7 * kOperand;
 constexpr int kThreads = 320;              // warp 0: TMA, warp 1: MMA, warps 2-9: statistics
 
 struct Misc {
-  uint64_t full, stage_free, tfull[2], tfree[2], qfull;
+  uint64_t full, stage_free, tfull[2], tfree[2], qfull, xready, xfree;
   uint32_t tmem_base;
   int abort_flag;
-  int fail;                                // sticky: a wait of the statistics warps ran out
-  int last;
-  float xbuf[kPairs * 5];                  // partial sums of the second statistics group
+  float xbuf[kPairs * 5];                  // partial sums of the second statistics group, for the first
 };
 constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc);
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 
-// all statistics threads / the first statistics group only
-__device__ __forceinline__ void stat_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-__device__ __forceinline__ void group0_barrier() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
-
-// Wait of all statistics warps on one mbarrier phase.  One lane per warp polls; the warps
-// then agree through shared memory, so that either all 256 threads go on or all of them leave
-// the tile loop (a thread that left alone would hang the others' barriers).
-__device__ __forceinline__ bool stat_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          volatile int* fail, int lane) {
-  if (lane == 0) {
-    if (!mbar_wait(bar, parity, abort_flag)) *fail = 1;
-  }
+// One lane polls, the warp follows.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int lane) {
+  int ok = 1;
+  if (lane == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+__device__ __forceinline__ void warp_arrive(uint64_t* bar, int lane) {
   __syncwarp();
-  stat_barrier();
-  return *fail == 0;
+  if (lane == 0) mbar_arrive(bar);
 }
 
 __device__ __forceinline__ float fast_sqrt(float x) {
@@ -69,67 +63,15 @@ __device__ __forceinline__ float fast_sqrt(float x) {
   return y;
 }
 
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
-  uint32_t r[16];
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
+  uint32_t r[8];
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
       : "r"(taddr)
       : "memory");
 #pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t saddr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-               : "r"(saddr)
-               : "memory");
-}
-// D(16x8, fp32) += A(16x16, bf16, row major) B(16x8, bf16, column major)
-__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
-      "{%0, %1, %2, %3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// For the 32 pairs of this warp's lane quarter: |x_l|^2, |x_r|^2 and <x_l, x_r> of the staged
-// rows of one operand (x = K or Vsum), delivered to the lane that owns the pair.
-// Eight pairs at a time, A = [x_l rows ; x_r rows] (16 x 128) against B = x_r and B = x_l
-// (8 rows each): the wanted values are diagonal elements of the two 16 x 8 products.
-__device__ __forceinline__ void pair_dots(const uint8_t* tl, const uint8_t* tr, int quarter, int lane,
-                                          float& ll, float& rr, float& lr) {
-  const uint32_t base_l = smem_u32(tl), base_r = smem_u32(tr);
-  const int mtx = lane >> 3, rin = lane & 7;                // ldmatrix: this lane feeds row rin of matrix mtx
-  const uint32_t opbase = (mtx & 1) ? base_r : base_l;      // matrices 0,2: left rows; 1,3: right rows
-  const int g = lane >> 2;                                  // accumulator row held by this lane
-  const int src = 4 * (lane & 7) + ((lane & 7) >> 1);       // lane that holds the diagonal of pair (lane & 7)
-  ll = rr = lr = 0.f;
-#pragma unroll
-  for (int blk = 0; blk < 4; ++blk) {
-    const int row = quarter * 32 + blk * 8 + rin;
-    float d1[4] = {0.f, 0.f, 0.f, 0.f}, d2[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
-      const int chunk = 2 * (kk & 3) + (mtx >> 1);          // 16-byte chunk inside the 128-byte row
-      const uint32_t addr = opbase + (kk >> 2) * kHalf + row * 128 + ((chunk ^ (row & 7)) << 4);
-      uint32_t a[4];
-      ldmatrix_x4(a, addr);
-      mma16816(d1, a, a[1], a[3]);                          // columns = right rows
-      mma16816(d2, a, a[0], a[2]);                          // columns = left rows
-    }
-    const float v_lr = (g & 1) ? d1[1] : d1[0];             // row g (left), column g (right)
-    const float v_rr = (g & 1) ? d1[3] : d1[2];             // row 8 + g (right), column g (right)
-    const float v_ll = (g & 1) ? d2[1] : d2[0];             // row g (left), column g (left)
-    const float s_lr = __shfl_sync(0xffffffffu, v_lr, src);
-    const float s_rr = __shfl_sync(0xffffffffu, v_rr, src);
-    const float s_ll = __shfl_sync(0xffffffffu, v_ll, src);
-    if ((lane >> 3) == blk) { lr = s_lr; rr = s_rr; ll = s_ll; }
-  }
+  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 __device__ __forceinline__ void finalize_pair(const StatsTcArgs& a, size_t pi, float Aj, float Ap, float N1j,
@@ -175,15 +117,15 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
 
   if (threadIdx.x == 0) {
     mbar_init(&misc->full, 1);
-    mbar_init(&misc->stage_free, 1 + 8);   // MMA commit + the eight statistics warps
+    mbar_init(&misc->stage_free, 1);       // MMA commit
     for (int s = 0; s < 2; ++s) {
       mbar_init(&misc->tfull[s], 1);
-      mbar_init(&misc->tfree[s], 8);
+      mbar_init(&misc->tfree[s], 8);       // statistics warps
     }
     mbar_init(&misc->qfull, 1);
+    mbar_init(&misc->xready, 4);           // warps of the second statistics group
+    mbar_init(&misc->xfree, 4);            // warps of the first statistics group
     misc->abort_flag = 0;
-    misc->fail = 0;
-    misc->last = 0;
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc(&misc->tmem_base, 512);
@@ -278,124 +220,109 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const int32_t* Cb = a.counts + (size_t)unit * a.n_max;
     const float2* qc = a.qc2 + (size_t)unit * a.M_pad + qblk * kQB;
-    volatile int* fail = &misc->fail;
+    const float4* norms = a.pair_norms + (size_t)unit * a.norm_stride;
+    // norms and counts of the next tile's pair travel while the current tile is reduced
+    float4 nrm_next = make_float4(1.f, 1.f, 1.f, 0.f);
+    float cl_next = 1.f, cr_next = 1.f;
+    {
+      const int p = t_begin * kPairs + lane_p;
+      if (p < P) { nrm_next = __ldg(norms + p); cl_next = (float)Cb[off + 2 * p]; cr_next = (float)Cb[off + 2 * p + 1]; }
+    }
     for (int li = 0; li < my_tiles; ++li) {
       const int tile = t_begin + li;
       const int p = tile * kPairs + lane_p;               // candidate pair of this thread
       const bool pair_ok = p < P;
       const int jl = off + 2 * p;                         // its left slot
-      float cl = 1.f, cr = 1.f;
-      if (pair_ok) { cl = (float)Cb[jl]; cr = (float)Cb[jl + 1]; }
-      if (!stat_wait(&misc->full, li & 1, abort_flag, fail, lane)) break;
-      // ---- norms and in-pair products of the staged rows (values for both groups, keys for group 0)
-      float vll, vrr, vlr, kll = 1.f, krr = 1.f, klr = 0.f;
-      pair_dots(smem + kSmemVl, smem + kSmemVr, quarter, lane, vll, vrr, vlr);
-      if (grp == 0) pair_dots(smem + kSmemKl, smem + kSmemKr, quarter, lane, kll, krr, klr);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&misc->stage_free);      // staged rows no longer needed by this warp
+      const float4 nrm = nrm_next;
+      const float cl = cl_next, cr = cr_next;
+      if (li + 1 < my_tiles) {
+        const int pn = p + kPairs;
+        if (pn < P) { nrm_next = __ldg(norms + pn); cl_next = (float)Cb[off + 2 * pn]; cr_next = (float)Cb[off + 2 * pn + 1]; }
+      }
       const float icl = 1.f / cl, icr = 1.f / cr;
-      const float r2l = vll * icl * icl, r2r = vrr * icr * icr;       // |vbar|^2
-      const float pc = r2l + r2r + 2.f * vlr * icl * icr;             // |vbar_l + vbar_r|^2
-      const float cosv = klr / fmaxf(sqrtf(kll) * sqrtf(krr), 1e-30f);
+      const float r2l = nrm.x, r2r = nrm.y, pc = nrm.z, cosv = nrm.w;
       const float n2cl = -2.f * cl, n2cr = -2.f * cr, n2il = -2.f * icl, n2ir = -2.f * icr;
 
       // beta = alpha / c = exp2(scale * s - (max + log2 Z)); sums are scaled by the counts at the end
       float sAl = 0.f, sAr = 0.f, sN1l = 0.f, sN1r = 0.f, sN12 = 0.f;
       bool broken = false;
       for (int hq = 0; hq < nh; ++hq) {
-        if (!stat_wait(&misc->tfull[hq], li & 1, abort_flag, fail, lane)) { broken = true; break; }
+        if (!warp_wait(&misc->tfull[hq], li & 1, abort_flag, lane)) { broken = true; break; }
         tc_fence_after();
-#pragma unroll 1
-        for (int c = 0; c < 2; ++c) {
-          const int q0 = grp * 32 + c * 16;               // first query of the chunk inside the half
-          const uint32_t col = tmem + lane_addr + hq * 256 + q0;
-          float sl[16], sr_[16], tl[16], tr[16];
-          tmem_ld16(col, sl);
-          tmem_ld16(col + 64, sr_);
-          tmem_ld16(col + 128, tl);
-          tmem_ld16(col + 192, tr);
-          const float4* qc4 = reinterpret_cast<const float4*>(qc + hq * kQH + q0);
-          float4 cst[8];
+        const uint32_t col0 = tmem + lane_addr + hq * 256 + grp * 32;
+        const float4* qc4 = reinterpret_cast<const float4*>(qc + hq * kQH + grp * 32);
+        // four chunks of 8 queries; the loads of chunk c + 1 are in flight while chunk c is reduced
+        float buf[2][4][8];
+        float4 cst[2][4];
+        auto issue = [&](int c, int b) {
+          const uint32_t col = col0 + c * 8;
+          tmem_ld8(col, buf[b][0]);
+          tmem_ld8(col + 64, buf[b][1]);
+          tmem_ld8(col + 128, buf[b][2]);
+          tmem_ld8(col + 192, buf[b][3]);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) cst[i] = __ldg(qc4 + i);       // (-(max + log2 Z), |o|^2) of two queries
+          for (int i = 0; i < 4; ++i) cst[b][i] = __ldg(qc4 + c * 4 + i);   // (-(max + log2 Z), |o|^2) x 2 queries
+        };
+        issue(0, 0);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int b = c & 1;
           tmem_ld_wait();
+          if (c < 3) issue(c + 1, b ^ 1);
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float ncq = (i & 1) ? cst[i >> 1].z : cst[i >> 1].x;
-            const float hq2 = (i & 1) ? cst[i >> 1].w : cst[i >> 1].y;
-            const float bl = fast_exp2(fmaf(sl[i], a.scale_log2, ncq));
-            const float br = fast_exp2(fmaf(sr_[i], a.scale_log2, ncq));
+          for (int i = 0; i < 8; ++i) {
+            const float ncq = (i & 1) ? cst[b][i >> 1].z : cst[b][i >> 1].x;
+            const float hq2 = (i & 1) ? cst[b][i >> 1].w : cst[b][i >> 1].y;
+            const float bl = fast_exp2(fmaf(buf[b][0][i], a.scale_log2, ncq));
+            const float br = fast_exp2(fmaf(buf[b][1][i], a.scale_log2, ncq));
             sAl += bl;
             sAr += br;
-            const float gl = bl * fabsf(fmaf(bl, n2cl, 1.f));        // beta |1 - 2 alpha|
+            const float gl = bl * fabsf(fmaf(bl, n2cl, 1.f));              // beta |1 - 2 alpha|
             const float gr = br * fabsf(fmaf(br, n2cr, 1.f));
-            const float dl = fmaf(tl[i], n2il, r2l + hq2);           // |vbar_l - o|^2
-            const float dr = fmaf(tr[i], n2ir, r2r + hq2);
+            const float dl = fmaf(buf[b][2][i], n2il, r2l + hq2);          // |vbar_l - o|^2
+            const float dr = fmaf(buf[b][3][i], n2ir, r2r + hq2);
             sN1l = fmaf(gl, fast_sqrt(fabsf(dl)), sN1l);
             sN1r = fmaf(gr, fast_sqrt(fabsf(dr)), sN1r);
-            const float u = fmaf(tl[i], icl, tr[i] * icr) - hq2;     // <vbar_l + vbar_r, o> - |o|^2
-            const float d12 = fmaf(u, -4.f, pc);                     // |vbar_l + vbar_r - 2 o|^2
+            const float u = fmaf(buf[b][2][i], icl, buf[b][3][i] * icr) - hq2;   // <vbar_l + vbar_r, o> - |o|^2
+            const float d12 = fmaf(u, -4.f, pc);                           // |vbar_l + vbar_r - 2 o|^2
             sN12 = fmaf(bl * br, fast_sqrt(fabsf(d12)), sN12);
           }
         }
         tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&misc->tfree[hq]);                // this half may be overwritten
+        warp_arrive(&misc->tfree[hq], lane);                               // this half may be overwritten
       }
       if (broken) break;
 
       // ---- the second group hands its sums to the first, which owns the outputs
       if (grp == 1) {
+        // the first group must have read the previous tile's sums
+        if (!warp_wait(&misc->xfree, (li & 1) ^ 1, abort_flag, lane)) break;
         float* x = misc->xbuf + lane_p * 5;
         x[0] = sAl; x[1] = sAr; x[2] = sN1l; x[3] = sN1r; x[4] = sN12;
-      }
-      stat_barrier();
-      if (grp == 0) {
+        warp_arrive(&misc->xready, lane);
+      } else {
+        if (!warp_wait(&misc->xready, li & 1, abort_flag, lane)) break;
         const float* x = misc->xbuf + lane_p * 5;
         const float Al = cl * (sAl + x[0]), Ar = cr * (sAr + x[1]);
         const float N1l = cl * (sN1l + x[2]), N1r = cr * (sN1r + x[3]);
         const float N12 = cl * cr * (sN12 + x[4]);
-        const size_t pi = (size_t)unit * a.pair_stride + p;
-        if (a.nqblk == 1) {
-          if (pair_ok) {
+        warp_arrive(&misc->xfree, lane);                                   // the buffer may be rewritten
+        if (pair_ok) {
+          if (a.nqblk == 1) {
+            const size_t pi = (size_t)unit * a.pair_stride + p;
             if (a.A) { a.A[(size_t)unit * a.n_max + jl] = Al; a.A[(size_t)unit * a.n_max + jl + 1] = Ar; }
             if (a.N1) { a.N1[(size_t)unit * a.n_max + jl] = N1l; a.N1[(size_t)unit * a.n_max + jl + 1] = N1r; }
             finalize_pair(a, pi, Al, Ar, N1l, N1r, N12, cosv);
-          }
-        } else {
-          // partials of this query block, then the last block of the tile sums them in order
-          const size_t slot_i = ((size_t)unit * a.nqblk + qblk) * a.n_max + (pair_ok ? jl : 0);
-          const size_t pair_i = ((size_t)unit * a.nqblk + qblk) * a.pair_stride + (pair_ok ? p : 0);
-          if (pair_ok) {
+          } else {
+            // partial sums of this query block; a separate kernel adds the blocks in order
+            const size_t slot_i = ((size_t)unit * a.nqblk + qblk) * a.n_max + jl;
+            const size_t pair_i = ((size_t)unit * a.nqblk + qblk) * a.pair_stride + p;
             a.partA[slot_i] = Al; a.partA[slot_i + 1] = Ar;
             a.partN1[slot_i] = N1l; a.partN1[slot_i + 1] = N1r;
             a.partN12[pair_i] = N12;
           }
-          __threadfence();
-          group0_barrier();
-          if (lane_p == 0) {
-            const uint32_t old = atomicAdd(&a.tile_counter[(size_t)unit * a.counter_stride + tile], 1u);
-            misc->last = ((old + 1) % (uint32_t)a.nqblk) == 0;
-          }
-          group0_barrier();
-          if (misc->last) {
-            __threadfence();
-            if (pair_ok) {
-              float tAl = 0.f, tAr = 0.f, tN1l = 0.f, tN1r = 0.f, tN12 = 0.f;
-              for (int qb = 0; qb < a.nqblk; ++qb) {
-                const size_t si = ((size_t)unit * a.nqblk + qb) * a.n_max + jl;
-                tAl += __ldcg(a.partA + si); tAr += __ldcg(a.partA + si + 1);
-                tN1l += __ldcg(a.partN1 + si); tN1r += __ldcg(a.partN1 + si + 1);
-                tN12 += __ldcg(a.partN12 + ((size_t)unit * a.nqblk + qb) * a.pair_stride + p);
-              }
-              if (a.A) { a.A[(size_t)unit * a.n_max + jl] = tAl; a.A[(size_t)unit * a.n_max + jl + 1] = tAr; }
-              if (a.N1) { a.N1[(size_t)unit * a.n_max + jl] = tN1l; a.N1[(size_t)unit * a.n_max + jl + 1] = tN1r; }
-              finalize_pair(a, pi, tAl, tAr, tN1l, tN1r, tN12, cosv);
-            }
-          }
         }
       }
-      stat_barrier();          // xbuf and misc->last are rewritten by the next tile
     }
   }
 
@@ -408,6 +335,28 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
     tmem_dealloc(tmem, 512);
   }
   if (threadIdx.x == 0 && misc->abort_flag && a.status_dev) atomicExch(a.status_dev, (int)KVS_ERR_TIMEOUT);
+}
+
+// Sum of the per-query-block partials in block order, then score and weight of each pair.
+__global__ void __launch_bounds__(256)
+stats_finalize_kernel(const StatsTcArgs a, const RoundTable tab) {
+  const SeqRound sr = tab.s[blockIdx.z];
+  if (sr.n <= 0) return;
+  const int unit = sr.b * a.Hkv + blockIdx.y;
+  const int p = blockIdx.x * 256 + threadIdx.x;
+  if (p >= sr.P) return;
+  const int jl = tab.off + 2 * p;
+  float Al = 0.f, Ar = 0.f, N1l = 0.f, N1r = 0.f, N12 = 0.f;
+  for (int qb = 0; qb < a.nqblk; ++qb) {
+    const size_t si = ((size_t)unit * a.nqblk + qb) * a.n_max + jl;
+    Al += a.partA[si]; Ar += a.partA[si + 1];
+    N1l += a.partN1[si]; N1r += a.partN1[si + 1];
+    N12 += a.partN12[((size_t)unit * a.nqblk + qb) * a.pair_stride + p];
+  }
+  const size_t pi = (size_t)unit * a.pair_stride + p;
+  if (a.A) { a.A[(size_t)unit * a.n_max + jl] = Al; a.A[(size_t)unit * a.n_max + jl + 1] = Ar; }
+  if (a.N1) { a.N1[(size_t)unit * a.n_max + jl] = N1l; a.N1[(size_t)unit * a.n_max + jl + 1] = N1r; }
+  finalize_pair(a, pi, Al, Ar, N1l, N1r, N12, a.pair_norms[(size_t)unit * a.norm_stride + p].w);
 }
 
 }  // namespace
@@ -423,5 +372,12 @@ cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const
   }
   dim3 grid(a.nqblk * a.splits, a.Hkv, t.nseq);
   hessian_stats_tc<<<grid, kThreads, kSmemBytes, st>>>(a, t, tmKp, tmVp, tmQ, tmOhi, tmOlo);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess || a.nqblk == 1) return e;
+  int pmax = 0;
+  for (int i = 0; i < t.nseq; ++i) pmax = pmax > t.s[i].P ? pmax : t.s[i].P;
+  if (pmax <= 0) return cudaSuccess;
+  dim3 fgrid((pmax + 255) / 256, a.Hkv, t.nseq);
+  stats_finalize_kernel<<<fgrid, 256, 0, st>>>(a, t);
   return cudaGetLastError();
 }
