@@ -4,8 +4,9 @@
 // of 128-slot tiles.  Per tile, TMA brings the K and V rows and one thread issues
 //   S[q, slot] = Q K_tile^T                         (fp32 in TMEM, double buffered)
 // Two groups of four warps each take 64 of the tile's slots.  A thread owns one query row:
-// it adds the count bias ln c_j, applies the causal/tail mask, keeps a running stabiliser
-// and sum, and writes P' = exp(s - m) / c_j, split into two bf16 terms, to shared memory.
+// it applies the causal/tail mask, keeps a running stabiliser m and the sum
+// l = sum_j c_j exp(s_j - m) (the count bias ln c_j of a merged slot is the factor c_j), and
+// writes P' = exp(s - m) = alpha_j l / c_j, split into two bf16 terms, to shared memory.
 // The same issuing thread then runs, per group,
 //   O_g[q, :] += (P'_hi + P'_lo) Vsum_tile          (V as the MN-major operand)
 // with O_g accumulating in TMEM across the tiles [Eq. attn_def_vec with merged slots:
@@ -36,11 +37,11 @@ constexpr int kThreads = 384;              // warp 0: TMA, 1: MMA, 2-9: softmax,
 constexpr float kRescaleGap = 8.f;         // log2 units
 
 struct Misc {
-  uint64_t full[2], kvfree[2], sfull[2], sfree[2], pready[2], ofull[2], qfull;
+  uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[2], sfree[2], pready[2], ofull[2], qfull;
   uint32_t tmem_base;
   int abort_flag;
   int wg_fail[2];
-  float2 cst[2][64];                       // per group, per slot: (log2 c, 1/c)
+  alignas(16) float cnt[2][64];            // per group: counts of the half tile's slots (read as float4)
 };
 constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc) + 1024;
 
@@ -180,8 +181,12 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&misc->full[s], 1);
-      mbar_init(&misc->kvfree[s], do_norms ? 3 : 1);    // MMA commit (+ the two pair-norm warps)
+      // the K rows of a stage are free once the logits are formed, the V rows only after P V: two
+      // rings, so that the next K tile is requested a whole softmax earlier than the next V tile
+      mbar_init(&misc->kfull[s], 1);
+      mbar_init(&misc->vfull[s], 1);
+      mbar_init(&misc->kfree[s], do_norms ? 3 : 1);     // MMA commit (+ the two pair-norm warps)
+      mbar_init(&misc->vfree[s], do_norms ? 3 : 1);
       mbar_init(&misc->sfull[s], 1);
       mbar_init(&misc->sfree[s], 2);
       mbar_init(&misc->pready[s], 1);
@@ -201,28 +206,34 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
 
   if (warp == 0) {
     // ================================================================ TMA producer
-    if (lane == 0) {
-      prefetch_tmap(&tmK); prefetch_tmap(&tmV); prefetch_tmap(&tmQ);
-      mbar_expect_tx(&misc->qfull, kOperand);
-      for (int hf = 0; hf < 2; ++hf)
-        tma_load_3d(smem + kSmemQ + hf * kHalf, &tmQ, &misc->qfull, hf * 64, qblk * 128, unit);
+    // lane 0 streams the K tiles, lane 1 the V tiles
+    if (lane < 2) {
+      const bool is_v = lane == 1;
+      if (!is_v) {
+        prefetch_tmap(&tmK); prefetch_tmap(&tmQ);
+        mbar_expect_tx(&misc->qfull, kOperand);
+        for (int hf = 0; hf < 2; ++hf)
+          tma_load_3d(smem + kSmemQ + hf * kHalf, &tmQ, &misc->qfull, hf * 64, qblk * 128, unit);
+      } else {
+        prefetch_tmap(&tmV);
+      }
+      const CUtensorMap* tm = is_v ? &tmV : &tmK;
+      uint64_t* fullb = is_v ? misc->vfull : misc->kfull;
+      uint64_t* freeb = is_v ? misc->vfree : misc->kfree;
       int issued = 0;
       for (int li = 0; li < my_tiles; ++li) {
         const int s = li & 1, k = li >> 1;
-        if (!mbar_wait(&misc->kvfree[s], (k & 1) ^ 1, abort_flag)) break;
-        uint8_t* st = smem + kSmemStage + s * kStage;
+        if (!mbar_wait(&freeb[s], (k & 1) ^ 1, abort_flag)) break;
+        uint8_t* st = smem + kSmemStage + s * kStage + (is_v ? kOperand : 0);
         const int row = (t_begin + li) * kTile - shift;
-        mbar_expect_tx(&misc->full[s], kStage);
-        for (int hf = 0; hf < 2; ++hf) {
-          tma_load_4d(st + hf * kHalf, &tmK, &misc->full[s], hf * 64, row, h, sr.b);
-          tma_load_4d(st + kOperand + hf * kHalf, &tmV, &misc->full[s], hf * 64, row, h, sr.b);
-        }
+        mbar_expect_tx(&fullb[s], kOperand);
+        for (int hf = 0; hf < 2; ++hf) tma_load_4d(st + hf * kHalf, tm, &fullb[s], hf * 64, row, h, sr.b);
         issued = li + 1;
       }
       if (*abort_flag) {
         for (int li = max(0, issued - 2); li < issued; ++li) {
           const uint64_t t0 = globaltimer_ns();
-          while (!mbar_try_wait(&misc->full[li & 1], (li >> 1) & 1) && globaltimer_ns() - t0 < 200000000ull) {}
+          while (!mbar_try_wait(&fullb[li & 1], (li >> 1) & 1) && globaltimer_ns() - t0 < 200000000ull) {}
         }
       }
     }
@@ -234,7 +245,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       const uint32_t q_addr = smem_u32(smem + kSmemQ);
       auto issue_s = [&](int li) -> bool {
         const int s = li & 1, k = li >> 1;
-        if (!mbar_wait(&misc->full[s], k & 1, abort_flag)) return false;
+        if (!mbar_wait(&misc->kfull[s], k & 1, abort_flag)) return false;
         if (!mbar_wait(&misc->sfree[s], (k & 1) ^ 1, abort_flag)) return false;
         tc_fence_after();
         const uint32_t k_addr = smem_u32(smem + kSmemStage + s * kStage);
@@ -245,6 +256,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
                     idesc_s, kk > 0);
         }
         tc_commit(&misc->sfull[s]);
+        tc_commit(&misc->kfree[s]);
         return true;
       };
       bool ok = mbar_wait(&misc->qfull, 0, abort_flag);
@@ -253,6 +265,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         if (li + 1 < my_tiles) ok = issue_s(li + 1);
         const int s = li & 1;
         const uint32_t v_addr = smem_u32(smem + kSmemStage + s * kStage + kOperand);
+        if (ok && !mbar_wait(&misc->vfull[s], (li >> 1) & 1, abort_flag)) ok = false;
         for (int g = 0; ok && g < 2; ++g) {
           if (!mbar_wait(&misc->pready[g], li & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
@@ -270,7 +283,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
           }
           tc_commit(&misc->ofull[g]);
         }
-        if (ok) tc_commit(&misc->kvfree[s]);
+        if (ok) tc_commit(&misc->vfree[s]);
       }
     }
   } else if (warp >= 10) {
@@ -287,14 +300,15 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         float cl = 1.f, cr = 1.f;
         if (pair_ok) { cl = (float)Cn[slot_l]; cr = (float)Cn[slot_l + 1]; }
         int ok = 1;
-        if (lane == 0) ok = mbar_wait(&misc->full[s], k & 1, abort_flag) ? 1 : 0;
+        if (lane == 0)
+          ok = (mbar_wait(&misc->kfull[s], k & 1, abort_flag) && mbar_wait(&misc->vfull[s], k & 1, abort_flag)) ? 1 : 0;
         if (!__shfl_sync(0xffffffffu, ok, 0)) break;
         const uint8_t* st = smem + kSmemStage + s * kStage;
         float kll, krr, klr, vll, vrr, vlr;
         pair_dots(st, hw, lane, kll, krr, klr);
         pair_dots(st + kOperand, hw, lane, vll, vrr, vlr);
         __syncwarp();
-        if (lane == 0) mbar_arrive(&misc->kvfree[s]);            // staged rows no longer needed here
+        if (lane == 0) { mbar_arrive(&misc->kfree[s]); mbar_arrive(&misc->vfree[s]); }   // staged rows no longer needed here
         if (pair_ok) {
           const float icl = 1.f / cl, icr = 1.f / cr;
           const float r2l = vll * icl * icl, r2r = vrr * icr * icr;
@@ -315,13 +329,19 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     uint8_t* pbuf = smem + kSmemP + wg * kPGroup;
     float m_stab = -INFINITY, l = 0.f;
     bool alive = true;
+    // the count of "its" slot of the next tile travels while the current tile is processed
+    int cnt_next = 1;
+    if (t128 < 64) {
+      const int j = t_begin * kTile - shift + wg * 64 + t128;
+      if (j >= 0 && j < n) cnt_next = Cb[j];
+    }
     for (int li = 0; li < my_tiles; ++li) {
       const int s = li & 1, k = li >> 1;
       const int j0 = (t_begin + li) * kTile - shift + wg * 64;    // first slot of this group's half tile
       if (t128 < 64) {
-        const int j = j0 + t128;
-        const float cnt = (j >= 0 && j < n) ? (float)Cb[j] : 1.f;
-        misc->cst[wg][t128] = make_float2(log2f(cnt), 1.f / cnt);
+        misc->cnt[wg][t128] = (float)cnt_next;
+        const int j = j0 + kTile + t128;
+        cnt_next = (li + 1 < my_tiles && j >= 0 && j < n) ? Cb[j] : 1;
       }
       if (!wg_wait(&misc->sfull[s], k & 1, abort_flag, &misc->wg_fail[wg], wg, lane)) { alive = false; break; }
       tc_fence_after();
@@ -332,23 +352,25 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       tc_fence_before();
       wg_barrier(wg);
       if (t128 == 0) mbar_arrive(&misc->sfree[s]);
-      // logits in log2 units, with count bias and mask
+      // logits in log2 units, with mask (the stabiliser ignores the counts: exp(s - m) <= 1 either way)
       float mt = -INFINITY;
       const bool need_mask = (j0 < 0) || (j0 + 63 > min(n - 1, a.causal ? n - a.Wq : n - 1));
+      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one
       if (!need_mask) {
 #pragma unroll
         for (int i = 0; i < 64; ++i) {
-          x[i] = fmaf(x[i], a.scale_log2, misc->cst[wg][i].x);
-          mt = fmaxf(mt, x[i]);
+          x[i] *= a.scale_log2;
+          mx[i & 3] = fmaxf(mx[i & 3], x[i]);
         }
       } else {
 #pragma unroll
         for (int i = 0; i < 64; ++i) {
-          const float v = fmaf(x[i], a.scale_log2, misc->cst[wg][i].x);
+          const float v = x[i] * a.scale_log2;
           x[i] = (j0 + i >= 0 && j0 + i <= last_vis) ? v : -INFINITY;
-          mt = fmaxf(mt, x[i]);
+          mx[i & 3] = fmaxf(mx[i & 3], x[i]);
         }
       }
+      mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
       const float m_new = fmaxf(m_stab, mt);
       const bool need = m_new > m_stab + kRescaleGap || (m_stab == -INFINITY && m_new > -INFINITY);
       const bool any_need = wg_any(wg, need && li > 0);
@@ -373,28 +395,34 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       }
       if (need) m_stab = m_new;
       const float ms = (m_stab == -INFINITY) ? 0.f : m_stab;      // row with nothing visible yet
-      // P' = exp2(x - m) / c as hi + lo bf16, written as the K-major operand [row][64 slots]
-      float lsum = 0.f;
+      // P' = exp2(x - m) as hi + lo bf16, written as the K-major operand [row][64 slots]
+      // The hi term is the value cut to bf16 (a byte permute, no conversion); the lo term rounds
+      // the exact remainder, so hi + lo carries 16 significant bits.
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         uint32_t hi[4], lo[4];
+        const float4 ca = *reinterpret_cast<const float4*>(&misc->cnt[wg][c * 8]);
+        const float4 cb = *reinterpret_cast<const float4*>(&misc->cnt[wg][c * 8 + 4]);
+        const float cc[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const int i = c * 8 + u * 2;
-          const float p0 = fast_exp2(x[i] - ms), p1 = fast_exp2(x[i + 1] - ms);
-          lsum += p0 + p1;
-          const float q0 = p0 * misc->cst[wg][i].y, q1 = p1 * misc->cst[wg][i + 1].y;
-          hi[u] = pack_bf16(q0, q1);
-          lo[u] = pack_bf16(q0 - bf16lo(hi[u]), q1 - bf16hi(hi[u]));
+          const float q0 = fast_exp2(x[i] - ms), q1 = fast_exp2(x[i + 1] - ms);
+          ls[u] = fmaf(cc[2 * u], q0, fmaf(cc[2 * u + 1], q1, ls[u]));
+          const uint32_t b0 = __float_as_uint(q0), b1 = __float_as_uint(q1);
+          hi[u] = __byte_perm(b0, b1, 0x7632);
+          lo[u] = pack_bf16(q0 - __uint_as_float(b0 & 0xffff0000u), q1 - __uint_as_float(b1 & 0xffff0000u));
         }
         const int off16 = row * 128 + ((c ^ (row & 7)) << 4);
         *reinterpret_cast<uint4*>(pbuf + off16) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
         *reinterpret_cast<uint4*>(pbuf + kHalf + off16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
       }
-      l += lsum;
+      l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       // rows of the V tile outside the sequence may hold anything: zero them
       const int tile_row0 = (t_begin + li) * kTile - shift;
       if (tile_row0 < 0 || tile_row0 + kTile > n) {
+        if (!wg_wait(&misc->vfull[s], k & 1, abort_flag, &misc->wg_fail[wg], wg, lane)) { alive = false; break; }
         uint8_t* vt = smem + kSmemStage + s * kStage + kOperand;
         for (int it = wg * 64 * 16 + t128; it < (wg * 64 + 64) * 16; it += 128) {
           const int r = it >> 4, ch = it & 15;
