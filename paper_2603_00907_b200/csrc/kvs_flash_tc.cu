@@ -104,8 +104,7 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t saddr) {
 }
 // D(16x8, fp32) += A(16x16, bf16, row major) B(16x8, bf16, column major)
 __device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
       "{%0, %1, %2, %3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
@@ -114,7 +113,9 @@ __device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], 
 // For the 32 pairs (rows 2i, 2i+1) of rows [64 * half, 64 * half + 64) of one staged operand:
 // |x_l|^2, |x_r|^2 and <x_l, x_r>, delivered to lane i.  Eight pairs at a time,
 // A = [x_l rows ; x_r rows] (16 x 128) against B = x_r and B = x_l (8 rows each): the wanted
-// values are diagonal elements of the two 16 x 8 products.
+// values are diagonal elements of the two 16 x 8 products.  Two blocks of eight pairs are in
+// flight at once: all their fragments are loaded first, then four independent accumulation
+// chains run through the tensor cores.
 __device__ __forceinline__ void pair_dots(const uint8_t* tile, int half, int lane, float& ll, float& rr, float& lr) {
   const uint32_t base = smem_u32(tile);
   const int mtx = lane >> 3, rin = lane & 7;                // ldmatrix: this lane feeds row rin of matrix mtx
@@ -122,25 +123,36 @@ __device__ __forceinline__ void pair_dots(const uint8_t* tile, int half, int lan
   const int src = 4 * (lane & 7) + ((lane & 7) >> 1);       // lane that holds the diagonal of pair (lane & 7)
   ll = rr = lr = 0.f;
 #pragma unroll
-  for (int blk = 0; blk < 4; ++blk) {
-    const int row = half * 64 + blk * 16 + 2 * rin + (mtx & 1);   // matrices 0,2: left rows; 1,3: right rows
-    float d1[4] = {0.f, 0.f, 0.f, 0.f}, d2[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int bp = 0; bp < 2; ++bp) {
+    uint32_t fr[2][8][4];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int row = half * 64 + (2 * bp + u) * 16 + 2 * rin + (mtx & 1);   // matrices 0,2: left rows; 1,3: right rows
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {
+        const int chunk = 2 * (kk & 3) + (mtx >> 1);        // 16-byte chunk inside the 128-byte row
+        ldmatrix_x4(fr[u][kk], base + (kk >> 2) * kHalf + row * 128 + ((chunk ^ (row & 7)) << 4));
+      }
+    }
+    float d1[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, d2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
     for (int kk = 0; kk < 8; ++kk) {
-      const int chunk = 2 * (kk & 3) + (mtx >> 1);          // 16-byte chunk inside the 128-byte row
-      const uint32_t addr = base + (kk >> 2) * kHalf + row * 128 + ((chunk ^ (row & 7)) << 4);
-      uint32_t a[4];
-      ldmatrix_x4(a, addr);
-      mma16816(d1, a, a[1], a[3]);                          // columns = right rows
-      mma16816(d2, a, a[0], a[2]);                          // columns = left rows
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        mma16816(d1[u], fr[u][kk], fr[u][kk][1], fr[u][kk][3]);   // columns = right rows
+        mma16816(d2[u], fr[u][kk], fr[u][kk][0], fr[u][kk][2]);   // columns = left rows
+      }
     }
-    const float v_lr = (g & 1) ? d1[1] : d1[0];             // row g (left), column g (right)
-    const float v_rr = (g & 1) ? d1[3] : d1[2];             // row 8 + g (right), column g (right)
-    const float v_ll = (g & 1) ? d2[1] : d2[0];             // row g (left), column g (left)
-    const float s_lr = __shfl_sync(0xffffffffu, v_lr, src);
-    const float s_rr = __shfl_sync(0xffffffffu, v_rr, src);
-    const float s_ll = __shfl_sync(0xffffffffu, v_ll, src);
-    if ((lane >> 3) == blk) { lr = s_lr; rr = s_rr; ll = s_ll; }
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const float v_lr = (g & 1) ? d1[u][1] : d1[u][0];     // row g (left), column g (right)
+      const float v_rr = (g & 1) ? d1[u][3] : d1[u][2];     // row 8 + g (right), column g (right)
+      const float v_ll = (g & 1) ? d2[u][1] : d2[u][0];     // row g (left), column g (left)
+      const float s_lr = __shfl_sync(0xffffffffu, v_lr, src);
+      const float s_rr = __shfl_sync(0xffffffffu, v_rr, src);
+      const float s_ll = __shfl_sync(0xffffffffu, v_ll, src);
+      if ((lane >> 3) == 2 * bp + u) { lr = s_lr; rr = s_rr; ll = s_ll; }
+    }
   }
 }
 
@@ -177,7 +189,10 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     }
     return;
   }
-  const bool do_norms = a.pair_norms != nullptr && qblk == 0;
+  // the pair norms of a KV head are shared work: the first query block forms the key cosines, the
+  // second one (the first again, if there is only one) the value norms
+  const bool norm_k = a.pair_norms != nullptr && qblk == 0;
+  const bool norm_v = a.pair_norms != nullptr && qblk == (a.nqblk > 1 ? 1 : 0);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2; ++s) {
@@ -185,8 +200,8 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       // rings, so that the next K tile is requested a whole softmax earlier than the next V tile
       mbar_init(&misc->kfull[s], 1);
       mbar_init(&misc->vfull[s], 1);
-      mbar_init(&misc->kfree[s], do_norms ? 3 : 1);     // MMA commit (+ the two pair-norm warps)
-      mbar_init(&misc->vfree[s], do_norms ? 3 : 1);
+      mbar_init(&misc->kfree[s], norm_k ? 3 : 1);       // MMA commit (+ the two pair-norm warps)
+      mbar_init(&misc->vfree[s], norm_v ? 3 : 1);
       mbar_init(&misc->sfull[s], 1);
       mbar_init(&misc->sfree[s], 2);
       mbar_init(&misc->pready[s], 1);
@@ -206,34 +221,51 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
 
   if (warp == 0) {
     // ================================================================ TMA producer
-    // lane 0 streams the K tiles, lane 1 the V tiles
-    if (lane < 2) {
-      const bool is_v = lane == 1;
-      if (!is_v) {
-        prefetch_tmap(&tmK); prefetch_tmap(&tmQ);
-        mbar_expect_tx(&misc->qfull, kOperand);
-        for (int hf = 0; hf < 2; ++hf)
-          tma_load_3d(smem + kSmemQ + hf * kHalf, &tmQ, &misc->qfull, hf * 64, qblk * 128, unit);
-      } else {
-        prefetch_tmap(&tmV);
-      }
-      const CUtensorMap* tm = is_v ? &tmV : &tmK;
-      uint64_t* fullb = is_v ? misc->vfull : misc->kfull;
-      uint64_t* freeb = is_v ? misc->vfree : misc->kfree;
-      int issued = 0;
-      for (int li = 0; li < my_tiles; ++li) {
-        const int s = li & 1, k = li >> 1;
-        if (!mbar_wait(&freeb[s], (k & 1) ^ 1, abort_flag)) break;
-        uint8_t* st = smem + kSmemStage + s * kStage + (is_v ? kOperand : 0);
-        const int row = (t_begin + li) * kTile - shift;
-        mbar_expect_tx(&fullb[s], kOperand);
-        for (int hf = 0; hf < 2; ++hf) tma_load_4d(st + hf * kHalf, tm, &fullb[s], hf * 64, row, h, sr.b);
-        issued = li + 1;
+    // one thread streams both rings: whichever of the next K tile and the next V tile has a free
+    // stage is requested first
+    if (lane == 0) {
+      prefetch_tmap(&tmK); prefetch_tmap(&tmV); prefetch_tmap(&tmQ);
+      mbar_expect_tx(&misc->qfull, kOperand);
+      for (int hf = 0; hf < 2; ++hf)
+        tma_load_3d(smem + kSmemQ + hf * kHalf, &tmQ, &misc->qfull, hf * 64, qblk * 128, unit);
+      int kli = 0, vli = 0;
+      uint64_t t0 = globaltimer_ns();
+      while (kli < my_tiles || vli < my_tiles) {
+        bool progress = false;
+        if (kli < my_tiles && mbar_try_wait(&misc->kfree[kli & 1], ((kli >> 1) & 1) ^ 1)) {
+          const int s = kli & 1;
+          uint8_t* st = smem + kSmemStage + s * kStage;
+          const int row = (t_begin + kli) * kTile - shift;
+          mbar_expect_tx(&misc->kfull[s], kOperand);
+          for (int hf = 0; hf < 2; ++hf) tma_load_4d(st + hf * kHalf, &tmK, &misc->kfull[s], hf * 64, row, h, sr.b);
+          ++kli;
+          progress = true;
+        }
+        if (vli < my_tiles && mbar_try_wait(&misc->vfree[vli & 1], ((vli >> 1) & 1) ^ 1)) {
+          const int s = vli & 1;
+          uint8_t* st = smem + kSmemStage + s * kStage + kOperand;
+          const int row = (t_begin + vli) * kTile - shift;
+          mbar_expect_tx(&misc->vfull[s], kOperand);
+          for (int hf = 0; hf < 2; ++hf) tma_load_4d(st + hf * kHalf, &tmV, &misc->vfull[s], hf * 64, row, h, sr.b);
+          ++vli;
+          progress = true;
+        }
+        if (progress) {
+          t0 = globaltimer_ns();
+        } else {
+          if (*abort_flag) break;
+          if (globaltimer_ns() - t0 > 1000000000ull) { *abort_flag = 1; break; }
+        }
       }
       if (*abort_flag) {
-        for (int li = max(0, issued - 2); li < issued; ++li) {
-          const uint64_t t0 = globaltimer_ns();
-          while (!mbar_try_wait(&fullb[li & 1], (li >> 1) & 1) && globaltimer_ns() - t0 < 200000000ull) {}
+        // drain: give the copies already issued a bounded time to land before the CTA leaves
+        for (int li = max(0, kli - 2); li < kli; ++li) {
+          const uint64_t t1 = globaltimer_ns();
+          while (!mbar_try_wait(&misc->kfull[li & 1], (li >> 1) & 1) && globaltimer_ns() - t1 < 200000000ull) {}
+        }
+        for (int li = max(0, vli - 2); li < vli; ++li) {
+          const uint64_t t1 = globaltimer_ns();
+          while (!mbar_try_wait(&misc->vfull[li & 1], (li >> 1) & 1) && globaltimer_ns() - t1 < 200000000ull) {}
         }
       }
     }
@@ -288,32 +320,51 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     }
   } else if (warp >= 10) {
     // ================================================================ pair-norm warps
-    if (do_norms) {
+    if (norm_k || norm_v) {
       const int hw = warp - 10;                                  // rows [64 hw, 64 hw + 64) of every tile
       const int off = tab.off;
       const int32_t* Cn = a.counts + (size_t)unit * a.n_max;
+      // counts of the next tile's pair travel while the current tile is processed
+      float cl_next = 1.f, cr_next = 1.f;
+      if (norm_v) {
+        const int sl = t_begin * kTile - shift + hw * 64 + 2 * lane;
+        if (sl >= off && ((sl - off) >> 1) < sr.P) { cl_next = (float)Cn[sl]; cr_next = (float)Cn[sl + 1]; }
+      }
       for (int li = 0; li < my_tiles; ++li) {
         const int s = li & 1, k = li >> 1;
         const int slot_l = (t_begin + li) * kTile - shift + hw * 64 + 2 * lane;   // left slot of this lane's pair
         const int p = (slot_l - off) >> 1;
         const bool pair_ok = slot_l >= off && p < sr.P;
-        float cl = 1.f, cr = 1.f;
-        if (pair_ok) { cl = (float)Cn[slot_l]; cr = (float)Cn[slot_l + 1]; }
-        int ok = 1;
-        if (lane == 0)
-          ok = (mbar_wait(&misc->kfull[s], k & 1, abort_flag) && mbar_wait(&misc->vfull[s], k & 1, abort_flag)) ? 1 : 0;
-        if (!__shfl_sync(0xffffffffu, ok, 0)) break;
+        const float cl = cl_next, cr = cr_next;
+        if (norm_v && li + 1 < my_tiles) {
+          const int sl = slot_l + kTile;
+          cl_next = cr_next = 1.f;
+          if (sl >= off && ((sl - off) >> 1) < sr.P) { cl_next = (float)Cn[sl]; cr_next = (float)Cn[sl + 1]; }
+        }
+        float* out = reinterpret_cast<float*>(a.pair_norms + (size_t)unit * a.pair_stride + (pair_ok ? p : 0));
         const uint8_t* st = smem + kSmemStage + s * kStage;
-        float kll, krr, klr, vll, vrr, vlr;
-        pair_dots(st, hw, lane, kll, krr, klr);
-        pair_dots(st + kOperand, hw, lane, vll, vrr, vlr);
-        __syncwarp();
-        if (lane == 0) { mbar_arrive(&misc->kfree[s]); mbar_arrive(&misc->vfree[s]); }   // staged rows no longer needed here
-        if (pair_ok) {
-          const float icl = 1.f / cl, icr = 1.f / cr;
-          const float r2l = vll * icl * icl, r2r = vrr * icr * icr;
-          a.pair_norms[(size_t)unit * a.pair_stride + p] =
-              make_float4(r2l, r2r, r2l + r2r + 2.f * vlr * icl * icr, klr / fmaxf(sqrtf(kll) * sqrtf(krr), 1e-30f));
+        int ok = 1;
+        if (norm_k) {
+          if (lane == 0) ok = mbar_wait(&misc->kfull[s], k & 1, abort_flag) ? 1 : 0;
+          if (!__shfl_sync(0xffffffffu, ok, 0)) break;
+          float kll, krr, klr;
+          pair_dots(st, hw, lane, kll, krr, klr);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&misc->kfree[s]);           // the K rows are no longer needed here
+          if (pair_ok) out[3] = klr / fmaxf(sqrtf(kll) * sqrtf(krr), 1e-30f);
+        }
+        if (norm_v) {
+          if (lane == 0) ok = mbar_wait(&misc->vfull[s], k & 1, abort_flag) ? 1 : 0;
+          if (!__shfl_sync(0xffffffffu, ok, 0)) break;
+          float vll, vrr, vlr;
+          pair_dots(st + kOperand, hw, lane, vll, vrr, vlr);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&misc->vfree[s]);
+          if (pair_ok) {
+            const float icl = 1.f / cl, icr = 1.f / cr;
+            const float r2l = vll * icl * icl, r2r = vrr * icr * icr;
+            out[0] = r2l; out[1] = r2r; out[2] = r2l + r2r + 2.f * vlr * icl * icr;
+          }
         }
       }
     }
