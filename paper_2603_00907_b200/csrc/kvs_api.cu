@@ -170,15 +170,38 @@ struct WsLayout {
   size_t sync_bytes;
 };
 
+// Number of key/pair ranges each (query block, KV head, sequence) item is cut into, so that the
+// CTAs (one per SM, equal length) fill whole waves of the 148 SMs.  With fewer items than SMs
+// the items are cut until the SMs are covered; with more, the cut that minimises
+// ceil(items * k / 148) / k (the makespan in item lengths) is taken, e.g. 512 items: k = 2 gives
+// 7 half-length waves instead of 4 full ones.
+constexpr int kNumSMs = 148;
+constexpr int kMaxTcSplits = 8;     // per item; the attention partials are sized for it
+
+int balanced_splits(int items, int ntiles, int* tiles_per_split) {
+  int best = 1;
+  if (items < kNumSMs) {
+    best = kNumSMs / items;
+  } else {
+    double best_cost = 1e30;
+    for (int k = 1; k <= kMaxTcSplits; ++k) {
+      if (k > 1 && ntiles / k < 4) break;                   // keep ranges long enough to amortise the set-up
+      const double cost = (double)((items * k + kNumSMs - 1) / kNumSMs) / k;
+      if (cost < best_cost - 1e-9) { best_cost = cost; best = k; }
+    }
+  }
+  if (best > ntiles) best = ntiles;
+  if (best < 1) best = 1;
+  int tps = (ntiles + best - 1) / best;
+  if (tps < 1) tps = 1;
+  *tiles_per_split = tps;
+  const int s = (ntiles + tps - 1) / tps;
+  return s > 0 ? s : 1;
+}
+
 int tc_splits(int M, int Hkv, int nseq, int ntiles, int* tiles_per_split) {
   const int nqblk = (M + 127) / 128;
-  int s = 148 / (nqblk * Hkv * nseq);          // one CTA per SM, one wave
-  if (s < 1) s = 1;
-  if (s > ntiles) s = ntiles;
-  if (s < 1) s = 1;
-  *tiles_per_split = (ntiles + s - 1) / s;
-  if (*tiles_per_split < 1) *tiles_per_split = 1;
-  return (ntiles + *tiles_per_split - 1) / *tiles_per_split > 0 ? (ntiles + *tiles_per_split - 1) / *tiles_per_split : 1;
+  return balanced_splits(nqblk * Hkv * nseq, ntiles, tiles_per_split);
 }
 
 // upper bound of the number of attention partials per query row (workspace sizing)
@@ -187,8 +210,8 @@ int splits_bound(int M, int Hkv) {
   int s = (2 * 148 + nqblk * Hkv - 1) / (nqblk * Hkv);
   if (s < 1) s = 1;
   if (s > KVS_MAX_SPLITS) s = KVS_MAX_SPLITS;
-  int tc = 148 / (nqblk * Hkv);
-  if (tc < 1) tc = 1;
+  int tc = kNumSMs / (nqblk * Hkv);
+  if (tc < kMaxTcSplits) tc = kMaxTcSplits;
   tc *= 2;                                      // two softmax groups per CTA
   return s > tc ? s : tc;
 }
@@ -397,11 +420,7 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
     int pmax = 0;
     for (int i = 0; i < tab.nseq; ++i) pmax = pmax > tab.s[i].P ? pmax : tab.s[i].P;
     const int ntiles = (pmax + 127) / 128;               // tiles of 128 candidate pairs
-    int splits = 148 / (ta.nqblk * ta.Hkv * tab.nseq);
-    if (splits < 1) splits = 1;
-    if (splits > ntiles) splits = ntiles;
-    ta.tiles_per_split = (ntiles + splits - 1) / splits;
-    ta.splits = (ntiles + ta.tiles_per_split - 1) / ta.tiles_per_split;
+    ta.splits = balanced_splits(ta.nqblk * ta.Hkv * tab.nseq, ntiles, &ta.tiles_per_split);
     ta.n_max = view.n_max; ta.pair_stride = c.L.pair_stride;
     ta.scale_log2 = scale_log2; ta.score_mode = p->score_mode;
     ta.counts = view.counts; ta.qc2 = ca.qc2; ta.M_pad = ca.M_pad;
