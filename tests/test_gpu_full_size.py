@@ -1,0 +1,93 @@
+"""Parity at the benchmark's full sequence length and in its launch configuration: layers folded
+into the batch, 32768-token caches of the Llama-3.1-8B layout (8 KV heads, 4 x 64 window rows).
+The oracle cannot redo all of it in a test, so sampled (layer, KV head) units are checked
+element by element and everything else through properties that hold at any size."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import kvs_oracle as oc
+from paper_2603_00907_b200 import workloads as wl
+from tests import kvs_testlib as tl
+
+pytestmark = pytest.mark.gpu
+
+LAYERS = 5          # 5 x 8 = 40 units: fewer than the SMs, so the launch also cuts key ranges
+
+
+@pytest.fixture(scope="module")
+def setup():
+    import torch
+    from paper_2603_00907_b200 import binding as kb, build
+    build.build()
+    w = wl.config(1)
+    layers = [wl.make_layer(w.scaled(n_decode=1), l) for l in range(LAYERS)]
+    cat = lambda k: np.concatenate([d[k] for d in layers], axis=0)
+    data = {k: cat(k) for k in ("K", "V", "counts", "q_win", "q_new")}
+    dev = tl.upload_layer(data)
+    p = kb.make_params(dev["K"], dev["V"], w.n_q_heads, w.window, sink=w.sink, round_frac=w.round_frac)
+    ws = torch.empty(kb.kvs_workspace_size(p, w.n_max, 1), dtype=torch.uint8, device="cuda")
+    return kb, w, data, dev, p, ws
+
+
+def test_round0_statistics_of_sampled_units(setup):
+    import torch
+    kb, w, data, dev, p, ws = setup
+    B, Hkv, Nmax, G = LAYERS, w.n_kv_heads, w.n_max, w.group
+    f32 = dict(dtype=torch.float32, device="cuda")
+    A, N1 = torch.zeros((B, Hkv, Nmax), **f32), torch.zeros((B, Hkv, Nmax), **f32)
+    N12, score = torch.zeros((B, Hkv, Nmax // 2), **f32), torch.zeros((B, Hkv, Nmax // 2), **f32)
+    mask = torch.zeros((B, Hkv, Nmax // 2), dtype=torch.uint8, device="cuda")
+    n, bud = w.seq_lens[0], w.budgets[0]
+    kb.kvs_window_stats(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], [n] * B, [bud] * B, ws,
+                        A=A, N1=N1, N12=N12, score=score, mask=mask)
+    torch.cuda.synchronize()
+    for (b, h) in ((0, 0), (3, 5)):
+        st = oc.round_stats(data["K"][b, h, :n], data["V"][b, h, :n], data["counts"][b, h, :n].astype(np.int64),
+                            data["q_win"][b, h * G:(h + 1) * G], bud, 0, window=w.window, sink=w.sink,
+                            recent=w.window, scale=1 / math.sqrt(128), causal=True, round_frac=w.round_frac,
+                            score_mode=0)
+        off, P, R = st["off"], st["P"], st["R"]
+        sl = slice(off, off + 2 * P)
+        for name, g, ref in (("A", A[b, h, sl], st["A"][sl]), ("N1", N1[b, h, sl], st["N1"][sl]),
+                             ("N12", N12[b, h, :P], st["N12"]), ("score", score[b, h, :P], st["score"])):
+            ok, ratio, plain = tl.stat_close(g.cpu().numpy(), ref)
+            assert ok, f"{name} unit {(b, h)}: err/allowed {ratio:.3g}, plain rel {plain:.3g}"
+        ok, nm, nout = tl.mask_band_ok(mask[b, h, :P].cpu().numpy(), st["mask"], st["score"], R)
+        assert ok, f"mask unit {(b, h)}: {nm} mismatches, {nout} outside the band"
+
+
+def test_full_pass_properties_and_sampled_decode(setup):
+    import torch
+    kb, w, data, dev, p, ws = setup
+    B, Hkv, G = LAYERS, w.n_kv_heads, w.group
+    n, bud = w.seq_lens[0], w.budgets[0]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    new_len = kb.kvs_merge_layer(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], [n] * B, [bud] * B, ws,
+                                 status_dev=status)
+    out = torch.zeros((B, w.n_q_heads, 1, 128), dtype=torch.bfloat16, device="cuda")
+    kb.kvs_decode_attn(p, dev["q_new"], dev["K"], dev["V"], dev["counts"], new_len, out, ws)
+    torch.cuda.synchronize()
+    assert status.item() == 0 and new_len == [bud] * B
+    Kg, Vg, Cg = tl.bits_of(dev["K"]), tl.bits_of(dev["V"]), dev["counts"].cpu().numpy()
+    og = tl.bits_of(out)
+    # properties that hold for every unit: the budget is met, every token is still counted, the
+    # protected prefix and suffix are untouched, value sums are conserved up to bf16 rounding
+    for b in range(B):
+        for h in range(Hkv):
+            c = Cg[b, h, :bud]
+            assert int(c.sum()) == n and c.min() >= 1
+            assert np.array_equal(Kg[b, h, :w.sink], data["K"][b, h, :w.sink])
+            assert np.array_equal(Kg[b, h, bud - w.window:bud], data["K"][b, h, n - w.window:n])
+            assert np.array_equal(Vg[b, h, bud - w.window:bud], data["V"][b, h, n - w.window:n])
+            assert np.all(c[:w.sink] == 1) and np.all(c[bud - w.window:] == 1)
+            tot = oc.bf16_to_f64(data["V"][b, h, :n]).sum(0)
+            got = oc.bf16_to_f64(Vg[b, h, :bud]).sum(0)
+            assert np.max(np.abs(got - tot)) < 0.02 * math.sqrt(n)      # bf16 roundings of ~n merges
+    # sampled units: decode over the GPU's merged cache against the oracle's attention
+    for (b, h) in ((1, 2), (4, 7)):
+        ref, _ = oc.decode_attention(data["q_new"][b, h * G:(h + 1) * G], Kg[b, h, :bud], Vg[b, h, :bud],
+                                     Cg[b, h, :bud])
+        ok, mx, _, _ = tl.bf16_close(og[b, h * G:(h + 1) * G], oc.f64_to_bf16(ref))
+        assert ok, mx

@@ -474,3 +474,29 @@ def test_noop_and_error_paths_on_device(kb):
     assert e.value.code == 3
     torch.cuda.synchronize()
     assert np.array_equal(tl.bits_of(dev["K"]), before)
+
+
+def test_window_stats_config_layouts(kb):
+    """The head layouts of the other benchmark configurations at reduced length: Qwen (7 query
+    heads per KV head, 224 window rows: a partial second query block), the 70B layout (8 x 128 =
+    1024 rows: eight query blocks), and a ragged batch of eight sequences."""
+    for seed, kw in ((14, dict(batch=1, n_q_heads=14, n_kv_heads=2, window=32, seq_lens=(1100,), budgets=(400,))),
+                     (15, dict(batch=1, n_q_heads=8, n_kv_heads=1, window=128, seq_lens=(1500,), budgets=(600,))),
+                     (16, dict(batch=8, n_q_heads=8, n_kv_heads=2, window=16,
+                               seq_lens=(300, 1201, 517, 64, 900, 433, 1000, 777),
+                               budgets=(37, 150, 64, 64, 112, 54, 125, 97)))):
+        w = _small(seed=seed, **kw)
+        data = wl.make_layer(w)
+        for r in (0, 1):
+            _check_round_stats(kb, w, data["K"], data["V"], data["counts"], data["q_win"], list(w.seq_lens), r)
+
+
+def test_merged_counts_statistics(kb):
+    """Statistics on a cache that already holds merged slots (counts > 1 carry the logit bias ln c
+    and divide the value sums)."""
+    w = _small(seed=17, batch=1, n_q_heads=8, n_kv_heads=2, window=16, seq_lens=(1300,), budgets=(300,))
+    data = wl.make_layer(w)
+    rng = np.random.default_rng(3)
+    data["counts"][:] = rng.integers(1, 5, size=data["counts"].shape)
+    _check_round_stats(kb, w, data["K"], data["V"], data["counts"], data["q_win"], list(w.seq_lens), 0)
+    _check_round_stats(kb, w, data["K"], data["V"], data["counts"], data["q_win"], list(w.seq_lens), 1)
