@@ -38,7 +38,7 @@ constexpr int kSmemMisc = 7 * kOperand;
 constexpr int kThreads = 320;              // warp 0: TMA, warp 1: MMA, warps 2-9: statistics
 
 struct Misc {
-  uint64_t full, stage_free, tfull[2], tfree[2], qfull, xready, xfree;
+  uint64_t kfull, vfull, kfree, vfree, tfull[2], tfree[2], qfull, xready, xfree;
   uint32_t tmem_base;
   int abort_flag;
   float xbuf[kPairs * 5];                  // partial sums of the second statistics group, for the first
@@ -116,8 +116,12 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    mbar_init(&misc->full, 1);
-    mbar_init(&misc->stage_free, 1);       // MMA commit
+    // the staged K rows are free once the last logits are formed, the Vsum rows only after the last
+    // T product: each operand is requested again as soon as its own buffer is free
+    mbar_init(&misc->kfull, 1);
+    mbar_init(&misc->vfull, 1);
+    mbar_init(&misc->kfree, 1);            // MMA commit
+    mbar_init(&misc->vfree, 1);            // MMA commit
     for (int s = 0; s < 2; ++s) {
       mbar_init(&misc->tfull[s], 1);
       mbar_init(&misc->tfree[s], 8);       // statistics warps
@@ -149,23 +153,54 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
         tma_load_3d(smem + kSmemOhi + hf * kHalf, &tmOhi, &misc->qfull, hf * 64, qblk * kQB, unit);
         tma_load_3d(smem + kSmemOlo + hf * kHalf, &tmOlo, &misc->qfull, hf * 64, qblk * kQB, unit);
       }
-      int issued = 0;
-      for (int li = 0; li < my_tiles; ++li) {
-        if (!mbar_wait(&misc->stage_free, (li & 1) ^ 1, abort_flag)) break;
+      // one thread streams both operands; every tile is first requested into L2 one tile ahead,
+      // so that the load that fills the (single) stage finds it there
+      auto prefetch = [&](int li, bool v) {
         const int p0 = (t_begin + li) * kPairs;
-        mbar_expect_tx(&misc->full, 4 * kOperand);
+        const CUtensorMap* tm = v ? &tmVp : &tmKp;
         for (int hf = 0; hf < 2; ++hf) {
-          tma_load_5d(smem + kSmemKl + hf * kHalf, &tmKp, &misc->full, hf * 64, par_l, rho_l0 + p0, h, sr.b);
-          tma_load_5d(smem + kSmemKr + hf * kHalf, &tmKp, &misc->full, hf * 64, par_r, rho_r0 + p0, h, sr.b);
-          tma_load_5d(smem + kSmemVl + hf * kHalf, &tmVp, &misc->full, hf * 64, par_l, rho_l0 + p0, h, sr.b);
-          tma_load_5d(smem + kSmemVr + hf * kHalf, &tmVp, &misc->full, hf * 64, par_r, rho_r0 + p0, h, sr.b);
+          tma_prefetch_5d(tm, hf * 64, par_l, rho_l0 + p0, h, sr.b);
+          tma_prefetch_5d(tm, hf * 64, par_r, rho_r0 + p0, h, sr.b);
         }
-        issued = li + 1;
+      };
+      int kli = 0, vli = 0;
+      uint64_t t0 = globaltimer_ns();
+      while (kli < my_tiles || vli < my_tiles) {
+        bool progress = false;
+        if (kli < my_tiles && mbar_try_wait(&misc->kfree, (kli & 1) ^ 1)) {
+          const int p0 = (t_begin + kli) * kPairs;
+          mbar_expect_tx(&misc->kfull, 2 * kOperand);
+          for (int hf = 0; hf < 2; ++hf) {
+            tma_load_5d(smem + kSmemKl + hf * kHalf, &tmKp, &misc->kfull, hf * 64, par_l, rho_l0 + p0, h, sr.b);
+            tma_load_5d(smem + kSmemKr + hf * kHalf, &tmKp, &misc->kfull, hf * 64, par_r, rho_r0 + p0, h, sr.b);
+          }
+          if (kli + 1 < my_tiles) prefetch(kli + 1, false);
+          ++kli;
+          progress = true;
+        }
+        if (vli < my_tiles && mbar_try_wait(&misc->vfree, (vli & 1) ^ 1)) {
+          const int p0 = (t_begin + vli) * kPairs;
+          mbar_expect_tx(&misc->vfull, 2 * kOperand);
+          for (int hf = 0; hf < 2; ++hf) {
+            tma_load_5d(smem + kSmemVl + hf * kHalf, &tmVp, &misc->vfull, hf * 64, par_l, rho_l0 + p0, h, sr.b);
+            tma_load_5d(smem + kSmemVr + hf * kHalf, &tmVp, &misc->vfull, hf * 64, par_r, rho_r0 + p0, h, sr.b);
+          }
+          if (vli + 1 < my_tiles) prefetch(vli + 1, true);
+          ++vli;
+          progress = true;
+        }
+        if (progress) {
+          t0 = globaltimer_ns();
+        } else {
+          if (*abort_flag) break;
+          if (globaltimer_ns() - t0 > 1000000000ull) { *abort_flag = 1; break; }
+        }
       }
-      if (*abort_flag && issued > 0) {
+      if (*abort_flag) {
         // drain: give the copies already issued a bounded time to land before the CTA leaves
-        const uint64_t t0 = globaltimer_ns();
-        while (!mbar_try_wait(&misc->full, (issued - 1) & 1) && globaltimer_ns() - t0 < 200000000ull) {}
+        const uint64_t t1 = globaltimer_ns();
+        while (kli > 0 && !mbar_try_wait(&misc->kfull, (kli - 1) & 1) && globaltimer_ns() - t1 < 200000000ull) {}
+        while (vli > 0 && !mbar_try_wait(&misc->vfull, (vli - 1) & 1) && globaltimer_ns() - t1 < 200000000ull) {}
       }
     }
   } else if (warp == 1) {
@@ -178,7 +213,7 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
                      vl = smem_u32(smem + kSmemVl), vr = smem_u32(smem + kSmemVr);
       bool ok = mbar_wait(&misc->qfull, 0, abort_flag);
       for (int li = 0; ok && li < my_tiles; ++li) {
-        if (!mbar_wait(&misc->full, li & 1, abort_flag)) break;
+        if (!mbar_wait(&misc->kfull, li & 1, abort_flag)) break;
         for (int hq = 0; hq < nh; ++hq) {
           if (!mbar_wait(&misc->tfree[hq], (li & 1) ^ 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
@@ -194,6 +229,8 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
             const uint32_t o = (kk >> 2) * kHalf + (kk & 3) * 32;
             umma_bf16(d0 + 64, smem_desc_sw128(kr + o, 16, 1024), smem_desc_sw128(q_addr + qrow + o, 16, 1024), idesc, kk > 0);
           }
+          if (hq == nh - 1) tc_commit(&misc->kfree);
+          if (hq == 0 && !mbar_wait(&misc->vfull, li & 1, abort_flag)) { ok = false; break; }
 #pragma unroll
           for (int kk = 0; kk < 16; ++kk) {
             const uint32_t o = ((kk & 7) >> 2) * kHalf + (kk & 3) * 32;
@@ -209,7 +246,7 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
           tc_commit(&misc->tfull[hq]);
         }
         if (!ok) break;
-        tc_commit(&misc->stage_free);
+        tc_commit(&misc->vfree);
       }
     }
   } else {
