@@ -83,6 +83,32 @@ class ClockSampler(threading.Thread):
                 "reasons": sorted(reasons), "samples": len(sm), "scope": scope}
 
 
+# DRAM traffic of each kernel kind as a multiple of its algorithmic bytes, from the ncu captures
+# summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of rounds 0 and 1 of a
+# 10-layer case, whose inputs exceed L2; traffic grows with the units processed, so the ratio
+# carries over to a full launch).  Each entry names the kernel source it was taken on: once that
+# file changes, the figure is stale and `traffic` is reported as null.
+NCU_TRAFFIC = {
+    "hessian_stats": (1.03, "kvs_stats_tc.cu", "000b7e86f391e522"),
+    "attn_partials": (1.01, "kvs_flash_tc.cu", "6a793f0316d260fb"),
+    "merge_compact": (0.98, "kvs_compact.cu", "c28752d898c08b93"),
+}
+
+
+def ncu_traffic_ratio(kind):
+    import hashlib
+    if kind not in NCU_TRAFFIC:
+        return None
+    ratio, fname, digest = NCU_TRAFFIC[kind]
+    path = os.path.join(ROOT, "paper_2603_00907_b200", "csrc", fname)
+    try:
+        with open(path, "rb") as f:
+            now = hashlib.sha256(f.read()).hexdigest()[:16]
+    except OSError:
+        return None
+    return ratio if now == digest else None
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -115,8 +141,10 @@ def algorithmic_bytes(w, n_layers):
     kept = sum(n - R for pl in plans for (n, _, _, R) in pl) * w.n_kv_heads * n_layers
     pairs = sum(P for pl in plans for (_, _, P, _) in pl) * w.n_kv_heads * n_layers
     return {
-        "attn_partials": slots * ROW_BYTES,
-        "hessian_stats": slots * ROW_BYTES + pairs * 8,
+        # every slot read once; the pair norms (16 B per candidate pair) written
+        "attn_partials": slots * ROW_BYTES + pairs * 16,
+        # the candidate slots read once, the pair norms read, score and weight written
+        "hessian_stats": 2 * pairs * ROW_BYTES + pairs * (16 + 8),
         "select": pairs * (4 + 1),
         "merge_compact": slots * ROW_BYTES + kept * ROW_BYTES + pairs * 5,
     }, slots
@@ -346,14 +374,30 @@ def main():
     peak, peak_src = measured_peaks()
     top_ms, top_launches = kinds[top]
     achieved = alg.get(top, 0) * n_prof / (top_ms * 1e-3) / 1e9 if top in alg else None
+    ratio = ncu_traffic_ratio(top)
+    traffic = (ratio * alg.get(top, 0) * n_prof / top_launches) if (ratio and top in alg) else None
     roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": (achieved / peak) if achieved else None, "traffic": None,
+                "frac": (achieved / peak) if achieved else None, "traffic": traffic,
                 "peak_source": f"of {peak_src}",
                 "avg_launch_us": 1e3 * top_ms / top_launches,
                 "algorithmic_bytes_per_launch": alg.get(top, 0) * n_prof / top_launches,
                 "per_kernel": {k: {"ms_per_step": v[0] / n_prof, "launches_per_step": v[1] // n_prof,
                                    "GBps": (alg[k] * n_prof / (v[0] * 1e-3) / 1e9) if k in alg else None}
                                for k, v in kinds.items()}}
+
+    # The two attention-shaped kernels are, at this window size, limited by the 16-lane special
+    # function pipe rather than by HBM: report that roofline beside the HBM one.  Peak = 148 SMs x
+    # 16 lanes x the maximum SM clock; operations per (window query, slot) element: statistics
+    # 2.5 (one exp2, 1.5 square roots), attention 1.5 (one exp2, half a pack conversion).
+    plans = plan_rounds(w)
+    M = w.group * W
+    sfu_peak = 148 * 16 * (clocks.get("sm_max_mhz") or 1965.0) * 1e6
+    for kind, per_elem, count in (("hessian_stats", 2.5, lambda n, P: 2 * P), ("attn_partials", 1.5, lambda n, P: n)):
+        if kind in kinds:
+            elems = sum(count(n, P) for pl in plans for (n, _, P, _) in pl) * Hkv * L * M
+            ops_per_s = per_elem * elems / (kinds[kind][0] / n_prof * 1e-3)
+            roofline["per_kernel"][kind]["sfu"] = {"bound": "alu", "achieved": ops_per_s / 1e12, "peak": sfu_peak / 1e12,
+                                                   "unit": "Tops/s", "frac": ops_per_s / sfu_peak}
 
     # ---- end to end through the C ABI with host buffers
     e2e = None
