@@ -40,35 +40,24 @@ struct Misc {
   uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[2], sfree[2], pready[2], ofull[2], qfull;
   uint32_t tmem_base;
   int abort_flag;
-  int wg_fail[2];
-  alignas(16) float cnt[2][64];            // per group: counts of the half tile's slots (read as float4)
+  alignas(16) float cnt[2][2][64];         // per tile parity and group: counts of the half tile's slots (read as float4)
 };
 constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc) + 1024;
 
 __device__ __forceinline__ void wg_barrier(int wg) {
   asm volatile("bar.sync %0, 128;" ::"r"(wg + 1) : "memory");
 }
-// OR over the 128 threads of a group, with barrier semantics.
-__device__ __forceinline__ bool wg_any(int wg, bool pred) {
-  uint32_t out;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
-      "setp.ne.u32 p, %2, 0;\n\t"
-      "bar.red.or.pred q, %1, 128, p;\n\t"
-      "selp.u32 %0, 1, 0, q;\n\t}"
-      : "=r"(out)
-      : "r"(wg + 1), "r"((uint32_t)pred)
-      : "memory");
-  return out != 0;
+// One lane polls, the warp follows.  A failed wait (time-out or abort) only makes the warp skip
+// its work: it still goes through the tile loop and its one named barrier per tile, so that no
+// other warp can be left waiting for it.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int lane) {
+  int ok = 1;
+  if (lane == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
-__device__ __forceinline__ bool wg_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                        volatile int* wg_fail, int wg, int lane) {
-  if (lane == 0) {
-    if (!mbar_wait(bar, parity, abort_flag)) *wg_fail = 1;
-  }
+__device__ __forceinline__ void warp_arrive(uint64_t* bar, int lane) {
   __syncwarp();
-  wg_barrier(wg);
-  return *wg_fail == 0;
+  if (lane == 0) mbar_arrive(bar);
 }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
   asm volatile(
@@ -203,13 +192,12 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       mbar_init(&misc->kfree[s], norm_k ? 3 : 1);       // MMA commit (+ the two pair-norm warps)
       mbar_init(&misc->vfree[s], norm_v ? 3 : 1);
       mbar_init(&misc->sfull[s], 1);
-      mbar_init(&misc->sfree[s], 2);
-      mbar_init(&misc->pready[s], 1);
+      mbar_init(&misc->sfree[s], 8);                    // softmax warps
+      mbar_init(&misc->pready[s], 4);                   // warps of one group
       mbar_init(&misc->ofull[s], 1);
     }
     mbar_init(&misc->qfull, 1);
     misc->abort_flag = 0;
-    misc->wg_fail[0] = misc->wg_fail[1] = 0;
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc(&misc->tmem_base, 512);
@@ -389,45 +377,51 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     for (int li = 0; li < my_tiles; ++li) {
       const int s = li & 1, k = li >> 1;
       const int j0 = (t_begin + li) * kTile - shift + wg * 64;    // first slot of this group's half tile
+      float* cnt = misc->cnt[s][wg];
       if (t128 < 64) {
-        misc->cnt[wg][t128] = (float)cnt_next;
+        cnt[t128] = (float)cnt_next;
         const int j = j0 + kTile + t128;
         cnt_next = (li + 1 < my_tiles && j >= 0 && j < n) ? Cb[j] : 1;
       }
-      if (!wg_wait(&misc->sfull[s], k & 1, abort_flag, &misc->wg_fail[wg], wg, lane)) { alive = false; break; }
-      tc_fence_after();
       float x[64];
-      tmem_ld32(tmem + lane_addr + s * 128 + wg * 64, x);
-      tmem_ld32(tmem + lane_addr + s * 128 + wg * 64 + 32, x + 32);
-      tmem_ld_wait();
-      tc_fence_before();
-      wg_barrier(wg);
-      if (t128 == 0) mbar_arrive(&misc->sfree[s]);
-      // logits in log2 units, with mask (the stabiliser ignores the counts: exp(s - m) <= 1 either way)
       float mt = -INFINITY;
-      const bool need_mask = (j0 < 0) || (j0 + 63 > min(n - 1, a.causal ? n - a.Wq : n - 1));
-      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one
-      if (!need_mask) {
+      if (alive) alive = warp_wait(&misc->sfull[s], k & 1, abort_flag, lane);
+      if (alive) {
+        tc_fence_after();
+        tmem_ld32(tmem + lane_addr + s * 128 + wg * 64, x);
+        tmem_ld32(tmem + lane_addr + s * 128 + wg * 64 + 32, x + 32);
+        tmem_ld_wait();
+        tc_fence_before();
+        warp_arrive(&misc->sfree[s], lane);
+        // logits in log2 units, with mask (the stabiliser ignores the counts: exp(s - m) <= 1 either way)
+        const bool need_mask = (j0 < 0) || (j0 + 63 > min(n - 1, a.causal ? n - a.Wq : n - 1));
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one
+        if (!need_mask) {
 #pragma unroll
-        for (int i = 0; i < 64; ++i) {
-          x[i] *= a.scale_log2;
-          mx[i & 3] = fmaxf(mx[i & 3], x[i]);
-        }
-      } else {
+          for (int i = 0; i < 64; ++i) {
+            x[i] *= a.scale_log2;
+            mx[i & 3] = fmaxf(mx[i & 3], x[i]);
+          }
+        } else {
 #pragma unroll
-        for (int i = 0; i < 64; ++i) {
-          const float v = x[i] * a.scale_log2;
-          x[i] = (j0 + i >= 0 && j0 + i <= last_vis) ? v : -INFINITY;
-          mx[i & 3] = fmaxf(mx[i & 3], x[i]);
+          for (int i = 0; i < 64; ++i) {
+            const float v = x[i] * a.scale_log2;
+            x[i] = (j0 + i >= 0 && j0 + i <= last_vis) ? v : -INFINITY;
+            mx[i & 3] = fmaxf(mx[i & 3], x[i]);
+          }
         }
+        mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
       }
-      mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+      // the one barrier of the tile: the counts staged above are visible to the whole group, and
+      // every warp has finished reading the buffer that the tile after next will overwrite
+      wg_barrier(wg);
+      if (!alive) continue;
       const float m_new = fmaxf(m_stab, mt);
       const bool need = m_new > m_stab + kRescaleGap || (m_stab == -INFINITY && m_new > -INFINITY);
-      const bool any_need = wg_any(wg, need && li > 0);
+      const bool any_need = __any_sync(0xffffffffu, need && li > 0);
       // the previous tile's P V product must be done before P is overwritten (and before a rescale)
       if (li > 0) {
-        if (!wg_wait(&misc->ofull[wg], (li - 1) & 1, abort_flag, &misc->wg_fail[wg], wg, lane)) { alive = false; break; }
+        if (!(alive = warp_wait(&misc->ofull[wg], (li - 1) & 1, abort_flag, lane))) continue;
         tc_fence_after();
       }
       if (any_need) {
@@ -453,8 +447,8 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         uint32_t hi[4], lo[4];
-        const float4 ca = *reinterpret_cast<const float4*>(&misc->cnt[wg][c * 8]);
-        const float4 cb = *reinterpret_cast<const float4*>(&misc->cnt[wg][c * 8 + 4]);
+        const float4 ca = *reinterpret_cast<const float4*>(&cnt[c * 8]);
+        const float4 cb = *reinterpret_cast<const float4*>(&cnt[c * 8 + 4]);
         const float cc[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
@@ -470,10 +464,10 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         *reinterpret_cast<uint4*>(pbuf + kHalf + off16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
       }
       l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-      // rows of the V tile outside the sequence may hold anything: zero them
+      // rows of the V tile outside the sequence may hold anything: each warp zeroes its share
       const int tile_row0 = (t_begin + li) * kTile - shift;
       if (tile_row0 < 0 || tile_row0 + kTile > n) {
-        if (!wg_wait(&misc->vfull[s], k & 1, abort_flag, &misc->wg_fail[wg], wg, lane)) { alive = false; break; }
+        if (!(alive = warp_wait(&misc->vfull[s], k & 1, abort_flag, lane))) continue;
         uint8_t* vt = smem + kSmemStage + s * kStage + kOperand;
         for (int it = wg * 64 * 16 + t128; it < (wg * 64 + 64) * 16; it += 128) {
           const int r = it >> 4, ch = it & 15;
@@ -483,11 +477,10 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       }
       fence_proxy_async();
       tc_fence_before();
-      wg_barrier(wg);
-      if (t128 == 0) mbar_arrive(&misc->pready[wg]);
+      warp_arrive(&misc->pready[wg], lane);
     }
     // ---- the partial of this (split, group)
-    if (alive && wg_wait(&misc->ofull[wg], (my_tiles - 1) & 1, abort_flag, &misc->wg_fail[wg], wg, lane)) {
+    if (alive && warp_wait(&misc->ofull[wg], (my_tiles - 1) & 1, abort_flag, lane)) {
       tc_fence_after();
       const size_t pidx = ((size_t)unit * (a.splits * 2) + split * 2 + wg) * a.M + m;
       if (m < a.M) a.part_ml[pidx] = make_float2(m_stab, l);
