@@ -212,7 +212,6 @@ int splits_bound(int M, int Hkv) {
   if (s > KVS_MAX_SPLITS) s = KVS_MAX_SPLITS;
   int tc = kNumSMs / (nqblk * Hkv);
   if (tc < kMaxTcSplits) tc = kMaxTcSplits;
-  tc *= 2;                                      // two softmax groups per CTA
   return s > tc ? s : tc;
 }
 
@@ -343,7 +342,7 @@ kvs_status_t enqueue_flash(const kvs_params_t* p, char* ws, const WsLayout& L, c
   ta.Wq = Wq; ta.causal = causal; ta.scale_log2 = scale_log2;
   ta.n_max = view.n_max; ta.counts = view.counts;
   ta.part_ml = part_ml; ta.part_o = part_o; ta.status_dev = status_dev;
-  *n_part = ta.splits * 2;
+  *n_part = ta.splits;
   return launch_fn([&] { return kvs_launch_flash_tc(ta, tab, tmK, tmV, tmQ, st); });
 }
 

@@ -1,21 +1,23 @@
 // Attention partials on the tensor cores (tcgen05 + TMEM + TMA), queries on TMEM lanes.
 //
 // One CTA owns a block of 128 query rows (Q stays in shared memory) and a contiguous range
-// of 128-slot tiles.  Per tile, TMA brings the K and V rows and one thread issues
+// of 128-slot tiles.  K and V tiles travel in two separate two-stage TMA rings; per tile one
+// thread issues
 //   S[q, slot] = Q K_tile^T                         (fp32 in TMEM, double buffered)
-// Two groups of four warps each take 64 of the tile's slots.  A thread owns one query row:
-// it applies the causal/tail mask, keeps a running stabiliser m and the sum
-// l = sum_j c_j exp(s_j - m) (the count bias ln c_j of a merged slot is the factor c_j), and
-// writes P' = exp(s - m) = alpha_j l / c_j, split into two bf16 terms, to shared memory.
-// The same issuing thread then runs, per group,
-//   O_g[q, :] += (P'_hi + P'_lo) Vsum_tile          (V as the MN-major operand)
-// with O_g accumulating in TMEM across the tiles [Eq. attn_def_vec with merged slots:
-// o = sum_j alpha_j Vsum_j / c_j].  The stabiliser only moves when the row maximum grows by
-// more than 2^8, in which case the group rescales its O_g rows in TMEM; otherwise O is never
-// touched until the end, where (stabiliser, sum, O) is written as the partial of this
-// (key split, group).  Window queries and decode queries use the same kernel.
+// Sixteen softmax warps share the tile: the four warps of a TMEM lane quarter own the same 32
+// query rows and 32 slot columns each.  A thread finds the maximum of its 32 logits; the four
+// threads of a row agree on the row maximum through a shared-memory atomic maximum, keep the
+// same stabiliser m (it only moves when the maximum grows by more than 2^8, in which case the
+// first of the four rescales the row of O in TMEM), and each writes P' = exp(s - m), split
+// into two bf16 terms, to shared memory, keeping its part of l = sum_j c_j exp(s_j - m): the
+// count bias ln c_j of a merged slot is just the factor c_j in that sum.  The issuing thread
+// then runs
+//   O[q, :] += (P'_hi + P'_lo) Vsum_tile            (V as the MN-major operand)
+// with O accumulating in TMEM across the tiles [Eq. attn_def_vec with merged slots:
+// o = sum_j alpha_j Vsum_j / c_j].  At the end (stabiliser, sum, O) is written as the partial
+// of this key range.  Window queries and decode queries use the same kernel.
 //
-// Two more warps serve the statistics pass that follows the window attention: tiles are then
+// Four more warps serve the statistics pass that follows the window attention: tiles are then
 // aligned with the round's candidate pairs, and for every pair they form |vbar_l|^2, |vbar_r|^2,
 // |vbar_l + vbar_r|^2 and the adjacent-key cosine from the staged rows (diagonals of small
 // mma.sync products), so that the statistics kernel does not have to touch the rows for it.
@@ -30,23 +32,40 @@ constexpr int kTile = 128;
 constexpr int kHalf = 16384;               // [128 rows x 64 bf16], 128-byte swizzle
 constexpr int kOperand = 2 * kHalf;
 constexpr int kStage = 2 * kOperand;       // K tile + V tile
-constexpr int kPGroup = 2 * kHalf;         // P'_hi and P'_lo of one group: [128 q x 64 slots] each
+constexpr int kPGroup = 2 * kHalf;         // P'_hi and P'_lo of 64 slots: [128 q x 64 slots] each
 constexpr int kSmemQ = 0, kSmemStage = kOperand, kSmemP = kSmemStage + 2 * kStage;
 constexpr int kSmemMisc = kSmemP + 2 * kPGroup;
-constexpr int kThreads = 384;              // warp 0: TMA, 1: MMA, 2-9: softmax, 10-11: pair norms
+constexpr int kSoftmaxWarps = 16, kNormWarps = 4;
+constexpr int kThreads = (2 + kSoftmaxWarps + kNormWarps) * 32;   // warp 0: TMA, 1: MMA, 2-17: softmax, 18-21: pair norms
 constexpr float kRescaleGap = 8.f;         // log2 units
 
 struct Misc {
-  uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[2], sfree[2], pready[2], ofull[2], qfull;
+  uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[2], sfree[2], pready, ofull, qfull;
   uint32_t tmem_base;
   int abort_flag;
-  alignas(16) float cnt[2][2][64];         // per tile parity and group: counts of the half tile's slots (read as float4)
+  union {
+    struct {
+      uint32_t rowmax[3][kTile];           // per tile (mod 3) and query row: maximum logit, as an ordered integer
+      alignas(16) float cnt[2][kTile];     // per tile parity: counts of the tile's slots (read as float4)
+    };
+    float lsum[4][kTile];                  // after the last tile: the column groups' parts of the row sums
+  };
 };
-constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc) + 1024;
+constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc);
+static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 
-__device__ __forceinline__ void wg_barrier(int wg) {
-  asm volatile("bar.sync %0, 128;" ::"r"(wg + 1) : "memory");
+constexpr uint32_t kOrdNegInf = 0x007fffffu;   // ordered-integer image of -infinity
+// monotone map float -> unsigned (so that an integer maximum is the float maximum) and back
+__device__ __forceinline__ uint32_t f2ord(float f) {
+  const uint32_t b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
+__device__ __forceinline__ float ord2f(uint32_t u) {
+  return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
+}
+
+__device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 1, 512;" ::: "memory"); }
+
 // One lane polls, the warp follows.  A failed wait (time-out or abort) only makes the warp skip
 // its work: it still goes through the tile loop and its one named barrier per tile, so that no
 // other warp can be left waiting for it.
@@ -99,57 +118,40 @@ __device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], 
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// For the 32 pairs (rows 2i, 2i+1) of rows [64 * half, 64 * half + 64) of one staged operand:
-// |x_l|^2, |x_r|^2 and <x_l, x_r>, delivered to lane i.  Eight pairs at a time,
-// A = [x_l rows ; x_r rows] (16 x 128) against B = x_r and B = x_l (8 rows each): the wanted
-// values are diagonal elements of the two 16 x 8 products.  Two blocks of eight pairs are in
-// flight at once: all their fragments are loaded first, then four independent accumulation
-// chains run through the tensor cores.
-__device__ __forceinline__ void pair_dots(const uint8_t* tile, int half, int lane, float& ll, float& rr, float& lr) {
+// For the 8 pairs (rows 2i, 2i+1) of rows [row0, row0 + 16) of one staged operand: |x_l|^2,
+// |x_r|^2 and <x_l, x_r>, delivered to lanes 0-7.  A = [x_l rows ; x_r rows] (16 x 128) against
+// B = x_r and B = x_l (8 rows each): the wanted values are diagonal elements of the two
+// 16 x 8 products.  All fragments are loaded first, then two accumulation chains run.
+__device__ __forceinline__ void pair_dots8(const uint8_t* tile, int row0, int lane, float& ll, float& rr, float& lr) {
   const uint32_t base = smem_u32(tile);
   const int mtx = lane >> 3, rin = lane & 7;                // ldmatrix: this lane feeds row rin of matrix mtx
   const int g = lane >> 2;                                  // accumulator row held by this lane
   const int src = 4 * (lane & 7) + ((lane & 7) >> 1);       // lane that holds the diagonal of pair (lane & 7)
-  ll = rr = lr = 0.f;
+  const int row = row0 + 2 * rin + (mtx & 1);               // matrices 0,2: left rows; 1,3: right rows
+  uint32_t fr[8][4];
 #pragma unroll
-  for (int bp = 0; bp < 2; ++bp) {
-    uint32_t fr[2][8][4];
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const int row = half * 64 + (2 * bp + u) * 16 + 2 * rin + (mtx & 1);   // matrices 0,2: left rows; 1,3: right rows
-#pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {
-        const int chunk = 2 * (kk & 3) + (mtx >> 1);        // 16-byte chunk inside the 128-byte row
-        ldmatrix_x4(fr[u][kk], base + (kk >> 2) * kHalf + row * 128 + ((chunk ^ (row & 7)) << 4));
-      }
-    }
-    float d1[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, d2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-#pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        mma16816(d1[u], fr[u][kk], fr[u][kk][1], fr[u][kk][3]);   // columns = right rows
-        mma16816(d2[u], fr[u][kk], fr[u][kk][0], fr[u][kk][2]);   // columns = left rows
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const float v_lr = (g & 1) ? d1[u][1] : d1[u][0];     // row g (left), column g (right)
-      const float v_rr = (g & 1) ? d1[u][3] : d1[u][2];     // row 8 + g (right), column g (right)
-      const float v_ll = (g & 1) ? d2[u][1] : d2[u][0];     // row g (left), column g (left)
-      const float s_lr = __shfl_sync(0xffffffffu, v_lr, src);
-      const float s_rr = __shfl_sync(0xffffffffu, v_rr, src);
-      const float s_ll = __shfl_sync(0xffffffffu, v_ll, src);
-      if ((lane >> 3) == 2 * bp + u) { lr = s_lr; rr = s_rr; ll = s_ll; }
-    }
+  for (int kk = 0; kk < 8; ++kk) {
+    const int chunk = 2 * (kk & 3) + (mtx >> 1);            // 16-byte chunk inside the 128-byte row
+    ldmatrix_x4(fr[kk], base + (kk >> 2) * kHalf + row * 128 + ((chunk ^ (row & 7)) << 4));
   }
+  float d1[4] = {0.f, 0.f, 0.f, 0.f}, d2[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) {
+    mma16816(d1, fr[kk], fr[kk][1], fr[kk][3]);             // columns = right rows
+    mma16816(d2, fr[kk], fr[kk][0], fr[kk][2]);             // columns = left rows
+  }
+  const float v_lr = (g & 1) ? d1[1] : d1[0];               // row g (left), column g (right)
+  const float v_rr = (g & 1) ? d1[3] : d1[2];               // row 8 + g (right), column g (right)
+  const float v_ll = (g & 1) ? d2[1] : d2[0];               // row g (left), column g (left)
+  lr = __shfl_sync(0xffffffffu, v_lr, src);
+  rr = __shfl_sync(0xffffffffu, v_rr, src);
+  ll = __shfl_sync(0xffffffffu, v_ll, src);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
 flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmQ) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  extern __shared__ __align__(1024) uint8_t smem[];
   Misc* misc = reinterpret_cast<Misc*>(smem + kSmemMisc);
 
   const int seq = blockIdx.z;
@@ -167,14 +169,15 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
   const int t_end = min(ntiles, t_begin + a.tiles_per_split);
   const int my_tiles = t_end - t_begin;
   if (n <= 0) return;
+  if (smem_u32(smem) & 1023u) {                        // the swizzled tiles need a 1024-byte aligned base
+    if (threadIdx.x == 0 && a.status_dev) atomicExch(a.status_dev, (int)KVS_ERR_CUDA);
+    return;
+  }
   if (my_tiles <= 0) {
-    // an empty split still owes its two (empty) partials to the combine
-    if (warp >= 2 && warp < 10) {
-      const int wg = (warp - 2) >> 2, row = (warp & 3) * 32 + lane, m = qblk * 128 + row;
-      if (m < a.M) {
-        const size_t pidx = ((size_t)unit * (a.splits * 2) + split * 2 + wg) * a.M + m;
-        a.part_ml[pidx] = make_float2(-INFINITY, 0.f);
-      }
+    // an empty key range still owes its (empty) partial to the combine
+    if (warp >= 2 && warp < 6) {
+      const int row = (warp & 3) * 32 + lane, m = qblk * 128 + row;
+      if (m < a.M) a.part_ml[((size_t)unit * a.splits + split) * a.M + m] = make_float2(-INFINITY, 0.f);
     }
     return;
   }
@@ -189,17 +192,18 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       // rings, so that the next K tile is requested a whole softmax earlier than the next V tile
       mbar_init(&misc->kfull[s], 1);
       mbar_init(&misc->vfull[s], 1);
-      mbar_init(&misc->kfree[s], norm_k ? 3 : 1);       // MMA commit (+ the two pair-norm warps)
-      mbar_init(&misc->vfree[s], norm_v ? 3 : 1);
+      mbar_init(&misc->kfree[s], norm_k ? 1 + kNormWarps : 1);   // MMA commit (+ the pair-norm warps)
+      mbar_init(&misc->vfree[s], norm_v ? 1 + kNormWarps : 1);
       mbar_init(&misc->sfull[s], 1);
-      mbar_init(&misc->sfree[s], 8);                    // softmax warps
-      mbar_init(&misc->pready[s], 4);                   // warps of one group
-      mbar_init(&misc->ofull[s], 1);
+      mbar_init(&misc->sfree[s], kSoftmaxWarps);
     }
+    mbar_init(&misc->pready, kSoftmaxWarps);
+    mbar_init(&misc->ofull, 1);
     mbar_init(&misc->qfull, 1);
     misc->abort_flag = 0;
     mbar_fence_init();
   }
+  if (threadIdx.x < 3 * kTile) misc->rowmax[threadIdx.x / kTile][threadIdx.x % kTile] = kOrdNegInf;
   if (warp == 1) tmem_alloc(&misc->tmem_base, 512);
   tc_fence_before();
   __syncthreads();
@@ -286,11 +290,13 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         const int s = li & 1;
         const uint32_t v_addr = smem_u32(smem + kSmemStage + s * kStage + kOperand);
         if (ok && !mbar_wait(&misc->vfull[s], (li >> 1) & 1, abort_flag)) ok = false;
-        for (int g = 0; ok && g < 2; ++g) {
-          if (!mbar_wait(&misc->pready[g], li & 1, abort_flag)) { ok = false; break; }
-          tc_fence_after();
+        if (ok && !mbar_wait(&misc->pready, li & 1, abort_flag)) ok = false;
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t dO = tmem + 256;
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {                      // slots 0-63, 64-127 of the tile
           const uint32_t p_addr = smem_u32(smem + kSmemP + g * kPGroup);
-          const uint32_t dO = tmem + 256 + g * 128;
 #pragma unroll
           for (int hl = 0; hl < 2; ++hl) {
 #pragma unroll
@@ -298,31 +304,32 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
               // A: 16 slots = 32 bytes along the swizzled row; B: 16 slots = two 8-row groups of V
               const uint64_t ad = smem_desc_sw128(p_addr + hl * kHalf + kk * 32, 16, 1024);
               const uint64_t bd = smem_desc_sw128(v_addr + (g * 64 + kk * 16) * 128, kHalf, 1024);
-              umma_bf16(dO, ad, bd, idesc_o, (li > 0 || hl > 0 || kk > 0) ? 1u : 0u);
+              umma_bf16(dO, ad, bd, idesc_o, (li > 0 || g > 0 || hl > 0 || kk > 0) ? 1u : 0u);
             }
           }
-          tc_commit(&misc->ofull[g]);
         }
-        if (ok) tc_commit(&misc->vfree[s]);
+        tc_commit(&misc->ofull);
+        tc_commit(&misc->vfree[s]);
       }
     }
-  } else if (warp >= 10) {
+  } else if (warp >= 2 + kSoftmaxWarps) {
     // ================================================================ pair-norm warps
     if (norm_k || norm_v) {
-      const int hw = warp - 10;                                  // rows [64 hw, 64 hw + 64) of every tile
+      const int nw = warp - (2 + kSoftmaxWarps);                 // rows [32 nw, 32 nw + 32) of every tile
       const int off = tab.off;
       const int32_t* Cn = a.counts + (size_t)unit * a.n_max;
+      const int pl = lane & 15;                                  // lanes 0-15 own the warp's 16 pairs
       // counts of the next tile's pair travel while the current tile is processed
       float cl_next = 1.f, cr_next = 1.f;
       if (norm_v) {
-        const int sl = t_begin * kTile - shift + hw * 64 + 2 * lane;
+        const int sl = t_begin * kTile - shift + nw * 32 + 2 * pl;
         if (sl >= off && ((sl - off) >> 1) < sr.P) { cl_next = (float)Cn[sl]; cr_next = (float)Cn[sl + 1]; }
       }
       for (int li = 0; li < my_tiles; ++li) {
         const int s = li & 1, k = li >> 1;
-        const int slot_l = (t_begin + li) * kTile - shift + hw * 64 + 2 * lane;   // left slot of this lane's pair
+        const int slot_l = (t_begin + li) * kTile - shift + nw * 32 + 2 * pl;   // left slot of this lane's pair
         const int p = (slot_l - off) >> 1;
-        const bool pair_ok = slot_l >= off && p < sr.P;
+        const bool pair_ok = lane < 16 && slot_l >= off && p < sr.P;
         const float cl = cl_next, cr = cr_next;
         if (norm_v && li + 1 < my_tiles) {
           const int sl = slot_l + kTile;
@@ -335,19 +342,25 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         if (norm_k) {
           if (lane == 0) ok = mbar_wait(&misc->kfull[s], k & 1, abort_flag) ? 1 : 0;
           if (!__shfl_sync(0xffffffffu, ok, 0)) break;
-          float kll, krr, klr;
-          pair_dots(st, hw, lane, kll, krr, klr);
+          float ll[2], rr[2], lr[2];
+          pair_dots8(st, nw * 32, lane, ll[0], rr[0], lr[0]);
+          pair_dots8(st, nw * 32 + 16, lane, ll[1], rr[1], lr[1]);
           __syncwarp();
           if (lane == 0) mbar_arrive(&misc->kfree[s]);           // the K rows are no longer needed here
+          const bool b = (lane >> 3) & 1;
+          const float kll = b ? ll[1] : ll[0], krr = b ? rr[1] : rr[0], klr = b ? lr[1] : lr[0];
           if (pair_ok) out[3] = klr / fmaxf(sqrtf(kll) * sqrtf(krr), 1e-30f);
         }
         if (norm_v) {
           if (lane == 0) ok = mbar_wait(&misc->vfull[s], k & 1, abort_flag) ? 1 : 0;
           if (!__shfl_sync(0xffffffffu, ok, 0)) break;
-          float vll, vrr, vlr;
-          pair_dots(st + kOperand, hw, lane, vll, vrr, vlr);
+          float ll[2], rr[2], lr[2];
+          pair_dots8(st + kOperand, nw * 32, lane, ll[0], rr[0], lr[0]);
+          pair_dots8(st + kOperand, nw * 32 + 16, lane, ll[1], rr[1], lr[1]);
           __syncwarp();
           if (lane == 0) mbar_arrive(&misc->vfree[s]);
+          const bool b = (lane >> 3) & 1;
+          const float vll = b ? ll[1] : ll[0], vrr = b ? rr[1] : rr[0], vlr = b ? lr[1] : lr[0];
           if (pair_ok) {
             const float icl = 1.f / cl, icr = 1.f / cr;
             const float r2l = vll * icl * icl, r2r = vrr * icr * icr;
@@ -357,85 +370,87 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       }
     }
   } else {
-    // ================================================================ softmax groups
-    const int wg = (warp - 2) >> 2;
+    // ================================================================ softmax warps
+    const int cg = (warp - 2) >> 2;                       // 32-slot column group of the tile
     const int row = (warp & 3) * 32 + lane;               // TMEM lane = query row in the block
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    const int t128 = threadIdx.x - 64 - wg * 128;         // 0..127 within the group
     const int m = qblk * 128 + row;
     const int last_vis = a.causal ? (n - a.Wq + (m % a.Wq)) : (n - 1);
     const int32_t* Cb = a.counts + (size_t)unit * a.n_max;
-    uint8_t* pbuf = smem + kSmemP + wg * kPGroup;
+    uint8_t* pbuf = smem + kSmemP + (cg >> 1) * kPGroup;  // hi at +0, lo at +kHalf; this thread's chunks 4 (cg & 1) ..
     float m_stab = -INFINITY, l = 0.f;
     bool alive = true;
-    // the count of "its" slot of the next tile travels while the current tile is processed
+    // (first column group) the count of slot `row` of the next tile travels while the current tile is processed
     int cnt_next = 1;
-    if (t128 < 64) {
-      const int j = t_begin * kTile - shift + wg * 64 + t128;
+    if (cg == 0) {
+      const int j = t_begin * kTile - shift + row;
       if (j >= 0 && j < n) cnt_next = Cb[j];
     }
     for (int li = 0; li < my_tiles; ++li) {
       const int s = li & 1, k = li >> 1;
-      const int j0 = (t_begin + li) * kTile - shift + wg * 64;    // first slot of this group's half tile
-      float* cnt = misc->cnt[s][wg];
-      if (t128 < 64) {
-        cnt[t128] = (float)cnt_next;
-        const int j = j0 + kTile + t128;
+      const int j0 = (t_begin + li) * kTile - shift + cg * 32;    // first slot of this thread's columns
+      float* cnt = misc->cnt[s];
+      uint32_t* rmax = misc->rowmax[li % 3];
+      if (cg == 0) {
+        cnt[row] = (float)cnt_next;
+        const int j = (t_begin + li + 1) * kTile - shift + row;
         cnt_next = (li + 1 < my_tiles && j >= 0 && j < n) ? Cb[j] : 1;
       }
-      float x[64];
-      float mt = -INFINITY;
+      float x[32];
       if (alive) alive = warp_wait(&misc->sfull[s], k & 1, abort_flag, lane);
       if (alive) {
         tc_fence_after();
-        tmem_ld32(tmem + lane_addr + s * 128 + wg * 64, x);
-        tmem_ld32(tmem + lane_addr + s * 128 + wg * 64 + 32, x + 32);
+        tmem_ld32(tmem + lane_addr + s * 128 + cg * 32, x);
         tmem_ld_wait();
         tc_fence_before();
         warp_arrive(&misc->sfree[s], lane);
         // logits in log2 units, with mask (the stabiliser ignores the counts: exp(s - m) <= 1 either way)
-        const bool need_mask = (j0 < 0) || (j0 + 63 > min(n - 1, a.causal ? n - a.Wq : n - 1));
+        const bool need_mask = (j0 < 0) || (j0 + 31 > min(n - 1, a.causal ? n - a.Wq : n - 1));
         float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one
         if (!need_mask) {
 #pragma unroll
-          for (int i = 0; i < 64; ++i) {
+          for (int i = 0; i < 32; ++i) {
             x[i] *= a.scale_log2;
             mx[i & 3] = fmaxf(mx[i & 3], x[i]);
           }
         } else {
 #pragma unroll
-          for (int i = 0; i < 64; ++i) {
+          for (int i = 0; i < 32; ++i) {
             const float v = x[i] * a.scale_log2;
             x[i] = (j0 + i >= 0 && j0 + i <= last_vis) ? v : -INFINITY;
             mx[i & 3] = fmaxf(mx[i & 3], x[i]);
           }
         }
-        mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+        atomicMax(&rmax[row], f2ord(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]))));
       }
-      // the one barrier of the tile: the counts staged above are visible to the whole group, and
-      // every warp has finished reading the buffer that the tile after next will overwrite
-      wg_barrier(wg);
+      // the one barrier of the tile: the row maxima and the staged counts are complete
+      softmax_barrier();
+      // the buffer of the tile after next was last read one tile ago: every thread is past that read now
+      if (cg == 0) misc->rowmax[(li + 2) % 3][row] = kOrdNegInf;
       if (!alive) continue;
+      const float mt = ord2f(rmax[row]);
       const float m_new = fmaxf(m_stab, mt);
       const bool need = m_new > m_stab + kRescaleGap || (m_stab == -INFINITY && m_new > -INFINITY);
       const bool any_need = __any_sync(0xffffffffu, need && li > 0);
       // the previous tile's P V product must be done before P is overwritten (and before a rescale)
       if (li > 0) {
-        if (!(alive = warp_wait(&misc->ofull[wg], (li - 1) & 1, abort_flag, lane))) continue;
+        if (!(alive = warp_wait(&misc->ofull, (li - 1) & 1, abort_flag, lane))) continue;
         tc_fence_after();
       }
+      const float f = (need && m_stab > -INFINITY) ? fast_exp2(m_stab - m_new) : 1.f;
       if (any_need) {
-        const float f = (need && m_stab > -INFINITY) ? fast_exp2(m_stab - m_new) : 1.f;
+        if (cg == 0) {                                     // the row of O is rescaled once
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          float ov[32];
-          tmem_ld32(tmem + lane_addr + 256 + wg * 128 + c * 32, ov);
-          tmem_ld_wait();
+          for (int c = 0; c < 4; ++c) {
+            float ov[32];
+            tmem_ld32(tmem + lane_addr + 256 + c * 32, ov);
+            tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) ov[i] *= f;
-          tmem_st32(tmem + lane_addr + 256 + wg * 128 + c * 32, ov);
+            for (int i = 0; i < 32; ++i) ov[i] *= f;
+            tmem_st32(tmem + lane_addr + 256 + c * 32, ov);
+          }
+          tmem_st_wait();
         }
-        tmem_st_wait();
         l *= f;
       }
       if (need) m_stab = m_new;
@@ -445,10 +460,10 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       // the exact remainder, so hi + lo carries 16 significant bits.
       float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
+      for (int c = 0; c < 4; ++c) {
         uint32_t hi[4], lo[4];
-        const float4 ca = *reinterpret_cast<const float4*>(&cnt[c * 8]);
-        const float4 cb = *reinterpret_cast<const float4*>(&cnt[c * 8 + 4]);
+        const float4 ca = *reinterpret_cast<const float4*>(&cnt[cg * 32 + c * 8]);
+        const float4 cb = *reinterpret_cast<const float4*>(&cnt[cg * 32 + c * 8 + 4]);
         const float cc[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
@@ -459,7 +474,8 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
           hi[u] = __byte_perm(b0, b1, 0x7632);
           lo[u] = pack_bf16(q0 - __uint_as_float(b0 & 0xffff0000u), q1 - __uint_as_float(b1 & 0xffff0000u));
         }
-        const int off16 = row * 128 + ((c ^ (row & 7)) << 4);
+        const int chunk = (cg & 1) * 4 + c;                // 16-byte chunk inside the 128-byte row
+        const int off16 = row * 128 + ((chunk ^ (row & 7)) << 4);
         *reinterpret_cast<uint4*>(pbuf + off16) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
         *reinterpret_cast<uint4*>(pbuf + kHalf + off16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
       }
@@ -469,7 +485,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       if (tile_row0 < 0 || tile_row0 + kTile > n) {
         if (!(alive = warp_wait(&misc->vfull[s], k & 1, abort_flag, lane))) continue;
         uint8_t* vt = smem + kSmemStage + s * kStage + kOperand;
-        for (int it = wg * 64 * 16 + t128; it < (wg * 64 + 64) * 16; it += 128) {
+        for (int it = threadIdx.x - 64; it < kTile * 16; it += kSoftmaxWarps * 32) {
           const int r = it >> 4, ch = it & 15;
           if (tile_row0 + r < 0 || tile_row0 + r >= n)
             *reinterpret_cast<uint4*>(vt + (ch >> 3) * kHalf + r * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
@@ -477,23 +493,25 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       }
       fence_proxy_async();
       tc_fence_before();
-      warp_arrive(&misc->pready[wg], lane);
+      warp_arrive(&misc->pready, lane);
     }
-    // ---- the partial of this (split, group)
-    if (alive && warp_wait(&misc->ofull[wg], (my_tiles - 1) & 1, abort_flag, lane)) {
+    // ---- the partial of this key range: the four column groups of a row add their sums, then each
+    //      writes 32 channels of the row of O
+    softmax_barrier();                                            // row maxima and counts are dead now
+    misc->lsum[cg][row] = l;
+    softmax_barrier();
+    if (alive && warp_wait(&misc->ofull, (my_tiles - 1) & 1, abort_flag, lane)) {
       tc_fence_after();
-      const size_t pidx = ((size_t)unit * (a.splits * 2) + split * 2 + wg) * a.M + m;
-      if (m < a.M) a.part_ml[pidx] = make_float2(m_stab, l);
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        float ov[32];
-        tmem_ld32(tmem + lane_addr + 256 + wg * 128 + c * 32, ov);
-        tmem_ld_wait();
-        if (m < a.M) {
-          float4* po = reinterpret_cast<float4*>(a.part_o + pidx * KVS_D + c * 32);
+      const size_t pidx = ((size_t)unit * a.splits + split) * a.M + m;
+      if (cg == 0 && m < a.M)
+        a.part_ml[pidx] = make_float2(m_stab, (misc->lsum[0][row] + misc->lsum[1][row]) + (misc->lsum[2][row] + misc->lsum[3][row]));
+      float ov[32];
+      tmem_ld32(tmem + lane_addr + 256 + cg * 32, ov);
+      tmem_ld_wait();
+      if (m < a.M) {
+        float4* po = reinterpret_cast<float4*>(a.part_o + pidx * KVS_D + cg * 32);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) po[i] = make_float4(ov[4 * i], ov[4 * i + 1], ov[4 * i + 2], ov[4 * i + 3]);
-        }
+        for (int i = 0; i < 8; ++i) po[i] = make_float4(ov[4 * i], ov[4 * i + 1], ov[4 * i + 2], ov[4 * i + 3]);
       }
     }
   }

@@ -68,8 +68,8 @@ struct FlashTcArgs {
   float scale_log2;
   int32_t n_max;
   const int32_t* counts;   // [U, n_max]
-  float2* part_ml;         // [U, 2 * splits, M]
-  float* part_o;           // [U, 2 * splits, M, 128]
+  float2* part_ml;         // [U, splits, M]
+  float* part_o;           // [U, splits, M, 128]
   float4* pair_norms;      // optional [U, pair_stride]: (|vbar_l|^2, |vbar_r|^2, |vbar_l + vbar_r|^2, cos(K_l, K_r))
   int32_t pair_stride;     //   of the round's candidate pairs; tiles are then aligned with the pairs
   int32_t* status_dev;
