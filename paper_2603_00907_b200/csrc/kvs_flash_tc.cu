@@ -40,7 +40,7 @@ constexpr int kThreads = (2 + kSoftmaxWarps + kNormWarps) * 32;   // warp 0: TMA
 constexpr float kRescaleGap = 8.f;         // log2 units
 
 struct Misc {
-  uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[2], sfree[2], pready, ofull, qfull;
+  uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[2], sfree[2], pready[2], ofull[2], qfull;
   uint32_t tmem_base;
   int abort_flag;
   union {
@@ -197,8 +197,12 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       mbar_init(&misc->sfull[s], 1);
       mbar_init(&misc->sfree[s], kSoftmaxWarps);
     }
-    mbar_init(&misc->pready, kSoftmaxWarps);
-    mbar_init(&misc->ofull, 1);
+    // P' is handed over in two halves (the first and the last 16 slots of every column group), so
+    // that the P V products of one half run while the other half is still being written
+    for (int hf = 0; hf < 2; ++hf) {
+      mbar_init(&misc->pready[hf], kSoftmaxWarps);
+      mbar_init(&misc->ofull[hf], 1);
+    }
     mbar_init(&misc->qfull, 1);
     misc->abort_flag = 0;
     mbar_fence_init();
@@ -290,26 +294,25 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         const int s = li & 1;
         const uint32_t v_addr = smem_u32(smem + kSmemStage + s * kStage + kOperand);
         if (ok && !mbar_wait(&misc->vfull[s], (li >> 1) & 1, abort_flag)) ok = false;
-        if (ok && !mbar_wait(&misc->pready, li & 1, abort_flag)) ok = false;
-        if (!ok) break;
-        tc_fence_after();
         const uint32_t dO = tmem + 256;
+        for (int hf = 0; ok && hf < 2; ++hf) {
+          if (!mbar_wait(&misc->pready[hf], li & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
-        for (int g = 0; g < 2; ++g) {                      // slots 0-63, 64-127 of the tile
-          const uint32_t p_addr = smem_u32(smem + kSmemP + g * kPGroup);
+          for (int cgi = 0; cgi < 4; ++cgi) {
+            const int kk = 2 * cgi + hf;                     // 16-slot step of the tile: slots [16 kk, 16 kk + 16)
+            const uint32_t p_addr = smem_u32(smem + kSmemP + (kk >> 2) * kPGroup);
 #pragma unroll
-          for (int hl = 0; hl < 2; ++hl) {
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
+            for (int hl = 0; hl < 2; ++hl) {
               // A: 16 slots = 32 bytes along the swizzled row; B: 16 slots = two 8-row groups of V
-              const uint64_t ad = smem_desc_sw128(p_addr + hl * kHalf + kk * 32, 16, 1024);
-              const uint64_t bd = smem_desc_sw128(v_addr + (g * 64 + kk * 16) * 128, kHalf, 1024);
-              umma_bf16(dO, ad, bd, idesc_o, (li > 0 || g > 0 || hl > 0 || kk > 0) ? 1u : 0u);
+              const uint64_t ad = smem_desc_sw128(p_addr + hl * kHalf + (kk & 3) * 32, 16, 1024);
+              const uint64_t bd = smem_desc_sw128(v_addr + (kk * 16) * 128, kHalf, 1024);
+              umma_bf16(dO, ad, bd, idesc_o, (li > 0 || hf > 0 || cgi > 0 || hl > 0) ? 1u : 0u);
             }
           }
+          tc_commit(&misc->ofull[hf]);
         }
-        tc_commit(&misc->ofull);
-        tc_commit(&misc->vfree[s]);
+        if (ok) tc_commit(&misc->vfree[s]);
       }
     }
   } else if (warp >= 2 + kSoftmaxWarps) {
@@ -432,9 +435,11 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       const float m_new = fmaxf(m_stab, mt);
       const bool need = m_new > m_stab + kRescaleGap || (m_stab == -INFINITY && m_new > -INFINITY);
       const bool any_need = __any_sync(0xffffffffu, need && li > 0);
-      // the previous tile's P V product must be done before P is overwritten (and before a rescale)
+      // the previous tile's P V products must be done before P is overwritten: half by half, or
+      // both before a rescale of O
       if (li > 0) {
-        if (!(alive = warp_wait(&misc->ofull, (li - 1) & 1, abort_flag, lane))) continue;
+        if (!(alive = warp_wait(&misc->ofull[0], (li - 1) & 1, abort_flag, lane))) continue;
+        if (any_need && !(alive = warp_wait(&misc->ofull[1], (li - 1) & 1, abort_flag, lane))) continue;
         tc_fence_after();
       }
       const float f = (need && m_stab > -INFINITY) ? fast_exp2(m_stab - m_new) : 1.f;
@@ -455,31 +460,6 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       }
       if (need) m_stab = m_new;
       const float ms = (m_stab == -INFINITY) ? 0.f : m_stab;      // row with nothing visible yet
-      // P' = exp2(x - m) as hi + lo bf16, written as the K-major operand [row][64 slots]
-      // The hi term is the value cut to bf16 (a byte permute, no conversion); the lo term rounds
-      // the exact remainder, so hi + lo carries 16 significant bits.
-      float ls[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t hi[4], lo[4];
-        const float4 ca = *reinterpret_cast<const float4*>(&cnt[cg * 32 + c * 8]);
-        const float4 cb = *reinterpret_cast<const float4*>(&cnt[cg * 32 + c * 8 + 4]);
-        const float cc[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int i = c * 8 + u * 2;
-          const float q0 = fast_exp2(x[i] - ms), q1 = fast_exp2(x[i + 1] - ms);
-          ls[u] = fmaf(cc[2 * u], q0, fmaf(cc[2 * u + 1], q1, ls[u]));
-          const uint32_t b0 = __float_as_uint(q0), b1 = __float_as_uint(q1);
-          hi[u] = __byte_perm(b0, b1, 0x7632);
-          lo[u] = pack_bf16(q0 - __uint_as_float(b0 & 0xffff0000u), q1 - __uint_as_float(b1 & 0xffff0000u));
-        }
-        const int chunk = (cg & 1) * 4 + c;                // 16-byte chunk inside the 128-byte row
-        const int off16 = row * 128 + ((chunk ^ (row & 7)) << 4);
-        *reinterpret_cast<uint4*>(pbuf + off16) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        *reinterpret_cast<uint4*>(pbuf + kHalf + off16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-      }
-      l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       // rows of the V tile outside the sequence may hold anything: each warp zeroes its share
       const int tile_row0 = (t_begin + li) * kTile - shift;
       if (tile_row0 < 0 || tile_row0 + kTile > n) {
@@ -491,16 +471,49 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
             *reinterpret_cast<uint4*>(vt + (ch >> 3) * kHalf + r * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
         }
       }
-      fence_proxy_async();
-      tc_fence_before();
-      warp_arrive(&misc->pready, lane);
+      // P' = exp2(x - m) as hi + lo bf16, written as the K-major operand [row][64 slots]
+      // The hi term is the value cut to bf16 (a byte permute, no conversion); the lo term rounds
+      // the exact remainder, so hi + lo carries 16 significant bits.
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        if (hf == 1 && li > 0 && !any_need) {
+          if (!(alive = warp_wait(&misc->ofull[1], (li - 1) & 1, abort_flag, lane))) break;
+        }
+#pragma unroll
+        for (int c = 2 * hf; c < 2 * hf + 2; ++c) {
+          uint32_t hi[4], lo[4];
+          const float4 ca = *reinterpret_cast<const float4*>(&cnt[cg * 32 + c * 8]);
+          const float4 cb = *reinterpret_cast<const float4*>(&cnt[cg * 32 + c * 8 + 4]);
+          const float cc[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int i = c * 8 + u * 2;
+            const float q0 = fast_exp2(x[i] - ms), q1 = fast_exp2(x[i + 1] - ms);
+            ls[u] = fmaf(cc[2 * u], q0, fmaf(cc[2 * u + 1], q1, ls[u]));
+            const uint32_t b0 = __float_as_uint(q0), b1 = __float_as_uint(q1);
+            hi[u] = __byte_perm(b0, b1, 0x7632);
+            lo[u] = pack_bf16(q0 - __uint_as_float(b0 & 0xffff0000u), q1 - __uint_as_float(b1 & 0xffff0000u));
+          }
+          const int chunk = (cg & 1) * 4 + c;                // 16-byte chunk inside the 128-byte row
+          const int off16 = row * 128 + ((chunk ^ (row & 7)) << 4);
+          *reinterpret_cast<uint4*>(pbuf + off16) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4*>(pbuf + kHalf + off16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        warp_arrive(&misc->pready[hf], lane);
+      }
+      if (!alive) continue;
+      l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
     }
     // ---- the partial of this key range: the four column groups of a row add their sums, then each
     //      writes 32 channels of the row of O
     softmax_barrier();                                            // row maxima and counts are dead now
     misc->lsum[cg][row] = l;
     softmax_barrier();
-    if (alive && warp_wait(&misc->ofull, (my_tiles - 1) & 1, abort_flag, lane)) {
+    if (alive && warp_wait(&misc->ofull[0], (my_tiles - 1) & 1, abort_flag, lane) &&
+        warp_wait(&misc->ofull[1], (my_tiles - 1) & 1, abort_flag, lane)) {
       tc_fence_after();
       const size_t pidx = ((size_t)unit * a.splits + split) * a.M + m;
       if (cg == 0 && m < a.M)
