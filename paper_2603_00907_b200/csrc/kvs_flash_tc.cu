@@ -9,10 +9,10 @@
 // threads of a row agree on the row maximum through a shared-memory atomic maximum, keep the
 // same stabiliser m (it only moves when the maximum grows by more than 2^8, in which case the
 // first of the four rescales the row of O in TMEM), and each writes P' = exp(s - m), split
-// into two bf16 terms, to shared memory, keeping its part of l = sum_j c_j exp(s_j - m): the
-// count bias ln c_j of a merged slot is just the factor c_j in that sum.  The issuing thread
-// then runs
-//   O[q, :] += (P'_hi + P'_lo) Vsum_tile            (V as the MN-major operand)
+// into two bf16 terms, back into the tensor-memory columns the logits came from, keeping its
+// part of l = sum_j c_j exp(s_j - m): the count bias ln c_j of a merged slot is just the factor
+// c_j in that sum.  The issuing thread then runs
+//   O[q, :] += (P'_hi + P'_lo) Vsum_tile            (P' from tensor memory, V as the MN-major operand)
 // with O accumulating in TMEM across the tiles [Eq. attn_def_vec with merged slots:
 // o = sum_j alpha_j Vsum_j / c_j].  At the end (stabiliser, sum, O) is written as the partial
 // of this key range.  Window queries and decode queries use the same kernel.
@@ -32,15 +32,14 @@ constexpr int kTile = 128;
 constexpr int kHalf = 16384;               // [128 rows x 64 bf16], 128-byte swizzle
 constexpr int kOperand = 2 * kHalf;
 constexpr int kStage = 2 * kOperand;       // K tile + V tile
-constexpr int kPGroup = 2 * kHalf;         // P'_hi and P'_lo of 64 slots: [128 q x 64 slots] each
-constexpr int kSmemQ = 0, kSmemStage = kOperand, kSmemP = kSmemStage + 2 * kStage;
-constexpr int kSmemMisc = kSmemP + 2 * kPGroup;
+constexpr int kSmemQ = 0, kSmemStage = kOperand;
+constexpr int kSmemMisc = kSmemStage + 2 * kStage;
 constexpr int kSoftmaxWarps = 16, kNormWarps = 4;
 constexpr int kThreads = (2 + kSoftmaxWarps + kNormWarps) * 32;   // warp 0: TMA, 1: MMA, 2-17: softmax, 18-21: pair norms
 constexpr float kRescaleGap = 8.f;         // log2 units
 
 struct Misc {
-  uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[2], sfree[2], pready[2], ofull[2], qfull;
+  uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[2], pready[2], ofull[2], qfull;
   uint32_t tmem_base;
   int abort_flag;
   union {
@@ -95,6 +94,11 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
         "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])),
         "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
       : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* v) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() {
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -195,7 +199,6 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       mbar_init(&misc->kfree[s], norm_k ? 1 + kNormWarps : 1);   // MMA commit (+ the pair-norm warps)
       mbar_init(&misc->vfree[s], norm_v ? 1 + kNormWarps : 1);
       mbar_init(&misc->sfull[s], 1);
-      mbar_init(&misc->sfree[s], kSoftmaxWarps);
     }
     // P' is handed over in two halves (the first and the last 16 slots of every column group), so
     // that the P V products of one half run while the other half is still being written
@@ -273,8 +276,8 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       const uint32_t q_addr = smem_u32(smem + kSmemQ);
       auto issue_s = [&](int li) -> bool {
         const int s = li & 1, k = li >> 1;
+        // buffer s last held P' of tile li - 2, whose products were issued by this thread before
         if (!mbar_wait(&misc->kfull[s], k & 1, abort_flag)) return false;
-        if (!mbar_wait(&misc->sfree[s], (k & 1) ^ 1, abort_flag)) return false;
         tc_fence_after();
         const uint32_t k_addr = smem_u32(smem + kSmemStage + s * kStage);
 #pragma unroll
@@ -301,13 +304,13 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
 #pragma unroll
           for (int cgi = 0; cgi < 4; ++cgi) {
             const int kk = 2 * cgi + hf;                     // 16-slot step of the tile: slots [16 kk, 16 kk + 16)
-            const uint32_t p_addr = smem_u32(smem + kSmemP + (kk >> 2) * kPGroup);
 #pragma unroll
             for (int hl = 0; hl < 2; ++hl) {
-              // A: 16 slots = 32 bytes along the swizzled row; B: 16 slots = two 8-row groups of V
-              const uint64_t ad = smem_desc_sw128(p_addr + hl * kHalf + (kk & 3) * 32, 16, 1024);
+              // A: 16 slots = 8 columns of P'_hi (columns 0-63 of the logit buffer) or P'_lo (64-127);
+              // B: 16 slots = two 8-row groups of V
+              const uint32_t ap = tmem + s * 128 + hl * 64 + kk * 8;
               const uint64_t bd = smem_desc_sw128(v_addr + (kk * 16) * 128, kHalf, 1024);
-              umma_bf16(dO, ad, bd, idesc_o, (li > 0 || hf > 0 || cgi > 0 || hl > 0) ? 1u : 0u);
+              umma_bf16_ts(dO, ap, bd, idesc_o, (li > 0 || hf > 0 || cgi > 0 || hl > 0) ? 1u : 0u);
             }
           }
           tc_commit(&misc->ofull[hf]);
@@ -380,7 +383,6 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     const int m = qblk * 128 + row;
     const int last_vis = a.causal ? (n - a.Wq + (m % a.Wq)) : (n - 1);
     const int32_t* Cb = a.counts + (size_t)unit * a.n_max;
-    uint8_t* pbuf = smem + kSmemP + (cg >> 1) * kPGroup;  // hi at +0, lo at +kHalf; this thread's chunks 4 (cg & 1) ..
     float m_stab = -INFINITY, l = 0.f;
     bool alive = true;
     // (first column group) the count of slot `row` of the next tile travels while the current tile is processed
@@ -405,8 +407,6 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         tc_fence_after();
         tmem_ld32(tmem + lane_addr + s * 128 + cg * 32, x);
         tmem_ld_wait();
-        tc_fence_before();
-        warp_arrive(&misc->sfree[s], lane);
         // logits in log2 units, with mask (the stabiliser ignores the counts: exp(s - m) <= 1 either way)
         const bool need_mask = (j0 < 0) || (j0 + 31 > min(n - 1, a.causal ? n - a.Wq : n - 1));
         float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one
@@ -470,19 +470,22 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
           if (tile_row0 + r < 0 || tile_row0 + r >= n)
             *reinterpret_cast<uint4*>(vt + (ch >> 3) * kHalf + r * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
         }
+        fence_proxy_async();                               // the tensor core reads these rows
       }
-      // P' = exp2(x - m) as hi + lo bf16, written as the K-major operand [row][64 slots]
-      // The hi term is the value cut to bf16 (a byte permute, no conversion); the lo term rounds
-      // the exact remainder, so hi + lo carries 16 significant bits.
+      // P' = exp2(x - m) as hi + lo bf16, two slots per 32-bit column, written over the logits of
+      // this buffer (every warp has read its logits: the barrier above) as the A operand of P' V:
+      // hi in columns 0-63, lo in columns 64-127.  The hi term is the value cut to bf16 (a byte
+      // permute, no conversion); the lo term rounds the exact remainder, so hi + lo carries 16
+      // significant bits.
       float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {
         if (hf == 1 && li > 0 && !any_need) {
           if (!(alive = warp_wait(&misc->ofull[1], (li - 1) & 1, abort_flag, lane))) break;
         }
+        uint32_t hi[8], lo[8];
 #pragma unroll
         for (int c = 2 * hf; c < 2 * hf + 2; ++c) {
-          uint32_t hi[4], lo[4];
           const float4 ca = *reinterpret_cast<const float4*>(&cnt[cg * 32 + c * 8]);
           const float4 cb = *reinterpret_cast<const float4*>(&cnt[cg * 32 + c * 8 + 4]);
           const float cc[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
@@ -492,15 +495,13 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
             const float q0 = fast_exp2(x[i] - ms), q1 = fast_exp2(x[i + 1] - ms);
             ls[u] = fmaf(cc[2 * u], q0, fmaf(cc[2 * u + 1], q1, ls[u]));
             const uint32_t b0 = __float_as_uint(q0), b1 = __float_as_uint(q1);
-            hi[u] = __byte_perm(b0, b1, 0x7632);
-            lo[u] = pack_bf16(q0 - __uint_as_float(b0 & 0xffff0000u), q1 - __uint_as_float(b1 & 0xffff0000u));
+            hi[(c & 1) * 4 + u] = __byte_perm(b0, b1, 0x7632);
+            lo[(c & 1) * 4 + u] = pack_bf16(q0 - __uint_as_float(b0 & 0xffff0000u), q1 - __uint_as_float(b1 & 0xffff0000u));
           }
-          const int chunk = (cg & 1) * 4 + c;                // 16-byte chunk inside the 128-byte row
-          const int off16 = row * 128 + ((chunk ^ (row & 7)) << 4);
-          *reinterpret_cast<uint4*>(pbuf + off16) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          *reinterpret_cast<uint4*>(pbuf + kHalf + off16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
         }
-        fence_proxy_async();
+        tmem_st8(tmem + lane_addr + s * 128 + cg * 16 + hf * 8, hi);
+        tmem_st8(tmem + lane_addr + s * 128 + 64 + cg * 16 + hf * 8, lo);
+        tmem_st_wait();
         tc_fence_before();
         warp_arrive(&misc->pready[hf], lane);
       }
