@@ -383,7 +383,9 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     const int m = qblk * 128 + row;
     const int last_vis = a.causal ? (n - a.Wq + (m % a.Wq)) : (n - 1);
     const int32_t* Cb = a.counts + (size_t)unit * a.n_max;
-    float m_stab = -INFINITY, l = 0.f;
+    // stabiliser in log2 units; until a row has seen a visible slot it is 0 (keeps the arithmetic finite)
+    float m_stab = 0.f, l = 0.f;
+    bool have_stab = false;
     bool alive = true;
     // (first column group) the count of slot `row` of the next tile travels while the current tile is processed
     int cnt_next = 1;
@@ -407,19 +409,20 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         tc_fence_after();
         tmem_ld32(tmem + lane_addr + s * 128 + cg * 32, x);
         tmem_ld_wait();
-        // logits in log2 units, with mask (the stabiliser ignores the counts: exp(s - m) <= 1 either way)
+        // logits in log2 units relative to the stabiliser (one multiply-add), with mask; the stabiliser
+        // ignores the counts: exp(s - m) <= 1 either way
         const bool need_mask = (j0 < 0) || (j0 + 31 > min(n - 1, a.causal ? n - a.Wq : n - 1));
         float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one
         if (!need_mask) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            x[i] *= a.scale_log2;
+            x[i] = fmaf(x[i], a.scale_log2, -m_stab);
             mx[i & 3] = fmaxf(mx[i & 3], x[i]);
           }
         } else {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            const float v = x[i] * a.scale_log2;
+            const float v = fmaf(x[i], a.scale_log2, -m_stab);
             x[i] = (j0 + i >= 0 && j0 + i <= last_vis) ? v : -INFINITY;
             mx[i & 3] = fmaxf(mx[i & 3], x[i]);
           }
@@ -431,9 +434,10 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       // the buffer of the tile after next was last read one tile ago: every thread is past that read now
       if (cg == 0) misc->rowmax[(li + 2) % 3][row] = kOrdNegInf;
       if (!alive) continue;
+      // row maximum relative to the stabiliser: the stabiliser moves up by it when the row has none
+      // yet or when the maximum has outgrown it by more than the gap
       const float mt = ord2f(rmax[row]);
-      const float m_new = fmaxf(m_stab, mt);
-      const bool need = m_new > m_stab + kRescaleGap || (m_stab == -INFINITY && m_new > -INFINITY);
+      const bool need = mt > -INFINITY && (!have_stab || mt > kRescaleGap);
       const bool any_need = __any_sync(0xffffffffu, need && li > 0);
       // the previous tile's P V products must be done before P is overwritten: half by half, or
       // both before a rescale of O
@@ -442,7 +446,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         if (any_need && !(alive = warp_wait(&misc->ofull[1], (li - 1) & 1, abort_flag, lane))) continue;
         tc_fence_after();
       }
-      const float f = (need && m_stab > -INFINITY) ? fast_exp2(m_stab - m_new) : 1.f;
+      const float f = (need && have_stab) ? fast_exp2(-mt) : 1.f;
       if (any_need) {
         if (cg == 0) {                                     // the row of O is rescaled once
 #pragma unroll 1
@@ -458,8 +462,12 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         }
         l *= f;
       }
-      if (need) m_stab = m_new;
-      const float ms = (m_stab == -INFINITY) ? 0.f : m_stab;      // row with nothing visible yet
+      if (need) {
+        m_stab += mt;
+        have_stab = true;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) x[i] -= mt;
+      }
       // rows of the V tile outside the sequence may hold anything: each warp zeroes its share
       const int tile_row0 = (t_begin + li) * kTile - shift;
       if (tile_row0 < 0 || tile_row0 + kTile > n) {
@@ -492,7 +500,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
             const int i = c * 8 + u * 2;
-            const float q0 = fast_exp2(x[i] - ms), q1 = fast_exp2(x[i + 1] - ms);
+            const float q0 = fast_exp2(x[i]), q1 = fast_exp2(x[i + 1]);
             ls[u] = fmaf(cc[2 * u], q0, fmaf(cc[2 * u + 1], q1, ls[u]));
             const uint32_t b0 = __float_as_uint(q0), b1 = __float_as_uint(q1);
             hi[(c & 1) * 4 + u] = __byte_perm(b0, b1, 0x7632);
@@ -518,7 +526,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       tc_fence_after();
       const size_t pidx = ((size_t)unit * a.splits + split) * a.M + m;
       if (cg == 0 && m < a.M)
-        a.part_ml[pidx] = make_float2(m_stab, (misc->lsum[0][row] + misc->lsum[1][row]) + (misc->lsum[2][row] + misc->lsum[3][row]));
+        a.part_ml[pidx] = make_float2(have_stab ? m_stab : -INFINITY, (misc->lsum[0][row] + misc->lsum[1][row]) + (misc->lsum[2][row] + misc->lsum[3][row]));
       float ov[32];
       tmem_ld32(tmem + lane_addr + 256 + cg * 32, ov);
       tmem_ld_wait();
