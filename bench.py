@@ -90,7 +90,7 @@ class ClockSampler(threading.Thread):
 # file changes, the figure is stale and `traffic` is reported as null.
 NCU_TRAFFIC = {
     "hessian_stats": (1.03, "kvs_stats_tc.cu", "000b7e86f391e522"),
-    "attn_partials": (1.01, "kvs_flash_tc.cu", "6a793f0316d260fb"),
+    "attn_partials": (1.01, "kvs_flash_tc.cu", "9633504f2a4cc309"),
     "merge_compact": (0.98, "kvs_compact.cu", "c28752d898c08b93"),
 }
 
