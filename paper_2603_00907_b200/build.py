@@ -35,7 +35,7 @@ def build(force: bool = False, verbose: bool = False, extra_flags=()) -> str:
     """Compile every .cu under csrc/ and link libkvs.so next to this file."""
     os.makedirs(OBJ, exist_ok=True)
     sources = sorted(f for f in os.listdir(CSRC) if f.endswith(".cu"))
-    headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".h")]
+    headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
     headers.append(os.path.join(ROOT, "include", "kvs.h"))
     nvcc = _nvcc()
     jobs = []

@@ -1,20 +1,25 @@
 // Attention partials on the tensor cores (tcgen05 + TMEM + TMA), queries on TMEM lanes.
 //
-// One CTA owns a block of 128 query rows (Q stays in shared memory) and a contiguous range
+// One CTA owns a block of 128 query rows (Q is staged once and copied into tensor memory) and a contiguous range
 // of 128-slot tiles.  K and V tiles travel in two separate two-stage TMA rings; per tile one
 // thread issues
-//   S[q, slot] = Q K_tile^T                         (fp32 in TMEM, double buffered)
-// Sixteen softmax warps share the tile: the four warps of a TMEM lane quarter own the same 32
-// query rows and 32 slot columns each.  A thread finds the maximum of its 32 logits; the four
-// threads of a row agree on the row maximum through a shared-memory atomic maximum, keep the
-// same stabiliser m (it only moves when the maximum grows by more than 2^8, in which case the
-// first of the four rescales the row of O in TMEM), and each writes P' = exp(s - m), split
-// into two bf16 terms, back into the tensor-memory columns the logits came from, keeping its
-// part of l = sum_j c_j exp(s_j - m): the count bias ln c_j of a merged slot is just the factor
-// c_j in that sum.  The issuing thread then runs
+//   S[q, slot] = Q K_tile^T                         (fp32 in TMEM, double buffered; Q is read from TMEM too,
+//                                                    so that only the K rows cross the shared-memory port)
+// Two teams of eight softmax warps take alternate tiles, so that one team's arithmetic overlaps
+// the other team's waits.  Inside a team the two warps of a TMEM lane quarter own the same 32
+// query rows and 64 slot columns each.  A thread reads its logits twice: once for the maximum
+// (the two threads of a row agree on the row maximum through a shared-memory atomic maximum),
+// once to form P' = exp(s - m), split into two bf16 terms and stored back into the very columns
+// the thread's logits came from (32 logits make 16 columns of hi and 16 of lo terms), keeping
+// its part of l = sum_j c_j exp(s_j - m): the count bias ln c_j of a merged slot is just the
+// factor c_j in that sum.  The stabiliser m of a row is one value for the whole CTA: it lives in
+// shared memory, is decided tile by tile in tile order (each team waits for the other team's
+// decision on the tile before) and only moves when the maximum has outgrown it by more than 2^8;
+// the team that moves it rescales the row of O, and every thread brings its own part of l along
+// when it next sees the new value.  The issuing thread then runs
 //   O[q, :] += (P'_hi + P'_lo) Vsum_tile            (P' from tensor memory, V as the MN-major operand)
-// with O accumulating in TMEM across the tiles [Eq. attn_def_vec with merged slots:
-// o = sum_j alpha_j Vsum_j / c_j].  At the end (stabiliser, sum, O) is written as the partial
+// with the one O accumulating in TMEM across all tiles [Eq. attn_def_vec with merged slots:
+// o = sum_j alpha_j Vsum_j / c_j].  At the end the CTA writes (stabiliser, sum, O) as the partial
 // of this key range.  Window queries and decode queries use the same kernel.
 //
 // Four more warps serve the statistics pass that follows the window attention: tiles are then
@@ -39,19 +44,17 @@ constexpr int kThreads = (2 + kSoftmaxWarps + kNormWarps) * 32;   // warp 0: TMA
 constexpr float kRescaleGap = 8.f;         // log2 units
 
 struct Misc {
-  uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[2], pready[2], ofull[2], qfull;
+  uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[2], pready[2][2], ofull[2], stabdone[2], qfull, qready;
   uint32_t tmem_base;
   int abort_flag;
-  union {
-    struct {
-      uint32_t rowmax[3][kTile];           // per tile (mod 3) and query row: maximum logit, as an ordered integer
-      alignas(16) float cnt[2][kTile];     // per tile parity: counts of the tile's slots (read as float4)
-    };
-    float lsum[4][kTile];                  // after the last tile: the column groups' parts of the row sums
-  };
+  uint32_t rowmax[2][3][kTile];            // per team, team tile (mod 3) and query row: maximum logit, as an ordered integer
+  alignas(16) float cnt[2][2][kTile];      // per team and tile parity: counts of the tile's slots (read as float4)
+  float mstab[2][kTile];                   // per tile parity and query row: the stabiliser after that tile (-inf: none yet)
+  float lsum[4][kTile];                    // the four parts of every row sum (team x column half)
 };
 constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc);
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
+constexpr uint32_t kColQ = 256, kColO = 384;   // TMEM columns: two logit buffers of 128, Q (64), O (128)
 
 constexpr uint32_t kOrdNegInf = 0x007fffffu;   // ordered-integer image of -infinity
 // monotone map float -> unsigned (so that an integer maximum is the float maximum) and back
@@ -63,7 +66,29 @@ __device__ __forceinline__ float ord2f(uint32_t u) {
   return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
 }
 
-__device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 1, 512;" ::: "memory"); }
+// A load that stays where it is written: the compiler may move a plain load of a value that is
+// only needed one tile later down to its use, which puts the memory latency back on the tile.
+__device__ __forceinline__ int ldg_here(const int32_t* p) {
+  int v;
+  asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+
+// tcgen05.mma, A from tensor memory, with the shared-memory descriptor given as its two words and
+// the accumulate flag known at compile time: two additions and the product itself per call.
+template <bool kAccumulate>
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 bd;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 bd, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(kAccumulate ? 1 : 0)
+      : "memory");
+}
+
+__device__ __forceinline__ void team_barrier(int team) { asm volatile("bar.sync %0, 256;" ::"r"(team + 1) : "memory"); }
+__device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 3, 512;" ::: "memory"); }
 
 // One lane polls, the warp follows.  A failed wait (time-out or abort) only makes the warp skip
 // its work: it still goes through the tile loop and its one named barrier per tile, so that no
@@ -123,15 +148,14 @@ __device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], 
 }
 
 // For the 8 pairs (rows 2i, 2i+1) of rows [row0, row0 + 16) of one staged operand: |x_l|^2,
-// |x_r|^2 and <x_l, x_r>, delivered to lanes 0-7.  A = [x_l rows ; x_r rows] (16 x 128) against
-// B = x_r and B = x_l (8 rows each): the wanted values are diagonal elements of the two
-// 16 x 8 products.  All fragments are loaded first, then two accumulation chains run.
+// |x_r|^2 and <x_l, x_r>, delivered to lanes 0-7 (and again to lanes 8-15).  The 16 rows are the
+// A operand and, eight at a time, the B operand of small tensor-core products: the wanted values
+// sit on and next to the diagonal of the 16 x 16 Gram matrix.  Every 8 x 8 fragment is eight
+// consecutive rows, which the 128-byte swizzle spreads over all banks.
 __device__ __forceinline__ void pair_dots8(const uint8_t* tile, int row0, int lane, float& ll, float& rr, float& lr) {
   const uint32_t base = smem_u32(tile);
   const int mtx = lane >> 3, rin = lane & 7;                // ldmatrix: this lane feeds row rin of matrix mtx
-  const int g = lane >> 2;                                  // accumulator row held by this lane
-  const int src = 4 * (lane & 7) + ((lane & 7) >> 1);       // lane that holds the diagonal of pair (lane & 7)
-  const int row = row0 + 2 * rin + (mtx & 1);               // matrices 0,2: left rows; 1,3: right rows
+  const int row = row0 + (mtx & 1) * 8 + rin;               // matrices 0,2: rows 0-7; 1,3: rows 8-15
   uint32_t fr[8][4];
 #pragma unroll
   for (int kk = 0; kk < 8; ++kk) {
@@ -141,15 +165,20 @@ __device__ __forceinline__ void pair_dots8(const uint8_t* tile, int row0, int la
   float d1[4] = {0.f, 0.f, 0.f, 0.f}, d2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
   for (int kk = 0; kk < 8; ++kk) {
-    mma16816(d1, fr[kk], fr[kk][1], fr[kk][3]);             // columns = right rows
-    mma16816(d2, fr[kk], fr[kk][0], fr[kk][2]);             // columns = left rows
+    mma16816(d1, fr[kk], fr[kk][0], fr[kk][2]);             // columns = rows 0-7
+    mma16816(d2, fr[kk], fr[kk][1], fr[kk][3]);             // columns = rows 8-15
   }
-  const float v_lr = (g & 1) ? d1[1] : d1[0];               // row g (left), column g (right)
-  const float v_rr = (g & 1) ? d1[3] : d1[2];               // row 8 + g (right), column g (right)
-  const float v_ll = (g & 1) ? d2[1] : d2[0];               // row g (left), column g (left)
-  lr = __shfl_sync(0xffffffffu, v_lr, src);
-  rr = __shfl_sync(0xffffffffu, v_rr, src);
-  ll = __shfl_sync(0xffffffffu, v_ll, src);
+  // lane 4 g + t holds rows g and g + 8, columns 2 t and 2 t + 1.  Pair q < 4 (rows 2q, 2q+1, first
+  // product): lane 9 q has <l,l> and <l,r>, lane 9 q + 4 has <r,r>; pair 4 + q the same lanes, in
+  // the lower half of the second product.
+  const int q = lane & 3, srcl = 9 * q, srcr = 9 * q + 4;
+  const bool upper = (lane & 4) != 0;
+  const float ll1 = __shfl_sync(0xffffffffu, d1[0], srcl), ll2 = __shfl_sync(0xffffffffu, d2[2], srcl);
+  const float lr1 = __shfl_sync(0xffffffffu, d1[1], srcl), lr2 = __shfl_sync(0xffffffffu, d2[3], srcl);
+  const float rr1 = __shfl_sync(0xffffffffu, d1[1], srcr), rr2 = __shfl_sync(0xffffffffu, d2[3], srcr);
+  ll = upper ? ll2 : ll1;
+  lr = upper ? lr2 : lr1;
+  rr = upper ? rr2 : rr1;
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -198,19 +227,19 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       mbar_init(&misc->vfull[s], 1);
       mbar_init(&misc->kfree[s], norm_k ? 1 + kNormWarps : 1);   // MMA commit (+ the pair-norm warps)
       mbar_init(&misc->vfree[s], norm_v ? 1 + kNormWarps : 1);
+      mbar_init(&misc->stabdone[s], kSoftmaxWarps / 2);
       mbar_init(&misc->sfull[s], 1);
-    }
-    // P' is handed over in two halves (the first and the last 16 slots of every column group), so
-    // that the P V products of one half run while the other half is still being written
-    for (int hf = 0; hf < 2; ++hf) {
-      mbar_init(&misc->pready[hf], kSoftmaxWarps);
-      mbar_init(&misc->ofull[hf], 1);
+      mbar_init(&misc->ofull[s], 1);
+      // P' is handed over in two halves (the last and the first 32 slots of every thread's 64), so
+      // that the P V products of one half run while the other half is still being written
+      for (int hf = 0; hf < 2; ++hf) mbar_init(&misc->pready[s][hf], kSoftmaxWarps / 2);
     }
     mbar_init(&misc->qfull, 1);
+    mbar_init(&misc->qready, kSoftmaxWarps);
     misc->abort_flag = 0;
     mbar_fence_init();
   }
-  if (threadIdx.x < 3 * kTile) misc->rowmax[threadIdx.x / kTile][threadIdx.x % kTile] = kOrdNegInf;
+  for (int i = threadIdx.x; i < 2 * 3 * kTile; i += kThreads) (&misc->rowmax[0][0][0])[i] = kOrdNegInf;
   if (warp == 1) tmem_alloc(&misc->tmem_base, 512);
   tc_fence_before();
   __syncthreads();
@@ -220,41 +249,39 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
 
   if (warp == 0) {
     // ================================================================ TMA producer
-    // one thread streams both rings: whichever of the next K tile and the next V tile has a free
-    // stage is requested first
+    // one thread streams both rings.  Stages come free in a fixed order (the logits of tile t + 1 are
+    // queued before the P V products of tile t), so the thread sleeps on one barrier at a time:
+    // K(0), K(1), V(0), K(2), V(1), ...
     if (lane == 0) {
       prefetch_tmap(&tmK); prefetch_tmap(&tmV); prefetch_tmap(&tmQ);
       mbar_expect_tx(&misc->qfull, kOperand);
       for (int hf = 0; hf < 2; ++hf)
         tma_load_3d(smem + kSmemQ + hf * kHalf, &tmQ, &misc->qfull, hf * 64, qblk * 128, unit);
       int kli = 0, vli = 0;
-      uint64_t t0 = globaltimer_ns();
-      while (kli < my_tiles || vli < my_tiles) {
-        bool progress = false;
-        if (kli < my_tiles && mbar_try_wait(&misc->kfree[kli & 1], ((kli >> 1) & 1) ^ 1)) {
-          const int s = kli & 1;
-          uint8_t* st = smem + kSmemStage + s * kStage;
-          const int row = (t_begin + kli) * kTile - shift;
-          mbar_expect_tx(&misc->kfull[s], kOperand);
-          for (int hf = 0; hf < 2; ++hf) tma_load_4d(st + hf * kHalf, &tmK, &misc->kfull[s], hf * 64, row, h, sr.b);
-          ++kli;
-          progress = true;
-        }
-        if (vli < my_tiles && mbar_try_wait(&misc->vfree[vli & 1], ((vli >> 1) & 1) ^ 1)) {
-          const int s = vli & 1;
-          uint8_t* st = smem + kSmemStage + s * kStage + kOperand;
-          const int row = (t_begin + vli) * kTile - shift;
-          mbar_expect_tx(&misc->vfull[s], kOperand);
-          for (int hf = 0; hf < 2; ++hf) tma_load_4d(st + hf * kHalf, &tmV, &misc->vfull[s], hf * 64, row, h, sr.b);
-          ++vli;
-          progress = true;
-        }
-        if (progress) {
-          t0 = globaltimer_ns();
-        } else {
-          if (*abort_flag) break;
-          if (globaltimer_ns() - t0 > 1000000000ull) { *abort_flag = 1; break; }
-        }
+      auto load_k = [&]() -> bool {
+        const int s = kli & 1;
+        if (!mbar_wait(&misc->kfree[s], ((kli >> 1) & 1) ^ 1, abort_flag)) return false;
+        uint8_t* st = smem + kSmemStage + s * kStage;
+        const int row = (t_begin + kli) * kTile - shift;
+        mbar_expect_tx(&misc->kfull[s], kOperand);
+        for (int hf = 0; hf < 2; ++hf) tma_load_4d(st + hf * kHalf, &tmK, &misc->kfull[s], hf * 64, row, h, sr.b);
+        ++kli;
+        return true;
+      };
+      auto load_v = [&]() -> bool {
+        const int s = vli & 1;
+        if (!mbar_wait(&misc->vfree[s], ((vli >> 1) & 1) ^ 1, abort_flag)) return false;
+        uint8_t* st = smem + kSmemStage + s * kStage + kOperand;
+        const int row = (t_begin + vli) * kTile - shift;
+        mbar_expect_tx(&misc->vfull[s], kOperand);
+        for (int hf = 0; hf < 2; ++hf) tma_load_4d(st + hf * kHalf, &tmV, &misc->vfull[s], hf * 64, row, h, sr.b);
+        ++vli;
+        return true;
+      };
+      bool ok = load_k();
+      while (ok && vli < my_tiles) {
+        if (kli < my_tiles) ok = load_k();
+        if (ok) ok = load_v();
       }
       if (*abort_flag) {
         // drain: give the copies already issued a bounded time to land before the CTA leaves
@@ -271,51 +298,64 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
   } else if (warp == 1) {
     // ================================================================ MMA issuer
     if (lane == 0) {
+      // One thread feeds the tensor pipe, so every instruction between two products counts: the
+      // descriptors are kept as a constant high word and a low word that only needs an addition.
       constexpr uint32_t idesc_s = idesc_bf16(128, 128);                 // Q (K-major) x K tile (K-major)
       constexpr uint32_t idesc_o = idesc_bf16(128, 128, false, true);    // P' (K-major) x V tile (MN-major)
-      const uint32_t q_addr = smem_u32(smem + kSmemQ);
+      const uint64_t kd0 = smem_desc_sw128(smem_u32(smem + kSmemStage), 16, 1024);
+      const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + kSmemStage + kOperand), kHalf, 1024);
+      const uint32_t kd_hi = (uint32_t)(kd0 >> 32), vd_hi = (uint32_t)(vd0 >> 32);
+      const uint32_t kd_lo0 = (uint32_t)kd0, vd_lo0 = (uint32_t)vd0;     // stage 0; stage 1 is kStage / 16 further
       auto issue_s = [&](int li) -> bool {
-        const int s = li & 1, k = li >> 1;
-        // buffer s last held P' of tile li - 2, whose products were issued by this thread before
+        const int s = li & 1, k = li >> 1;                 // K stage = logit buffer
+        // the buffer last held P' of tile li - 2, whose products were issued by this thread before
         if (!mbar_wait(&misc->kfull[s], k & 1, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t k_addr = smem_u32(smem + kSmemStage + s * kStage);
+        const uint32_t kd_lo = kd_lo0 + s * (kStage >> 4), ds = tmem + s * 128;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           const uint32_t o = (kk >> 2) * kHalf + (kk & 3) * 32;
-          umma_bf16(tmem + s * 128, smem_desc_sw128(q_addr + o, 16, 1024), smem_desc_sw128(k_addr + o, 16, 1024),
-                    idesc_s, kk > 0);
+          if (kk == 0) umma_ts<false>(ds, tmem + kColQ, kd_lo, kd_hi, idesc_s);
+          else umma_ts<true>(ds, tmem + kColQ + 8 * kk, kd_lo + (o >> 4), kd_hi, idesc_s);
         }
         tc_commit(&misc->sfull[s]);
         tc_commit(&misc->kfree[s]);
         return true;
       };
-      bool ok = mbar_wait(&misc->qfull, 0, abort_flag);
+      bool ok = mbar_wait(&misc->qready, 0, abort_flag);
+      if (ok) tc_fence_after();
       ok = ok && issue_s(0);
       for (int li = 0; ok && li < my_tiles; ++li) {
+        // the next tile's logits are queued before this tile's P V products
         if (li + 1 < my_tiles) ok = issue_s(li + 1);
-        const int s = li & 1;
-        const uint32_t v_addr = smem_u32(smem + kSmemStage + s * kStage + kOperand);
-        if (ok && !mbar_wait(&misc->vfull[s], (li >> 1) & 1, abort_flag)) ok = false;
-        const uint32_t dO = tmem + 256;
-        for (int hf = 0; ok && hf < 2; ++hf) {
-          if (!mbar_wait(&misc->pready[hf], li & 1, abort_flag)) { ok = false; break; }
-          tc_fence_after();
+        const int s = li & 1, ph = (li >> 1) & 1;          // V stage = logit buffer
+        if (ok && !mbar_wait(&misc->vfull[s], ph, abort_flag)) ok = false;
+        const uint32_t vd_lo = vd_lo0 + s * (kStage >> 4), ps = tmem + s * 128;
 #pragma unroll
-          for (int cgi = 0; cgi < 4; ++cgi) {
-            const int kk = 2 * cgi + hf;                     // 16-slot step of the tile: slots [16 kk, 16 kk + 16)
+        for (int hf = 0; hf < 2; ++hf) {
+          if (ok && !mbar_wait(&misc->pready[s][hf], ph, abort_flag)) ok = false;
+          if (!ok) break;
+          tc_fence_after();
+          const int sub = 1 - hf;                            // the last 32 slots of a thread's 64 come first
+#pragma unroll
+          for (int c4 = 0; c4 < 4; ++c4) {
+            const int ch = c4 >> 1, k2 = c4 & 1;
+            const int kk = 4 * ch + 2 * sub + k2;            // 16-slot step of the tile: slots [16 kk, 16 kk + 16)
 #pragma unroll
             for (int hl = 0; hl < 2; ++hl) {
-              // A: 16 slots = 8 columns of P'_hi (columns 0-63 of the logit buffer) or P'_lo (64-127);
-              // B: 16 slots = two 8-row groups of V
-              const uint32_t ap = tmem + s * 128 + hl * 64 + kk * 8;
-              const uint64_t bd = smem_desc_sw128(v_addr + (kk * 16) * 128, kHalf, 1024);
-              umma_bf16_ts(dO, ap, bd, idesc_o, (li > 0 || hf > 0 || cgi > 0 || hl > 0) ? 1u : 0u);
+              // A: 16 slots = 8 columns of hi (or, 16 columns further, lo) terms inside the owner's
+              // 64 logit columns; B: 16 slots = two 8-row groups of V
+              const uint32_t ap = ps + 64 * ch + 32 * sub + 16 * hl + 8 * k2;
+              const uint32_t bl = vd_lo + ((kk * 16 * 128) >> 4);
+              if (hf == 0 && c4 == 0 && hl == 0) umma_bf16_ts(tmem + kColO, ap, ((uint64_t)vd_hi << 32) | bl, idesc_o, li > 0 ? 1u : 0u);
+              else umma_ts<true>(tmem + kColO, ap, bl, vd_hi, idesc_o);
             }
           }
-          tc_commit(&misc->ofull[hf]);
         }
-        if (ok) tc_commit(&misc->vfree[s]);
+        if (ok) {
+          tc_commit(&misc->ofull[s]);
+          tc_commit(&misc->vfree[s]);
+        }
       }
     }
   } else if (warp >= 2 + kSoftmaxWarps) {
@@ -326,21 +366,21 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       const int32_t* Cn = a.counts + (size_t)unit * a.n_max;
       const int pl = lane & 15;                                  // lanes 0-15 own the warp's 16 pairs
       // counts of the next tile's pair travel while the current tile is processed
-      float cl_next = 1.f, cr_next = 1.f;
+      int cl_next = 1, cr_next = 1;
       if (norm_v) {
         const int sl = t_begin * kTile - shift + nw * 32 + 2 * pl;
-        if (sl >= off && ((sl - off) >> 1) < sr.P) { cl_next = (float)Cn[sl]; cr_next = (float)Cn[sl + 1]; }
+        if (sl >= off && ((sl - off) >> 1) < sr.P) { cl_next = ldg_here(Cn + sl); cr_next = ldg_here(Cn + sl + 1); }
       }
       for (int li = 0; li < my_tiles; ++li) {
         const int s = li & 1, k = li >> 1;
         const int slot_l = (t_begin + li) * kTile - shift + nw * 32 + 2 * pl;   // left slot of this lane's pair
         const int p = (slot_l - off) >> 1;
         const bool pair_ok = lane < 16 && slot_l >= off && p < sr.P;
-        const float cl = cl_next, cr = cr_next;
+        const int cl = cl_next, cr = cr_next;
         if (norm_v && li + 1 < my_tiles) {
           const int sl = slot_l + kTile;
-          cl_next = cr_next = 1.f;
-          if (sl >= off && ((sl - off) >> 1) < sr.P) { cl_next = (float)Cn[sl]; cr_next = (float)Cn[sl + 1]; }
+          cl_next = cr_next = 1;
+          if (sl >= off && ((sl - off) >> 1) < sr.P) { cl_next = ldg_here(Cn + sl); cr_next = ldg_here(Cn + sl + 1); }
         }
         float* out = reinterpret_cast<float*>(a.pair_norms + (size_t)unit * a.pair_stride + (pair_ok ? p : 0));
         const uint8_t* st = smem + kSmemStage + s * kStage;
@@ -368,7 +408,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
           const bool b = (lane >> 3) & 1;
           const float vll = b ? ll[1] : ll[0], vrr = b ? rr[1] : rr[0], vlr = b ? lr[1] : lr[0];
           if (pair_ok) {
-            const float icl = 1.f / cl, icr = 1.f / cr;
+            const float icl = 1.f / (float)cl, icr = 1.f / (float)cr;
             const float r2l = vll * icl * icl, r2r = vrr * icr * icr;
             out[0] = r2l; out[1] = r2r; out[2] = r2l + r2r + 2.f * vlr * icl * icr;
           }
@@ -377,161 +417,202 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     }
   } else {
     // ================================================================ softmax warps
-    const int cg = (warp - 2) >> 2;                       // 32-slot column group of the tile
+    const int team = (warp - 2) >> 3;                     // takes tiles li = team, team + 2, ...
+    const int ch = ((warp - 2) >> 2) & 1;                 // 64-slot column half of the tile
     const int row = (warp & 3) * 32 + lane;               // TMEM lane = query row in the block
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
     const int m = qblk * 128 + row;
     const int last_vis = a.causal ? (n - a.Wq + (m % a.Wq)) : (n - 1);
+    const int last_free = min(n - 1, a.causal ? n - a.Wq : n - 1);   // slots up to here need no mask
     const int32_t* Cb = a.counts + (size_t)unit * a.n_max;
-    // stabiliser in log2 units; until a row has seen a visible slot it is 0 (keeps the arithmetic finite)
+    const int team_tiles = (my_tiles - team + 1) / 2;
+    // The stabiliser (log2 units) this thread's logits and its part of l refer to.  Until the row
+    // has seen a visible slot there is none (-inf in shared memory) and 0 stands in for it, which
+    // keeps the arithmetic finite.
     float m_stab = 0.f, l = 0.f;
     bool have_stab = false;
     bool alive = true;
-    // (first column group) the count of slot `row` of the next tile travels while the current tile is processed
-    int cnt_next = 1;
-    if (cg == 0) {
-      const int j = t_begin * kTile - shift + row;
-      if (j >= 0 && j < n) cnt_next = Cb[j];
+    // Q into tensor memory: row on its lane, two channels per 32-bit column; each of the four
+    // warps of a lane quarter copies 32 channels (rows past the last query were staged as zeros)
+    {
+      const int part = ((warp - 2) >> 2);                  // channels [32 part, 32 part + 32)
+      alive = warp_wait(&misc->qfull, 0, abort_flag, lane);
+      const uint8_t* qrow = smem + kSmemQ + (part >> 1) * kHalf + row * 128;
+      uint32_t qv[16];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int c = (part & 1) * 4 + i;
+        const uint4 v = *reinterpret_cast<const uint4*>(qrow + ((c ^ (row & 7)) << 4));
+        qv[4 * i] = v.x; qv[4 * i + 1] = v.y; qv[4 * i + 2] = v.z; qv[4 * i + 3] = v.w;
+      }
+      tmem_st8(tmem + lane_addr + kColQ + part * 16, qv);
+      tmem_st8(tmem + lane_addr + kColQ + part * 16 + 8, qv + 8);
+      tmem_st_wait();
+      tc_fence_before();
+      warp_arrive(&misc->qready, lane);
     }
-    for (int li = 0; li < my_tiles; ++li) {
-      const int s = li & 1, k = li >> 1;
-      const int j0 = (t_begin + li) * kTile - shift + cg * 32;    // first slot of this thread's columns
-      float* cnt = misc->cnt[s];
-      uint32_t* rmax = misc->rowmax[li % 3];
-      if (cg == 0) {
-        cnt[row] = (float)cnt_next;
-        const int j = (t_begin + li + 1) * kTile - shift + row;
-        cnt_next = (li + 1 < my_tiles && j >= 0 && j < n) ? Cb[j] : 1;
-      }
-      float x[32];
-      if (alive) alive = warp_wait(&misc->sfull[s], k & 1, abort_flag, lane);
-      if (alive) {
-        tc_fence_after();
-        tmem_ld32(tmem + lane_addr + s * 128 + cg * 32, x);
-        tmem_ld_wait();
-        // logits in log2 units relative to the stabiliser (one multiply-add), with mask; the stabiliser
-        // ignores the counts: exp(s - m) <= 1 either way
-        const bool need_mask = (j0 < 0) || (j0 + 31 > min(n - 1, a.causal ? n - a.Wq : n - 1));
-        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one
-        if (!need_mask) {
+    // (first column half) the count of slot `row` of the team's next tile travels meanwhile
+    int cnt_next = 1;
+    if (ch == 0 && team_tiles > 0) {
+      const int jj = (t_begin + team) * kTile - shift + row;
+      if (jj >= 0 && jj < n) cnt_next = ldg_here(Cb + jj);
+    }
+    // logits of 32 columns, relative to the stabiliser (one multiply-add), masked where needed
+    auto load32 = [&](uint32_t col, int j0, float* x) {
+      tmem_ld32(col, x);
+      tmem_ld_wait();
+      if (j0 >= 0 && j0 + 31 <= last_free) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            x[i] = fmaf(x[i], a.scale_log2, -m_stab);
-            mx[i & 3] = fmaxf(mx[i & 3], x[i]);
-          }
-        } else {
+        for (int i = 0; i < 32; ++i) x[i] = fmaf(x[i], a.scale_log2, -m_stab);
+      } else {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float v = fmaf(x[i], a.scale_log2, -m_stab);
-            x[i] = (j0 + i >= 0 && j0 + i <= last_vis) ? v : -INFINITY;
-            mx[i & 3] = fmaxf(mx[i & 3], x[i]);
-          }
-        }
-        atomicMax(&rmax[row], f2ord(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]))));
+        for (int i = 0; i < 32; ++i)
+          x[i] = (j0 + i >= 0 && j0 + i <= last_vis) ? fmaf(x[i], a.scale_log2, -m_stab) : -INFINITY;
       }
-      // the one barrier of the tile: the row maxima and the staged counts are complete
-      softmax_barrier();
-      // the buffer of the tile after next was last read one tile ago: every thread is past that read now
-      if (cg == 0) misc->rowmax[(li + 2) % 3][row] = kOrdNegInf;
-      if (!alive) continue;
-      // row maximum relative to the stabiliser: the stabiliser moves up by it when the row has none
-      // yet or when the maximum has outgrown it by more than the gap
-      const float mt = ord2f(rmax[row]);
-      const bool need = mt > -INFINITY && (!have_stab || mt > kRescaleGap);
-      const bool any_need = __any_sync(0xffffffffu, need && li > 0);
-      // the previous tile's P V products must be done before P is overwritten: half by half, or
-      // both before a rescale of O
-      if (li > 0) {
-        if (!(alive = warp_wait(&misc->ofull[0], (li - 1) & 1, abort_flag, lane))) continue;
-        if (any_need && !(alive = warp_wait(&misc->ofull[1], (li - 1) & 1, abort_flag, lane))) continue;
-        tc_fence_after();
-      }
-      const float f = (need && have_stab) ? fast_exp2(-mt) : 1.f;
-      if (any_need) {
-        if (cg == 0) {                                     // the row of O is rescaled once
-#pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            float ov[32];
-            tmem_ld32(tmem + lane_addr + 256 + c * 32, ov);
-            tmem_ld_wait();
+    };
+    auto max32 = [&](const float* x) {
+      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one
 #pragma unroll
-            for (int i = 0; i < 32; ++i) ov[i] *= f;
-            tmem_st32(tmem + lane_addr + 256 + c * 32, ov);
-          }
-          tmem_st_wait();
-        }
-        l *= f;
-      }
-      if (need) {
-        m_stab += mt;
-        have_stab = true;
-#pragma unroll
-        for (int i = 0; i < 32; ++i) x[i] -= mt;
-      }
-      // rows of the V tile outside the sequence may hold anything: each warp zeroes its share
-      const int tile_row0 = (t_begin + li) * kTile - shift;
-      if (tile_row0 < 0 || tile_row0 + kTile > n) {
-        if (!(alive = warp_wait(&misc->vfull[s], k & 1, abort_flag, lane))) continue;
-        uint8_t* vt = smem + kSmemStage + s * kStage + kOperand;
-        for (int it = threadIdx.x - 64; it < kTile * 16; it += kSoftmaxWarps * 32) {
-          const int r = it >> 4, ch = it & 15;
-          if (tile_row0 + r < 0 || tile_row0 + r >= n)
-            *reinterpret_cast<uint4*>(vt + (ch >> 3) * kHalf + r * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
-        }
-        fence_proxy_async();                               // the tensor core reads these rows
-      }
-      // P' = exp2(x - m) as hi + lo bf16, two slots per 32-bit column, written over the logits of
-      // this buffer (every warp has read its logits: the barrier above) as the A operand of P' V:
-      // hi in columns 0-63, lo in columns 64-127.  The hi term is the value cut to bf16 (a byte
-      // permute, no conversion); the lo term rounds the exact remainder, so hi + lo carries 16
-      // significant bits.
+      for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], x[i]);
+      return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+    };
+    // P' = exp2(x) of 32 slots as hi + lo bf16, two slots per 32-bit column, stored over the first
+    // 16 (hi) and the last 16 (lo) of the 32 columns the logits were read from.  The hi term is the
+    // value cut to bf16 (a byte permute, no conversion); the lo term rounds the exact remainder, so
+    // hi + lo carries 16 significant bits.  Returns sum_j c_j P'_j.
+    auto emit32 = [&](uint32_t col, const float* x, const float* cnt32) {
       float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        if (hf == 1 && li > 0 && !any_need) {
-          if (!(alive = warp_wait(&misc->ofull[1], (li - 1) & 1, abort_flag, lane))) break;
-        }
+      for (int c = 0; c < 4; c += 2) {
         uint32_t hi[8], lo[8];
 #pragma unroll
-        for (int c = 2 * hf; c < 2 * hf + 2; ++c) {
-          const float4 ca = *reinterpret_cast<const float4*>(&cnt[cg * 32 + c * 8]);
-          const float4 cb = *reinterpret_cast<const float4*>(&cnt[cg * 32 + c * 8 + 4]);
+        for (int c2 = c; c2 < c + 2; ++c2) {
+          const float4 ca = *reinterpret_cast<const float4*>(&cnt32[c2 * 8]);
+          const float4 cb = *reinterpret_cast<const float4*>(&cnt32[c2 * 8 + 4]);
           const float cc[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
-            const int i = c * 8 + u * 2;
+            const int i = c2 * 8 + u * 2;
             const float q0 = fast_exp2(x[i]), q1 = fast_exp2(x[i + 1]);
             ls[u] = fmaf(cc[2 * u], q0, fmaf(cc[2 * u + 1], q1, ls[u]));
             const uint32_t b0 = __float_as_uint(q0), b1 = __float_as_uint(q1);
-            hi[(c & 1) * 4 + u] = __byte_perm(b0, b1, 0x7632);
-            lo[(c & 1) * 4 + u] = pack_bf16(q0 - __uint_as_float(b0 & 0xffff0000u), q1 - __uint_as_float(b1 & 0xffff0000u));
+            hi[(c2 & 1) * 4 + u] = __byte_perm(b0, b1, 0x7632);
+            lo[(c2 & 1) * 4 + u] = pack_bf16(q0 - __uint_as_float(b0 & 0xffff0000u), q1 - __uint_as_float(b1 & 0xffff0000u));
           }
         }
-        tmem_st8(tmem + lane_addr + s * 128 + cg * 16 + hf * 8, hi);
-        tmem_st8(tmem + lane_addr + s * 128 + 64 + cg * 16 + hf * 8, lo);
-        tmem_st_wait();
-        tc_fence_before();
-        warp_arrive(&misc->pready[hf], lane);
+        tmem_st8(col + (c >> 1) * 8, hi);
+        tmem_st8(col + 16 + (c >> 1) * 8, lo);
       }
+      tmem_st_wait();
+      return (ls[0] + ls[1]) + (ls[2] + ls[3]);
+    };
+    for (int j = 0; j < team_tiles; ++j) {
+      const int li = 2 * j + team;
+      const int s = li & 1, b = li & 1, ph = j & 1;        // K/V stage, logit buffer and its phase
+      const uint32_t scol = tmem + lane_addr + b * 128 + ch * 64;   // this thread's 64 logit columns
+      const int tile_row0 = (t_begin + li) * kTile - shift;
+      const int jA = tile_row0 + ch * 64, jB = jA + 32;    // first slots of this thread's two column groups
+      float* cnt = misc->cnt[team][j & 1];
+      uint32_t* rmax = misc->rowmax[team][j % 3];
+      if (ch == 0) {
+        cnt[row] = (float)cnt_next;
+        const int jj = tile_row0 + 2 * kTile + row;
+        cnt_next = 1;
+        if (j + 1 < team_tiles && jj >= 0 && jj < n) cnt_next = ldg_here(Cb + jj);
+      }
+      float x[32];
+      if (alive) alive = warp_wait(&misc->sfull[b], ph, abort_flag, lane);
+      if (alive) {
+        tc_fence_after();
+        load32(scol, jA, x);
+        const float mA = max32(x);
+        load32(scol + 32, jB, x);                          // these stay in registers: they are exponentiated first
+        atomicMax(&rmax[row], f2ord(fmaxf(mA, max32(x))));
+      }
+      // the one barrier of the tile: the row maxima and the staged counts of the team are complete
+      team_barrier(team);
+      // the buffer of the team's tile after next was last read one tile ago: every thread is past that read now
+      if (ch == 0) misc->rowmax[team][(j + 2) % 3][row] = kOrdNegInf;
+      // ---- the stabiliser after this tile, from the one after the tile before (the other team's decision)
+      float m_prev = -INFINITY;
+      if (li > 0) {
+        if (alive) alive = warp_wait(&misc->stabdone[team ^ 1], ((li - 1) >> 1) & 1, abort_flag, lane);
+        m_prev = misc->mstab[(li - 1) & 1][row];
+      }
+      // row maximum of the tile: it becomes the stabiliser when the row has none yet or when it
+      // has outgrown the stabiliser by more than the gap
+      const float mt = alive ? ord2f(rmax[row]) + m_stab : -INFINITY;
+      const bool need = mt > -INFINITY && (m_prev == -INFINITY || mt - m_prev > kRescaleGap);
+      const float m_new = need ? mt : m_prev;
+      if (ch == 0) misc->mstab[li & 1][row] = m_new;
+      warp_arrive(&misc->stabdone[team], lane);            // also when this warp has given up: the other team waits for it
       if (!alive) continue;
-      l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+      const bool rescale = need && m_prev > -INFINITY;
+      if (__any_sync(0xffffffffu, rescale)) {
+        // all earlier P V products must be done before O is touched
+        if (!(alive = warp_wait(&misc->ofull[(li - 1) & 1], ((li - 1) >> 1) & 1, abort_flag, lane))) continue;
+        tc_fence_after();
+        if (ch == 0) {                                     // the row of O is rescaled once
+          const float f = rescale ? fast_exp2(m_prev - m_new) : 1.f;
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            float ov[32];
+            tmem_ld32(tmem + lane_addr + kColO + c * 32, ov);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) ov[i] *= f;
+            tmem_st32(tmem + lane_addr + kColO + c * 32, ov);
+          }
+          tmem_st_wait();
+        }
+      }
+      // this thread's logits and its part of l follow (the stabiliser may have moved one tile ago too)
+      const float m_eff = m_new > -INFINITY ? m_new : 0.f;
+      if (m_eff != m_stab) {
+        const float d = m_eff - m_stab;
+        if (have_stab) l *= fast_exp2(-d);                 // (without one, l is still 0 and d may be anything)
+        m_stab = m_eff;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) x[i] -= d;
+      }
+      have_stab = m_new > -INFINITY;
+      // rows of the V tile outside the sequence may hold anything: the team zeroes them
+      if (tile_row0 < 0 || tile_row0 + kTile > n) {
+        if (!(alive = warp_wait(&misc->vfull[s], (li >> 1) & 1, abort_flag, lane))) continue;
+        uint8_t* vt = smem + kSmemStage + s * kStage + kOperand;
+        for (int it = (threadIdx.x - 64) & 255; it < kTile * 16; it += 256) {
+          const int r = it >> 4, c16 = it & 15;
+          if (tile_row0 + r < 0 || tile_row0 + r >= n)
+            *reinterpret_cast<uint4*>(vt + (c16 >> 3) * kHalf + r * 128 + ((c16 & 7) << 4)) = make_uint4(0, 0, 0, 0);
+        }
+        fence_proxy_async();                               // the tensor core reads these rows
+      }
+      // the last 32 slots first (their logits are still in registers), then the first 32 again from TMEM
+      l += emit32(scol + 32, x, cnt + ch * 64 + 32);
+      tc_fence_before();
+      warp_arrive(&misc->pready[b][0], lane);
+      load32(scol, jA, x);
+      l += emit32(scol, x, cnt + ch * 64);
+      tc_fence_before();
+      warp_arrive(&misc->pready[b][1], lane);
     }
-    // ---- the partial of this key range: the four column groups of a row add their sums, then each
-    //      writes 32 channels of the row of O
-    softmax_barrier();                                            // row maxima and counts are dead now
-    misc->lsum[cg][row] = l;
+    // ---- the partial of this key range: every thread brings its part of l to the final stabiliser,
+    //      the four parts of a row are added, and each thread writes 32 channels of the row of O
+    softmax_barrier();                                     // the last tile's stabiliser is in place
+    const float m_fin = misc->mstab[(my_tiles - 1) & 1][row];
+    const int part = team * 2 + ch;
+    misc->lsum[part][row] = have_stab ? l * fast_exp2(m_stab - m_fin) : 0.f;
     softmax_barrier();
-    if (alive && warp_wait(&misc->ofull[0], (my_tiles - 1) & 1, abort_flag, lane) &&
-        warp_wait(&misc->ofull[1], (my_tiles - 1) & 1, abort_flag, lane)) {
+    const size_t pidx = ((size_t)unit * a.splits + split) * a.M + m;
+    if (alive && warp_wait(&misc->ofull[(my_tiles - 1) & 1], ((my_tiles - 1) >> 1) & 1, abort_flag, lane)) {
       tc_fence_after();
-      const size_t pidx = ((size_t)unit * a.splits + split) * a.M + m;
-      if (cg == 0 && m < a.M)
-        a.part_ml[pidx] = make_float2(have_stab ? m_stab : -INFINITY, (misc->lsum[0][row] + misc->lsum[1][row]) + (misc->lsum[2][row] + misc->lsum[3][row]));
+      if (part == 0 && m < a.M)
+        a.part_ml[pidx] = make_float2(m_fin, (misc->lsum[0][row] + misc->lsum[1][row]) + (misc->lsum[2][row] + misc->lsum[3][row]));
       float ov[32];
-      tmem_ld32(tmem + lane_addr + 256 + cg * 32, ov);
+      tmem_ld32(tmem + lane_addr + kColO + part * 32, ov);
       tmem_ld_wait();
       if (m < a.M) {
-        float4* po = reinterpret_cast<float4*>(a.part_o + pidx * KVS_D + cg * 32);
+        float4* po = reinterpret_cast<float4*>(a.part_o + pidx * KVS_D + part * 32);
 #pragma unroll
         for (int i = 0; i < 8; ++i) po[i] = make_float4(ov[4 * i], ov[4 * i + 1], ov[4 * i + 2], ov[4 * i + 3]);
       }

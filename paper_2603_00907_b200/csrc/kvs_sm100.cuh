@@ -57,11 +57,36 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parit
       : "memory");
   return ok != 0;
 }
+// Up to `tries` attempts in one tight loop (each attempt may itself sleep in hardware for a short
+// while).  Returns whether the phase completed.
+__device__ __forceinline__ bool mbar_poll(uint64_t* bar, uint32_t parity, uint32_t tries) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
+      "mov.u32 n, %3;\n"
+      "KVS_POLL:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "@p bra KVS_POLL_DONE;\n\t"
+      "sub.u32 n, n, 1;\n\t"
+      "setp.ne.u32 q, n, 0;\n\t"
+      "@q bra KVS_POLL;\n"
+      "KVS_POLL_DONE:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(tries)
+      : "memory");
+  return ok != 0;
+}
 // Bounded wait: false after ~1 s (or when another role already flagged an abort).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// These kernels are chains of hand-offs, so the wake-up latency of a wait counts for more than
+// the issue slots its polling takes: a wait on the critical path (`eager`) polls in a tight
+// loop and looks at the clock only between bursts; a role that runs ahead of the others anyway
+// lets the hardware suspend it between attempts.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          bool eager = false) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
-  while (!mbar_try_wait_hint(bar, parity, 10000u)) {
+  while (!(eager ? mbar_poll(bar, parity, 256) : mbar_try_wait_hint(bar, parity, 10000u))) {
     if (*abort_flag) return false;
     if (globaltimer_ns() - t0 > 1000000000ull) { *abort_flag = 1; return false; }
   }
