@@ -194,7 +194,9 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
   const int qblk = blockIdx.x % a.nqblk;
   const int split = blockIdx.x / a.nqblk;
   const int unit = sr.b * a.Hkv + h;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // (read from one lane, so that the compiler knows the warp index and all that follows from it
+  // -- roles, TMEM and barrier addresses -- to be the same in every lane)
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   // with pair norms, tile t covers slots [128 t - shift, 128 t - shift + 128): aligned with the pairs
   const int shift = a.pair_norms ? (tab.off & 1) : 0;
   const int ntiles = (n + shift + kTile - 1) / kTile;
@@ -244,7 +246,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = misc->tmem_base;
+  const uint32_t tmem = __shfl_sync(0xffffffffu, misc->tmem_base, 0);   // (uniform for the compiler too)
   volatile int* abort_flag = &misc->abort_flag;
 
   if (warp == 0) {

@@ -113,7 +113,9 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
   const int my_tiles = t_end - t_begin;
   const int nh = (min(kQB, a.M - qblk * kQB) > kQH) ? 2 : 1;   // accumulator halves in use
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // (read from one lane, so that the compiler knows the warp index and all that follows from it
+  // -- roles, TMEM and barrier addresses -- to be the same in every lane)
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
     // the staged K rows are free once the last logits are formed, the Vsum rows only after the last
@@ -136,7 +138,7 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = misc->tmem_base;
+  const uint32_t tmem = __shfl_sync(0xffffffffu, misc->tmem_base, 0);   // (uniform for the compiler too)
   volatile int* abort_flag = &misc->abort_flag;
 
   // tensor-map coordinates of the pair members: slot = 2 * rho + parity
