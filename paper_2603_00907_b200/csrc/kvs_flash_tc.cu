@@ -66,27 +66,6 @@ __device__ __forceinline__ float ord2f(uint32_t u) {
   return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
 }
 
-// A load that stays where it is written: the compiler may move a plain load of a value that is
-// only needed one tile later down to its use, which puts the memory latency back on the tile.
-__device__ __forceinline__ int ldg_here(const int32_t* p) {
-  int v;
-  asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(v) : "l"(p));
-  return v;
-}
-
-// tcgen05.mma, A from tensor memory, with the shared-memory descriptor given as its two words and
-// the accumulate flag known at compile time: two additions and the product itself per call.
-template <bool kAccumulate>
-__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t.reg .b64 bd;\n\t"
-      "setp.ne.b32 p, %5, 0;\n\t"
-      "mov.b64 bd, {%2, %3};\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %4, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(kAccumulate ? 1 : 0)
-      : "memory");
-}
-
 __device__ __forceinline__ void team_barrier(int team) { asm volatile("bar.sync %0, 256;" ::"r"(team + 1) : "memory"); }
 __device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 3, 512;" ::: "memory"); }
 

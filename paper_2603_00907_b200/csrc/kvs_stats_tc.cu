@@ -8,8 +8,8 @@
 //   S_l = K_l Q^T, S_r = K_r Q^T                    (logits, fp32 in TMEM)
 //   T_l = Vsum_l (O_hi + O_lo)^T, T_r likewise      (value/output inner products)
 // into one of two TMEM buffers; while the statistics warps reduce one half, the tensor
-// core fills the other.  Each statistics thread owns one pair and reduces over its queries,
-// in registers and with no cross-lane traffic,
+// core fills the other.  Each statistics thread owns one pair and a share of the queries and
+// reduces, in registers and with no cross-lane traffic,
 //   A_j   = sum_q alpha_qj
 //   N1_j  = sum_q alpha |1 - 2 alpha| |vbar_j - o_q|                    [Eqs. c11_def, c22_def]
 //   N12_p = sum_q alpha_j alpha_j+1 |vbar_j + vbar_j+1 - 2 o_q|         [Eq. c12_def]
@@ -35,13 +35,16 @@ constexpr int kOperand = 2 * kHalf;        // a [128 x 128] bf16 operand
 constexpr int kSmemQ = 0, kSmemOhi = kOperand, kSmemOlo = 2 * kOperand;
 constexpr int kSmemKl = 3 * kOperand, kSmemKr = 4 * kOperand, kSmemVl = 5 * kOperand, kSmemVr = 6 * kOperand;
 constexpr int kSmemMisc = 7 * kOperand;
-constexpr int kThreads = 320;              // warp 0: TMA, warp 1: MMA, warps 2-9: statistics
+constexpr int kGroups = 2;                 // statistics groups: a group reduces 64 / kGroups queries of every half
+constexpr int kStatWarps = 4 * kGroups;    // (more warps did not pay: the tensor pipe, not their latency, sets the pace)
+constexpr int kQG = kQH / kGroups;         // queries of a half per group
+constexpr int kThreads = (2 + kStatWarps) * 32;   // warp 0: TMA, warp 1: MMA, warps 2-17: statistics
 
 struct Misc {
-  uint64_t kfull, vfull, kfree, vfree, tfull[2], tfree[2], qfull, xready, xfree;
+  uint64_t kfull, vfull, kfree, vfree, tfull[2], tfree[2], qfull, xhand[kGroups - 1][4], xfree[4];
   uint32_t tmem_base;
   int abort_flag;
-  float xbuf[kPairs * 5];                  // partial sums of the second statistics group, for the first
+  float xbuf[kPairs * 5];                  // partial sums of a pair on their way from the last group down to group 0
 };
 constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc);
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
@@ -126,11 +129,13 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
     mbar_init(&misc->vfree, 1);            // MMA commit
     for (int s = 0; s < 2; ++s) {
       mbar_init(&misc->tfull[s], 1);
-      mbar_init(&misc->tfree[s], 8);       // statistics warps
+      mbar_init(&misc->tfree[s], kStatWarps);   // statistics warps
     }
     mbar_init(&misc->qfull, 1);
-    mbar_init(&misc->xready, 4);           // warps of the second statistics group
-    mbar_init(&misc->xfree, 4);            // warps of the first statistics group
+    for (int q = 0; q < 4; ++q) {          // per TMEM lane quarter: one warp hands over to one warp
+      for (int g = 0; g < kGroups - 1; ++g) mbar_init(&misc->xhand[g][q], 1);
+      mbar_init(&misc->xfree[q], 1);
+    }
     misc->abort_flag = 0;
     mbar_fence_init();
   }
@@ -208,11 +213,13 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
   } else if (warp == 1) {
     // ================================================================ MMA issuer
     if (lane == 0) {
+      // (one thread feeds the tensor pipe with 96 products per tile: descriptors are kept as a
+      // constant high word and low words that only need an addition per product)
       constexpr uint32_t idesc = idesc_bf16(kPairs, kQH);
-      const uint32_t q_addr = smem_u32(smem + kSmemQ), ohi_addr = smem_u32(smem + kSmemOhi),
-                     olo_addr = smem_u32(smem + kSmemOlo);
-      const uint32_t kl = smem_u32(smem + kSmemKl), kr = smem_u32(smem + kSmemKr),
-                     vl = smem_u32(smem + kSmemVl), vr = smem_u32(smem + kSmemVr);
+      const uint32_t dhi = (uint32_t)(smem_desc_sw128(0, 16, 1024) >> 32);
+      auto dlo = [&](int off_bytes) { return (uint32_t)smem_desc_sw128(smem_u32(smem + off_bytes), 16, 1024); };
+      const uint32_t q_lo = dlo(kSmemQ), ohi_lo = dlo(kSmemOhi), olo_lo = dlo(kSmemOlo);
+      const uint32_t kl_lo = dlo(kSmemKl), kr_lo = dlo(kSmemKr), vl_lo = dlo(kSmemVl), vr_lo = dlo(kSmemVr);
       bool ok = mbar_wait(&misc->qfull, 0, abort_flag);
       for (int li = 0; ok && li < my_tiles; ++li) {
         if (!mbar_wait(&misc->kfull, li & 1, abort_flag)) break;
@@ -220,30 +227,35 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
           if (!mbar_wait(&misc->tfree[hq], (li & 1) ^ 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t d0 = tmem + hq * 256;
-          const uint32_t qrow = hq * (kQH * 128);          // rows 64.. of the query-side operands
+          const uint32_t qrow = (uint32_t)(hq * (kQH * 128)) >> 4;   // rows 64.. of the query-side operands
+          const uint32_t qh = q_lo + qrow, oh = ohi_lo + qrow, ol = olo_lo + qrow;
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t o = (kk >> 2) * kHalf + (kk & 3) * 32;
-            umma_bf16(d0, smem_desc_sw128(kl + o, 16, 1024), smem_desc_sw128(q_addr + qrow + o, 16, 1024), idesc, kk > 0);
+            const uint32_t o = ((kk >> 2) * kHalf + (kk & 3) * 32) >> 4;
+            if (kk == 0) umma_ss<false>(d0, kl_lo, dhi, qh, dhi, idesc);
+            else umma_ss<true>(d0, kl_lo + o, dhi, qh + o, dhi, idesc);
           }
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t o = (kk >> 2) * kHalf + (kk & 3) * 32;
-            umma_bf16(d0 + 64, smem_desc_sw128(kr + o, 16, 1024), smem_desc_sw128(q_addr + qrow + o, 16, 1024), idesc, kk > 0);
+            const uint32_t o = ((kk >> 2) * kHalf + (kk & 3) * 32) >> 4;
+            if (kk == 0) umma_ss<false>(d0 + 64, kr_lo, dhi, qh, dhi, idesc);
+            else umma_ss<true>(d0 + 64, kr_lo + o, dhi, qh + o, dhi, idesc);
           }
           if (hq == nh - 1) tc_commit(&misc->kfree);
           if (hq == 0 && !mbar_wait(&misc->vfull, li & 1, abort_flag)) { ok = false; break; }
 #pragma unroll
           for (int kk = 0; kk < 16; ++kk) {
-            const uint32_t o = ((kk & 7) >> 2) * kHalf + (kk & 3) * 32;
-            const uint32_t ob = (kk < 8 ? ohi_addr : olo_addr) + qrow + o;
-            umma_bf16(d0 + 128, smem_desc_sw128(vl + o, 16, 1024), smem_desc_sw128(ob, 16, 1024), idesc, kk > 0);
+            const uint32_t o = (((kk & 7) >> 2) * kHalf + (kk & 3) * 32) >> 4;
+            const uint32_t ob = (kk < 8 ? oh : ol) + o;
+            if (kk == 0) umma_ss<false>(d0 + 128, vl_lo, dhi, ob, dhi, idesc);
+            else umma_ss<true>(d0 + 128, vl_lo + o, dhi, ob, dhi, idesc);
           }
 #pragma unroll
           for (int kk = 0; kk < 16; ++kk) {
-            const uint32_t o = ((kk & 7) >> 2) * kHalf + (kk & 3) * 32;
-            const uint32_t ob = (kk < 8 ? ohi_addr : olo_addr) + qrow + o;
-            umma_bf16(d0 + 192, smem_desc_sw128(vr + o, 16, 1024), smem_desc_sw128(ob, 16, 1024), idesc, kk > 0);
+            const uint32_t o = (((kk & 7) >> 2) * kHalf + (kk & 3) * 32) >> 4;
+            const uint32_t ob = (kk < 8 ? oh : ol) + o;
+            if (kk == 0) umma_ss<false>(d0 + 192, vr_lo, dhi, ob, dhi, idesc);
+            else umma_ss<true>(d0 + 192, vr_lo + o, dhi, ob, dhi, idesc);
           }
           tc_commit(&misc->tfull[hq]);
         }
@@ -253,19 +265,19 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
     }
   } else {
     // ================================================================ statistics warps
-    const int grp = (warp - 2) >> 2;                      // 0: queries 0-31 of each half, 1: queries 32-63
+    const int grp = (warp - 2) >> 2;                      // queries [kQG grp, kQG grp + kQG) of each half
     const int quarter = warp & 3;                         // TMEM lane quarter this warp may read
     const int lane_p = quarter * 32 + lane;               // pair within the tile
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const int32_t* Cb = a.counts + (size_t)unit * a.n_max;
-    const float2* qc = a.qc2 + (size_t)unit * a.M_pad + qblk * kQB;
     const float4* norms = a.pair_norms + (size_t)unit * a.norm_stride;
+    const float2* qc = a.qc2 + (size_t)unit * a.M_pad + qblk * kQB;   // per query: (-(max + log2 Z), |o|^2)
     // norms and counts of the next tile's pair travel while the current tile is reduced
     float4 nrm_next = make_float4(1.f, 1.f, 1.f, 0.f);
-    float cl_next = 1.f, cr_next = 1.f;
+    int cl_next = 1, cr_next = 1;
     {
       const int p = t_begin * kPairs + lane_p;
-      if (p < P) { nrm_next = __ldg(norms + p); cl_next = (float)Cb[off + 2 * p]; cr_next = (float)Cb[off + 2 * p + 1]; }
+      if (p < P) { nrm_next = ldg_here(norms + p); cl_next = ldg_here(Cb + off + 2 * p); cr_next = ldg_here(Cb + off + 2 * p + 1); }
     }
     for (int li = 0; li < my_tiles; ++li) {
       const int tile = t_begin + li;
@@ -273,10 +285,10 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
       const bool pair_ok = p < P;
       const int jl = off + 2 * p;                         // its left slot
       const float4 nrm = nrm_next;
-      const float cl = cl_next, cr = cr_next;
+      const float cl = (float)cl_next, cr = (float)cr_next;
       if (li + 1 < my_tiles) {
         const int pn = p + kPairs;
-        if (pn < P) { nrm_next = __ldg(norms + pn); cl_next = (float)Cb[off + 2 * pn]; cr_next = (float)Cb[off + 2 * pn + 1]; }
+        if (pn < P) { nrm_next = ldg_here(norms + pn); cl_next = ldg_here(Cb + off + 2 * pn); cr_next = ldg_here(Cb + off + 2 * pn + 1); }
       }
       const float icl = 1.f / cl, icr = 1.f / cr;
       const float r2l = nrm.x, r2r = nrm.y, pc = nrm.z, cosv = nrm.w;
@@ -288,30 +300,28 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
       for (int hq = 0; hq < nh; ++hq) {
         if (!warp_wait(&misc->tfull[hq], li & 1, abort_flag, lane)) { broken = true; break; }
         tc_fence_after();
-        const uint32_t col0 = tmem + lane_addr + hq * 256 + grp * 32;
-        const float4* qc4 = reinterpret_cast<const float4*>(qc + hq * kQH + grp * 32);
-        // four chunks of 8 queries; the loads of chunk c + 1 are in flight while chunk c is reduced
+        const uint32_t col0 = tmem + lane_addr + hq * 256 + grp * kQG;
+        const float4* qc4 = reinterpret_cast<const float4*>(qc + hq * kQH + grp * kQG);
+        // chunks of 8 queries; the loads of chunk c + 1 are in flight while chunk c is reduced
         float buf[2][4][8];
-        float4 cst[2][4];
         auto issue = [&](int c, int b) {
           const uint32_t col = col0 + c * 8;
           tmem_ld8(col, buf[b][0]);
           tmem_ld8(col + 64, buf[b][1]);
           tmem_ld8(col + 128, buf[b][2]);
           tmem_ld8(col + 192, buf[b][3]);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) cst[b][i] = __ldg(qc4 + c * 4 + i);   // (-(max + log2 Z), |o|^2) x 2 queries
         };
         issue(0, 0);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < kQG / 8; ++c) {
           const int b = c & 1;
           tmem_ld_wait();
-          if (c < 3) issue(c + 1, b ^ 1);
+          if (c + 1 < kQG / 8) issue(c + 1, b ^ 1);
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const float ncq = (i & 1) ? cst[b][i >> 1].z : cst[b][i >> 1].x;
-            const float hq2 = (i & 1) ? cst[b][i >> 1].w : cst[b][i >> 1].y;
+            const float4 cq = __ldg(qc4 + c * 4 + (i >> 1));               // two queries' constants (the same address in every lane)
+            const float ncq = (i & 1) ? cq.z : cq.x;
+            const float hq2 = (i & 1) ? cq.w : cq.y;
             const float bl = fast_exp2(fmaf(buf[b][0][i], a.scale_log2, ncq));
             const float br = fast_exp2(fmaf(buf[b][1][i], a.scale_log2, ncq));
             sAl += bl;
@@ -332,20 +342,24 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
       }
       if (broken) break;
 
-      // ---- the second group hands its sums to the first, which owns the outputs
-      if (grp == 1) {
+      // ---- the sums of a pair travel from the last group down to group 0, which owns the outputs: each
+      //      group adds its own to what it receives (a fixed order, so the result is reproducible)
+      float* x = misc->xbuf + lane_p * 5;
+      if (grp == kGroups - 1) {
         // the first group must have read the previous tile's sums
-        if (!warp_wait(&misc->xfree, (li & 1) ^ 1, abort_flag, lane)) break;
-        float* x = misc->xbuf + lane_p * 5;
-        x[0] = sAl; x[1] = sAr; x[2] = sN1l; x[3] = sN1r; x[4] = sN12;
-        warp_arrive(&misc->xready, lane);
+        if (!warp_wait(&misc->xfree[quarter], (li & 1) ^ 1, abort_flag, lane)) break;
       } else {
-        if (!warp_wait(&misc->xready, li & 1, abort_flag, lane)) break;
-        const float* x = misc->xbuf + lane_p * 5;
-        const float Al = cl * (sAl + x[0]), Ar = cr * (sAr + x[1]);
-        const float N1l = cl * (sN1l + x[2]), N1r = cr * (sN1r + x[3]);
-        const float N12 = cl * cr * (sN12 + x[4]);
-        warp_arrive(&misc->xfree, lane);                                   // the buffer may be rewritten
+        if (!warp_wait(&misc->xhand[kGroups - 2 - grp][quarter], li & 1, abort_flag, lane)) break;
+        sAl += x[0]; sAr += x[1]; sN1l += x[2]; sN1r += x[3]; sN12 += x[4];
+      }
+      if (grp != 0) {
+        x[0] = sAl; x[1] = sAr; x[2] = sN1l; x[3] = sN1r; x[4] = sN12;
+        warp_arrive(&misc->xhand[kGroups - 1 - grp][quarter], lane);
+      } else {
+        warp_arrive(&misc->xfree[quarter], lane);                          // the buffer may be rewritten
+        const float Al = cl * sAl, Ar = cr * sAr;
+        const float N1l = cl * sN1l, N1r = cr * sN1r;
+        const float N12 = cl * cr * sN12;
         if (pair_ok) {
           if (a.nqblk == 1) {
             const size_t pi = (size_t)unit * a.pair_stride + p;
