@@ -233,6 +233,8 @@ def main():
                     help="one kvs_merge_layer call per layer instead of one call over all layers")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-groups", type=int, default=4,
+                    help="end-to-end leg: layer groups whose host copies overlap the other groups' kernels")
     args = ap.parse_args()
     w = wl.config(args.config)
     if args.layers:
@@ -311,15 +313,58 @@ def main():
                                          status_dev=status)
             kb.kvs_decode_attn(p, bf(dQn[l]), bf(wK[l]), bf(wV[l]), wC[l], new_len, bf(out[l]), ws)
 
+    # End to end the layers go through in groups: while one group's kernels run, the next groups'
+    # inputs arrive on a copy stream and the previous group's results leave on another (the link
+    # is full duplex), so a step costs about the host->device time of the cache plus one group.
+    n_groups = max(1, min(args.e2e_groups, L)) if fold else 1
+    bounds = [L * g // n_groups for g in range(n_groups + 1)]
+    groups = []
+    for g in range(n_groups):
+        sl = slice(bounds[g], bounds[g + 1])
+        Lg = bounds[g + 1] - bounds[g]
+        if fold:
+            gv = lambda t: t[sl].view(Lg * B, *t.shape[2:])
+            groups.append({"sl": sl, "K": gv(wK), "V": gv(wV), "C": gv(wC), "Q": gv(dQ), "Qn": gv(dQn), "out": gv(out),
+                           "p": kb.make_params(bf(gv(wK)), bf(gv(wV)), Hq, W, sink=w.sink, round_frac=w.round_frac),
+                           "seq_len": list(w.seq_lens) * Lg, "budget": list(w.budgets) * Lg})
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+
     def e2e_step():
-        wK.copy_(hK, non_blocking=True); wV.copy_(hV, non_blocking=True)
-        wC.copy_(hC, non_blocking=True)
-        dQ.copy_(hQ, non_blocking=True); dQn.copy_(hQn, non_blocking=True)
-        step()
-        hRes[0].copy_(wK[:, :, :, :bud_max], non_blocking=True)
-        hRes[1].copy_(wV[:, :, :, :bud_max], non_blocking=True)
-        hResC.copy_(wC[:, :, :, :bud_max], non_blocking=True)
-        hOut.copy_(out, non_blocking=True)
+        main = torch.cuda.current_stream()
+        if not fold:
+            wK.copy_(hK, non_blocking=True); wV.copy_(hV, non_blocking=True)
+            wC.copy_(hC, non_blocking=True)
+            dQ.copy_(hQ, non_blocking=True); dQn.copy_(hQn, non_blocking=True)
+            step()
+            hRes[0].copy_(wK[:, :, :, :bud_max], non_blocking=True)
+            hRes[1].copy_(wV[:, :, :, :bud_max], non_blocking=True)
+            hResC.copy_(wC[:, :, :, :bud_max], non_blocking=True)
+            hOut.copy_(out, non_blocking=True)
+            return
+        s_in.wait_stream(main)                 # the device buffers are free once the step before has left
+        s_in.wait_stream(s_out)
+        arrived = []
+        with torch.cuda.stream(s_in):
+            for g in groups:
+                sl = g["sl"]
+                wK[sl].copy_(hK[sl], non_blocking=True); wV[sl].copy_(hV[sl], non_blocking=True)
+                wC[sl].copy_(hC[sl], non_blocking=True)
+                dQ[sl].copy_(hQ[sl], non_blocking=True); dQn[sl].copy_(hQn[sl], non_blocking=True)
+                ev = torch.cuda.Event(); ev.record(s_in); arrived.append(ev)
+        for g, ev in zip(groups, arrived):
+            sl = g["sl"]
+            main.wait_event(ev)
+            new_len = kb.kvs_merge_layer(g["p"], bf(g["K"]), bf(g["V"]), g["C"], bf(g["Q"]), g["seq_len"],
+                                         g["budget"], ws, status_dev=status)
+            kb.kvs_decode_attn(g["p"], bf(g["Qn"]), bf(g["K"]), bf(g["V"]), g["C"], new_len, bf(g["out"]), ws)
+            done = torch.cuda.Event(); done.record(main)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(done)
+                hRes[0][sl].copy_(wK[sl][:, :, :, :bud_max], non_blocking=True)
+                hRes[1][sl].copy_(wV[sl][:, :, :, :bud_max], non_blocking=True)
+                hResC[sl].copy_(wC[sl][:, :, :, :bud_max], non_blocking=True)
+                hOut[sl].copy_(out[sl], non_blocking=True)
+        main.wait_stream(s_out)                # the step ends when its last result is on the host
 
     def timed(fn, steps, prepare=None):
         total = 0.0
@@ -408,7 +453,8 @@ def main():
         h2d = sum(t.numel() * t.element_size() for t in (hK, hV, hC, hQ, hQn))
         d2h = sum(t.numel() * t.element_size() for t in (hRes, hResC, hOut))
         e2e = {"value": tokens_per_step / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "pipeline": f"{n_groups} layer groups: copies of one group overlap the kernels of another"}
 
     # ---- CPU oracle on a bounded sample (rank 0, N = 1 only)
     cpu = None
