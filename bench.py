@@ -89,8 +89,8 @@ class ClockSampler(threading.Thread):
 # carries over to a full launch).  Each entry names the kernel source it was taken on: once that
 # file changes, the figure is stale and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "hessian_stats": (1.03, "kvs_stats_tc.cu", "000b7e86f391e522"),
-    "attn_partials": (1.01, "kvs_flash_tc.cu", "9633504f2a4cc309"),
+    "hessian_stats": (1.06, "kvs_stats_tc.cu", "6aa90ad0e6355729"),
+    "attn_partials": (1.08, "kvs_flash_tc.cu", "f30ea49ea8ead9d6"),
     "merge_compact": (0.98, "kvs_compact.cu", "c28752d898c08b93"),
 }
 
