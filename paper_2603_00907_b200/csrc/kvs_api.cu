@@ -170,28 +170,28 @@ struct WsLayout {
   size_t sync_bytes;
 };
 
-// Number of key/pair ranges each (query block, KV head, sequence) item is cut into, so that the
-// CTAs (one per SM, equal length) fill whole waves of the 148 SMs.  With fewer items than SMs
-// the items are cut until the SMs are covered; with more, the cut that minimises
-// ceil(items * k / 148) / k (the makespan in item lengths) is taken, e.g. 512 items: k = 2 gives
-// 7 half-length waves instead of 4 full ones.
+// Number of key/pair ranges each (query block, KV head, sequence) item is cut into.  The CTAs run
+// one per SM in waves of 148; a CTA costs its tiles plus about two tile times of set-up and
+// write-back.  The cut k that minimises  waves(items * k) * (ceil(tiles / k) + 2)  is taken (the
+// smaller k when two are within 1 %): 512 items of 256 tiles: k = 2 (7 half-length waves instead
+// of 4 full ones); 64 items of 1024 tiles: k = 9 (576 CTAs in 4 waves of 114 tiles instead of 128
+// CTAs of 512 tiles on 148 SMs); 8 items of 16 tiles: k = 16.
 constexpr int kNumSMs = 148;
-constexpr int kMaxTcSplits = 8;     // per item; the attention partials are sized for it
+constexpr int kMaxTcSplits = 16;    // per item (more only while items * k <= 148); the attention partials are sized for it
 
 int balanced_splits(int items, int ntiles, int* tiles_per_split) {
+  if (items < 1) items = 1;
+  if (ntiles < 1) ntiles = 1;
+  int kmax = kNumSMs / items > kMaxTcSplits ? kNumSMs / items : kMaxTcSplits;
+  if (kmax > ntiles) kmax = ntiles;
   int best = 1;
-  if (items < kNumSMs) {
-    best = kNumSMs / items;
-  } else {
-    double best_cost = 1e30;
-    for (int k = 1; k <= kMaxTcSplits; ++k) {
-      if (k > 1 && ntiles / k < 4) break;                   // keep ranges long enough to amortise the set-up
-      const double cost = (double)((items * k + kNumSMs - 1) / kNumSMs) / k;
-      if (cost < best_cost - 1e-9) { best_cost = cost; best = k; }
-    }
+  double best_cost = 1e30;
+  for (int k = 1; k <= kmax; ++k) {
+    const int tps = (ntiles + k - 1) / k;
+    const int ctas = items * ((ntiles + tps - 1) / tps);      // ranges that are not empty
+    const double cost = (double)((ctas + kNumSMs - 1) / kNumSMs) * (tps + 2);
+    if (cost < best_cost * 0.99) { best_cost = cost; best = k; }
   }
-  if (best > ntiles) best = ntiles;
-  if (best < 1) best = 1;
   int tps = (ntiles + best - 1) / best;
   if (tps < 1) tps = 1;
   *tiles_per_split = tps;
