@@ -33,15 +33,25 @@ select_pairs_kernel(const SelectArgs a, const RoundTable tab) {
       const int shift = 24 - 8 * pass;
       if (tid < 256) hist[tid] = 0;
       __syncthreads();
-      for (int p0 = 0; p0 < P; p0 += 1024) {
-        const int p = p0 + tid;
-        const uint32_t v = (p < P) ? key[p] : 0u;
-        const bool in = (p < P) && (v & pmask) == prefix;
-        const uint32_t d = (v >> shift) & 255u;
-        const uint32_t act = __ballot_sync(0xffffffffu, in);
-        if (in) {
-          const uint32_t same = __match_any_sync(act, d);
-          if (lane == (__ffs(same) - 1)) atomicAdd(&hist[d], (uint32_t)__popc(same));
+      // four loads in flight per thread: the sweep is a chain of L2 latencies otherwise
+      for (int p0 = 0; p0 < P; p0 += 4 * 1024) {
+        uint32_t v4[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int p = p0 + u * 1024 + tid;
+          v4[u] = (p < P) ? __ldg(key + p) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int p = p0 + u * 1024 + tid;
+          const uint32_t v = v4[u];
+          const bool in = (p < P) && (v & pmask) == prefix;
+          const uint32_t d = (v >> shift) & 255u;
+          const uint32_t act = __ballot_sync(0xffffffffu, in);
+          if (in) {
+            const uint32_t same = __match_any_sync(act, d);
+            if (lane == (__ffs(same) - 1)) atomicAdd(&hist[d], (uint32_t)__popc(same));
+          }
         }
       }
       __syncthreads();
@@ -80,14 +90,18 @@ select_pairs_kernel(const SelectArgs a, const RoundTable tab) {
   const int ntiles = (n - tab.off + KVS_CTILE - 1) / KVS_CTILE;
   int32_t* tp = a.tile_prefix + (size_t)unit * a.tile_stride;
   const int sweep = ((ntiles * 32 + 1023) / 1024) * 1024;
+  // (the value of the chunk after this one is requested before this chunk's barriers)
+  uint32_t v_next = 0;
+  if (tid < P) v_next = a.from_mask ? (uint32_t)mask[tid] : __ldg(key + tid);
   for (int p0 = 0; p0 < sweep; p0 += 1024) {
     const int p = p0 + tid;
     bool tie = false, less = false, sel = false;
+    const uint32_t v = v_next;
+    if (p + 1024 < P) v_next = a.from_mask ? (uint32_t)mask[p + 1024] : __ldg(key + p + 1024);
     if (p < P) {
       if (a.from_mask) {
-        sel = mask[p] != 0;
+        sel = v != 0;
       } else {
-        const uint32_t v = key[p];
         less = v < prefix;
         tie = v == prefix;
       }
