@@ -505,10 +505,14 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       if (alive) alive = warp_wait(&misc->sfull[b], ph, abort_flag, lane);
       if (alive) {
         tc_fence_after();
-        load32(scol, jA, x);
-        const float mA = max32(x);
-        load32(scol + 32, jB, x);                          // these stay in registers: they are exponentiated first
-        atomicMax(&rmax[row], f2ord(fmaxf(mA, max32(x))));
+        // (loops that are not unrolled keep the code of the four roles within the instruction cache)
+        float mx = -INFINITY;
+#pragma unroll 1
+        for (int sub = 0; sub < 2; ++sub) {                // the second 32 stay in registers: they are exponentiated first
+          load32(scol + 32 * sub, jA + 32 * sub, x);
+          mx = fmaxf(mx, max32(x));
+        }
+        atomicMax(&rmax[row], f2ord(mx));
       }
       // the one barrier of the tile: the row maxima and the staged counts of the team are complete
       team_barrier(team);
@@ -569,13 +573,14 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         fence_proxy_async();                               // the tensor core reads these rows
       }
       // the last 32 slots first (their logits are still in registers), then the first 32 again from TMEM
-      l += emit32(scol + 32, x, cnt + ch * 64 + 32);
-      tc_fence_before();
-      warp_arrive(&misc->pready[b][0], lane);
-      load32(scol, jA, x);
-      l += emit32(scol, x, cnt + ch * 64);
-      tc_fence_before();
-      warp_arrive(&misc->pready[b][1], lane);
+#pragma unroll 1
+      for (int hf = 0; hf < 2; ++hf) {
+        const int o32 = hf == 0 ? 32 : 0;
+        if (hf == 1) load32(scol, jA, x);
+        l += emit32(scol + o32, x, cnt + ch * 64 + o32);
+        tc_fence_before();
+        warp_arrive(&misc->pready[b][hf], lane);
+      }
     }
     // ---- the partial of this key range: every thread brings its part of l to the final stabiliser,
     //      the four parts of a row are added, and each thread writes 32 channels of the row of O
