@@ -158,6 +158,49 @@ def test_attention_partials_with_late_spikes(kb):
         assert np.max(np.abs(lse[0, h].cpu().numpy() - lse_ref)) < 2e-4
 
 
+def test_attention_partials_with_spikes_in_consecutive_tiles(kb):
+    """Keys aligned with one query, each stronger than the one before, in six consecutive
+    128-slot tiles (and in the last tile before the window): the row's stabiliser moves in tile
+    after tile, so each of the kernel's two softmax teams has to pick up the value the other one
+    left, rescale the shared output and carry its own part of the row sum along."""
+    import torch
+    w = _small(seed=12, batch=1, n_q_heads=32, n_kv_heads=8, window=16, seq_lens=(4000,), budgets=(1500,))
+    data = wl.make_layer(w)
+    K, q = data["K"], data["q_win"]
+    qf = wl.bf16_bits_to_f32(q)
+    spikes = [(128 * t + 5 + t, 0.9 + 0.65 * i) for i, t in enumerate(range(8, 14))] + [(3900, 5.2)]
+    for h in range(w.n_kv_heads):
+        row = 5 + 3 * h                               # a different query row per head
+        g, i = divmod(row, w.window)
+        for j, amp in spikes:
+            K[0, h, j] = wl.f32_to_bf16_bits(amp * qf[0, h * w.group + g, i])
+    dev, p, ws = _setup(kb, w, data)
+    B, Hkv, Nmax, M = 1, w.n_kv_heads, w.n_max, w.group * w.window
+    f32 = dict(dtype=torch.float32, device="cuda")
+    A = torch.zeros((B, Hkv, Nmax), **f32)
+    o_win, lse = torch.zeros((B, Hkv, M, 128), **f32), torch.zeros((B, Hkv, M), **f32)
+    kb.kvs_window_stats(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], [4000], [1500], ws, A=A,
+                        o_win=o_win, lse_win=lse)
+    torch.cuda.synchronize()
+    for h in range(Hkv):
+        Kf, Vf = oc.bf16_to_f64(K[0, h]), oc.bf16_to_f64(data["V"][0, h])
+        Qf = oc.bf16_to_f64(q[0, h * w.group:(h + 1) * w.group])
+        alpha, o, _ = oc.window_probabilities(Kf, Vf, np.ones(4000), Qf, w.window, 1 / math.sqrt(128), True)
+        s = (Qf.reshape(M, 128) @ Kf.T) / math.sqrt(128)
+        row = 5 + 3 * h
+        growth = np.diff([s[row, j] for j, _ in spikes]) * math.log2(math.e)
+        assert growth.min() > 8.0                     # every spike outgrows the stabiliser's slack of 2^8
+        ok, ratio, plain = tl.stat_close(o_win[0, h].cpu().numpy(), o, rtol=tl.O_RTOL)
+        assert ok, (h, ratio, plain)
+        off, P, _ = oc.round_plan(4000, 1500, w.sink, w.window, 0.5, 0)
+        ok, ratio, plain = tl.stat_close(A[0, h, off:off + 2 * P].cpu().numpy(), alpha.sum(0)[off:off + 2 * P])
+        assert ok, (h, ratio, plain)
+        i = np.tile(np.arange(w.window), w.group)
+        s = np.where(np.arange(4000)[None, :] > (4000 - w.window + i)[:, None], -np.inf, s)
+        lse_ref = np.log(np.exp(s - s.max(1, keepdims=True)).sum(1)) + s.max(1)
+        assert np.max(np.abs(lse[0, h].cpu().numpy() - lse_ref)) < 2e-4
+
+
 def test_window_stats_modes(kb):
     w = _small(seed=2, seq_lens=(260, 131), budgets=(90, 60))
     data = wl.make_layer(w)
