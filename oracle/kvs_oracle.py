@@ -23,7 +23,9 @@ What is computed (paper passages in brackets):
   rounds until the budget is met; the first `sink` tokens are never merged
   [Section 5.1, implementation details];
 * attention over the merged cache for new queries (numerator uses value sums,
-  denominator weights each slot by its count).
+  denominator weights each slot by its count);
+* the streaming step: a chunk of fresh tokens is appended and the pass brings the cache
+  back to the budget [Section 3.1; Section 5.1: budget 2048, chunk 512].
 
 Readings where the paper is silent are fixed here and listed in the design notes:
 aligned candidate pairs with alternating parity, pair score = attention mass times
@@ -346,6 +348,21 @@ def merge_unit(K_bits: np.ndarray, V_bits: np.ndarray, c: np.ndarray, Q_bits: np
         r += 1
         done += 1
     return K_bits, V_bits, c.astype(np.int32)
+
+
+def append_and_merge(K_bits: np.ndarray, V_bits: np.ndarray, c: np.ndarray,
+                     chunk_K_bits: np.ndarray, chunk_V_bits: np.ndarray, Q_bits: np.ndarray,
+                     budget: int, **merge_kwargs) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """One streaming step on one (sequence, KV head)  [Section 3.1: the cache is compressed each
+    time a chunk of new tokens has arrived; Section 5.1: budget 2048, chunk 512].
+
+    The chunk's tokens are appended after the slots in use as fresh slots (count 1, value sum =
+    value), then the merge pass brings the cache back to `budget` with `Q_bits`, the queries of
+    the chunk's last W positions, as observation window.  Keyword arguments as `merge_unit`."""
+    K_all = np.concatenate([K_bits, chunk_K_bits], axis=0)
+    V_all = np.concatenate([V_bits, chunk_V_bits], axis=0)
+    c_all = np.concatenate([np.asarray(c).astype(np.int64), np.ones(chunk_K_bits.shape[0], dtype=np.int64)])
+    return merge_unit(K_all, V_all, c_all, Q_bits, budget, **merge_kwargs)
 
 
 def decode_attention(q_bits: np.ndarray, K_bits: np.ndarray, V_bits: np.ndarray, c: np.ndarray,

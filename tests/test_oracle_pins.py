@@ -460,3 +460,43 @@ def test_n1_is_a_norm_when_attention_is_peaked():
     _, N1 = oc.slot_stats(alpha, o, vbar)
     c11, _, _ = oc.c_vectors(alpha[0, 1], alpha[0, 1], V[1], V[1], o[0])
     assert N1[1] > 0 and abs(N1[1] - np.linalg.norm(c11)) < 1e-14
+
+
+def test_streaming_steps_keep_the_token_and_value_books():
+    """Three streaming steps (append a chunk, merge back to the budget): after every step the
+    cache holds exactly `budget` slots, the counts add up to all tokens seen, the sink slots
+    and the chunk's last `window` tokens are bit-identical to what was appended, the value sums
+    add up to the sum of all token values (each merge adds two bf16 numbers and rounds once),
+    and a step whose chunk fits the budget leaves the cache as the plain concatenation."""
+    rng = np.random.default_rng(5)
+    d, W, G, sink, budget, chunk = 16, 4, 2, 4, 40, 12
+    bits = lambda x: oc.f64_to_bf16(np.asarray(x, dtype=np.float64))
+    K = bits(rng.standard_normal((30, d))); V = bits(rng.standard_normal((30, d)))
+    c = np.ones(30, dtype=np.int64)
+    total_v = oc.bf16_to_f64(V).sum(0)
+    seen = 30
+    for step in range(3):
+        cK = bits(rng.standard_normal((chunk, d))); cV = bits(rng.standard_normal((chunk, d)))
+        Q = bits(rng.standard_normal((G, W, d)))
+        n_before = K.shape[0]
+        K2, V2, c2 = oc.append_and_merge(K, V, c, cK, cV, Q, budget, window=W, sink=sink)
+        seen += chunk
+        total_v = total_v + oc.bf16_to_f64(cV).sum(0)
+        assert K2.shape[0] == min(budget, n_before + chunk) and int(c2.sum()) == seen
+        if n_before + chunk <= budget:                     # nothing to merge yet: a plain append
+            assert np.array_equal(K2, np.concatenate([K, cK])) and np.array_equal(V2, np.concatenate([V, cV]))
+        assert np.array_equal(K2[:sink], K[:sink]) and np.array_equal(V2[:sink], V[:sink])
+        assert np.array_equal(K2[-W:], cK[-W:]) and np.array_equal(V2[-W:], cV[-W:])
+        assert np.all(c2[-W:] == 1)
+        # value sums: every merged slot rounds a sum of bf16 numbers once per merge
+        err = np.abs(oc.bf16_to_f64(V2).sum(0) - total_v)
+        assert np.all(err <= 2.0 ** -8 * np.abs(oc.bf16_to_f64(V2)).sum(0) + 1e-12)
+        K, V, c = K2, V2, c2.astype(np.int64)
+    assert K.shape[0] == budget and c.max() > 1
+
+
+def test_streaming_step_in_the_paper_setting_is_one_round():
+    """Budget 2048 + chunk 512 with 32 sink tokens [Section 5.1]: the schedule needs one round,
+    which merges exactly 512 of the candidate pairs."""
+    plan = oc.full_plan(2048 + 512, 2048, 32, 64, 0.5)
+    assert len(plan) == 1 and plan[0][3] == 512 and plan[0][2] >= 2 * 512
