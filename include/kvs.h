@@ -115,6 +115,27 @@ kvs_status_t kvs_merge_layer(const kvs_params_t* params, void* K, void* V, int32
                              size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
 
 /*
+ * One streaming step of a decoder layer, in place  [Section 3.1: the cache is compressed each
+ * time a chunk of new tokens has arrived; Section 5.1 (implementation details): budget 2048,
+ * chunk 512].  The chunk's tokens are appended after the slots in use as fresh slots (count 1,
+ * value sum = value), then the merge pass of kvs_merge_layer brings every sequence back to its
+ * budget with q_win, the queries of the chunk's last W positions, as observation window.
+ *   K, V, counts, q_win, budget, n_max, new_len, workspace: as kvs_merge_layer
+ *   chunk_k, chunk_v  DEVICE bf16 [B,Hkv,chunk_len,128] contiguous, 16-byte aligned; read only
+ *   chunk_len         tokens appended to every sequence (>= 0)
+ *   cur_len           HOST int32[B]: slots in use before the call; cur_len[b] + chunk_len <= n_max
+ *   new_len           HOST int32[B] out: min(cur_len[b] + chunk_len, budget[b])
+ * The workspace must cover kvs_workspace_size(params, max(cur_len) + chunk_len, 0).
+ * Errors that the host can detect (ranges, an unreachable budget) are returned before anything
+ * is enqueued, the append included.  Asynchronous on the stream; the caller owns all buffers.
+ */
+kvs_status_t kvs_append_and_merge(const kvs_params_t* params, void* K, void* V, int32_t* counts,
+                                  const void* chunk_k, const void* chunk_v, int32_t chunk_len,
+                                  const void* q_win, const int32_t* cur_len, const int32_t* budget,
+                                  int32_t n_max, int32_t* new_len, void* workspace,
+                                  size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
+
+/*
  * One round of merge + stable in-place compaction with a caller-supplied decision
  * [Eq. kstar_final for the key, v* = v_m + v_{m+1} for the value sum].
  *   merge_mask DEVICE uint8 [B,Hkv,Nmax/2]: 1 where candidate pair p is merged; pair p of

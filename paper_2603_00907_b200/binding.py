@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "KVS_OK", 1: "KVS_ERR_INVALID_ARG", 2: "KVS_ERR_UNSUPPORTED",
 EXPORTS = ["kvs_version", "kvs_last_error_string", "kvs_launch_count", "kvs_round_plan",
            "kvs_workspace_size", "kvs_merge_layer", "kvs_compact", "kvs_decode_attn",
            "kvs_window_stats", "kvs_profile_begin", "kvs_profile_end", "kvs_profile_kind_name",
-           "kvs_compact_static", "kvs_static_scratch_bytes"]
+           "kvs_compact_static", "kvs_static_scratch_bytes", "kvs_append_and_merge"]
 
 
 class KvsError(RuntimeError):
@@ -136,6 +136,22 @@ def kvs_merge_layer(params: kvs_params_t, K, V, counts, q_win, seq_len: Sequence
                                  new_len, _ptr(workspace),
                                  ctypes.c_size_t(workspace.numel() * workspace.element_size()),
                                  _ptr(status_dev), _stream()))
+    return list(new_len)
+
+
+def kvs_append_and_merge(params: kvs_params_t, K, V, counts, chunk_k, chunk_v, q_win,
+                         cur_len: Sequence[int], budget: Sequence[int], workspace,
+                         status_dev=None) -> List[int]:
+    """One streaming step in place: append the chunk [B,Hkv,chunk_len,128] after the slots in use,
+    then merge back to the budget.  Returns new_len per sequence."""
+    B = params.batch
+    new_len = (ctypes.c_int32 * B)()
+    _check(lib().kvs_append_and_merge(ctypes.byref(params), _ptr(K), _ptr(V), _ptr(counts), _ptr(chunk_k),
+                                      _ptr(chunk_v), ctypes.c_int32(chunk_k.shape[2]), _ptr(q_win),
+                                      _i32(cur_len), _i32(budget), ctypes.c_int32(counts.shape[-1]),
+                                      new_len, _ptr(workspace),
+                                      ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+                                      _ptr(status_dev), _stream()))
     return list(new_len)
 
 

@@ -604,10 +604,17 @@ kvs_status_t kvs_workspace_size(const kvs_params_t* p, int32_t max_seq_len, int3
   return KVS_OK;
 }
 
-kvs_status_t kvs_merge_layer(const kvs_params_t* p, void* K, void* V, int32_t* counts,
-                             const void* q_win, const int32_t* seq_len, const int32_t* budget,
-                             int32_t n_max, int32_t* new_len, void* workspace,
-                             size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+namespace {
+
+// The merge pass; with `chunk_k` the rows of a chunk are appended first (seq_len then counts them
+// already, `cur_len` holds the slots in use before).  Everything the host can detect is detected
+// before the first launch.
+kvs_status_t merge_layer_impl(const kvs_params_t* p, void* K, void* V, int32_t* counts,
+                              const void* q_win, const int32_t* seq_len, const int32_t* budget,
+                              int32_t n_max, int32_t* new_len, void* workspace,
+                              size_t workspace_bytes, int32_t* status_dev, void* cuda_stream,
+                              const void* chunk_k, const void* chunk_v, int32_t chunk_len,
+                              const int32_t* cur_len) {
   Common c;
   kvs_status_t s = check_common(p, K, V, counts, seq_len, n_max, workspace, workspace_bytes, 0, &c, cuda_stream);
   if (s != KVS_OK) return s;
@@ -632,15 +639,30 @@ kvs_status_t kvs_merge_layer(const kvs_params_t* p, void* K, void* V, int32_t* c
   }
   if (rounds > KVS_MAX_ROUNDS) return fail(KVS_ERR_UNSUPPORTED, "more than %d rounds", KVS_MAX_ROUNDS);
   for (int b = 0; b < B; ++b) new_len[b] = seq_len[b] < budget[b] ? seq_len[b] : budget[b];
-  if (rounds == 0) return KVS_OK;
-
   c.status_dev = status_dev;
-  s = make_call_tmaps(&c, K, V, q_win, n_max);
-  if (s != KVS_OK) return s;
+  if (rounds > 0) {
+    s = make_call_tmaps(&c, K, V, q_win, n_max);
+    if (s != KVS_OK) return s;
+  }
+  const CacheView view = make_view(p, K, V, counts, n_max);
+  if (chunk_k && chunk_len > 0) {
+    AppendArgs aa;
+    aa.c = view;
+    aa.chunk_k = static_cast<const __nv_bfloat16*>(chunk_k);
+    aa.chunk_v = static_cast<const __nv_bfloat16*>(chunk_v);
+    aa.chunk_len = chunk_len;
+    for (int b0 = 0; b0 < B; b0 += KVS_SEQ_CHUNK) {
+      RoundTable tab;
+      tab.nseq = 0;
+      tab.off = 0;
+      for (int b = b0; b < B && tab.nseq < KVS_SEQ_CHUNK; ++b) tab.s[tab.nseq++] = {cur_len[b], 0, 0, b};
+      CUDA_TRY(launch(KVS_K_MISC, c.st, [&] { return kvs_launch_append(aa, tab, c.st); }));
+    }
+  }
+  if (rounds == 0) return KVS_OK;
   CUDA_TRY(cudaMemsetAsync(c.ws + c.L.sync, 0, c.L.sync_bytes, c.st));
   uint32_t* tickets = reinterpret_cast<uint32_t*>(c.ws + c.L.sync);
   uint32_t* flags = tickets + (size_t)KVS_MAX_ROUNDS * c.L.U;
-  const CacheView view = make_view(p, K, V, counts, n_max);
 
   for (int i = 0; i < rounds; ++i) {
     const int r = p->first_round + i;
@@ -676,6 +698,37 @@ kvs_status_t kvs_merge_layer(const kvs_params_t* p, void* K, void* V, int32_t* c
     }
   }
   return KVS_OK;
+}
+
+}  // namespace
+
+kvs_status_t kvs_merge_layer(const kvs_params_t* p, void* K, void* V, int32_t* counts,
+                             const void* q_win, const int32_t* seq_len, const int32_t* budget,
+                             int32_t n_max, int32_t* new_len, void* workspace,
+                             size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+  return merge_layer_impl(p, K, V, counts, q_win, seq_len, budget, n_max, new_len, workspace, workspace_bytes,
+                          status_dev, cuda_stream, nullptr, nullptr, 0, nullptr);
+}
+
+kvs_status_t kvs_append_and_merge(const kvs_params_t* p, void* K, void* V, int32_t* counts,
+                                  const void* chunk_k, const void* chunk_v, int32_t chunk_len,
+                                  const void* q_win, const int32_t* cur_len, const int32_t* budget,
+                                  int32_t n_max, int32_t* new_len, void* workspace,
+                                  size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+  kvs_status_t s = check_params(p);
+  if (s != KVS_OK) return s;
+  if (!cur_len) return fail(KVS_ERR_INVALID_ARG, "NULL pointer argument");
+  if (chunk_len < 0) return fail(KVS_ERR_INVALID_ARG, "chunk_len must be >= 0");
+  if (chunk_len > 0 && (!chunk_k || !chunk_v)) return fail(KVS_ERR_INVALID_ARG, "NULL pointer argument");
+  if (!aligned16(chunk_k) || !aligned16(chunk_v)) return fail(KVS_ERR_INVALID_ARG, "the chunk must be 16-byte aligned");
+  std::vector<int32_t> seq_len(p->batch);
+  for (int b = 0; b < p->batch; ++b) {
+    if (cur_len[b] < 0 || cur_len[b] > n_max - chunk_len)
+      return fail(KVS_ERR_INVALID_ARG, "cur_len[%d] + chunk_len exceeds n_max", b);
+    seq_len[b] = cur_len[b] + chunk_len;
+  }
+  return merge_layer_impl(p, K, V, counts, q_win, seq_len.data(), budget, n_max, new_len, workspace,
+                          workspace_bytes, status_dev, cuda_stream, chunk_k, chunk_v, chunk_len, cur_len);
 }
 
 kvs_status_t kvs_compact(const kvs_params_t* p, void* K, void* V, int32_t* counts,

@@ -164,6 +164,14 @@ cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const
                                 const CUtensorMap& tmOlo, cudaStream_t st);
 cudaError_t kvs_launch_flash_tc(const FlashTcArgs& a, const RoundTable& t, const CUtensorMap& tmK,
                                 const CUtensorMap& tmV, const CUtensorMap& tmQ, cudaStream_t st);
+// Chunk of fresh tokens appended after the slots in use (table entry n = slots in use).
+struct AppendArgs {
+  CacheView c;
+  const __nv_bfloat16* chunk_k;   // [B, Hkv, chunk_len, 128] contiguous
+  const __nv_bfloat16* chunk_v;
+  int32_t chunk_len;
+};
+cudaError_t kvs_launch_append(const AppendArgs& a, const RoundTable& t, cudaStream_t st);
 cudaError_t kvs_launch_select(const SelectArgs& a, const RoundTable& t, cudaStream_t st);
 cudaError_t kvs_launch_compact(const CompactArgs& a, const RoundTable& t, cudaStream_t st);
 

@@ -406,6 +406,81 @@ def test_merge_layer_stagewise_and_end_to_end(kb):
     print(f"band flips followed: {flips}")
 
 
+def test_streaming_steps_match_the_oracle(kb):
+    """Three streaming steps (a chunk is appended, the pass merges back to the budget) through
+    kvs_append_and_merge: each step must equal, bit for bit, a plain device copy of the chunk
+    followed by kvs_merge_layer, and the oracle that follows the GPU's near-cutoff choices;
+    the first step's chunk still fits the budget of the second sequence (a plain append)."""
+    import torch
+    # (generated 240 and 140 slots long so that there is room behind the 200 and 100 slots in use)
+    w = _small(seed=21, batch=2, n_q_heads=8, n_kv_heads=2, window=8, seq_lens=(240, 140), budgets=(200, 140))
+    B, Hkv, G, W, chunk = w.batch, w.n_kv_heads, w.group, w.window, 36
+    base = wl.make_layer(w)
+    Nmax = base["K"].shape[2]
+    cur0 = [200, 100]
+    assert Nmax >= max(cur0) + chunk
+    rng = np.random.default_rng(77)
+    bits = lambda shape: wl.f32_to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
+    dev, p, ws = _setup(kb, w, base)        # streamed through the new entry point
+    dev2, _, ws2 = _setup(kb, w, base)      # the same steps from existing calls, recording masks
+    cur = list(cur0)
+    ora = {(b, h): (base["K"][b, h, :cur[b]].copy(), base["V"][b, h, :cur[b]].copy(),
+                    base["counts"][b, h, :cur[b]].astype(np.int64)) for b in range(B) for h in range(Hkv)}
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    flips = 0
+    for step in range(3):
+        cK, cV = bits((B, Hkv, chunk, 128)), bits((B, Hkv, chunk, 128))
+        qw = bits((B, w.n_q_heads, W, 128))
+        dcK, dcV, dq = tl.to_dev_bf16(cK), tl.to_dev_bf16(cV), tl.to_dev_bf16(qw)
+        new_len = kb.kvs_append_and_merge(p, dev["K"], dev["V"], dev["counts"], dcK, dcV, dq, cur,
+                                          list(w.budgets), ws, status_dev=status)
+        # the same step from a device copy + the single-round calls
+        n_list = [c + chunk for c in cur]
+        for b in range(B):
+            dev2["K"][b, :, cur[b]:cur[b] + chunk] = dcK[b]
+            dev2["V"][b, :, cur[b]:cur[b] + chunk] = dcV[b]
+            dev2["counts"][b, :, cur[b]:cur[b] + chunk] = 1
+        plans = [oc.full_plan(n, bud, w.sink, W, w.round_frac) if n > bud else [] for n, bud in zip(n_list, w.budgets)]
+        gpu_masks = []
+        for r in range(max(len(pl) for pl in plans)):
+            pr = kb.make_params(dev2["K"], dev2["V"], w.n_q_heads, W, sink=w.sink, round_frac=w.round_frac,
+                                first_round=r)
+            mask = torch.zeros((B, Hkv, Nmax // 2), dtype=torch.uint8, device="cuda")
+            kb.kvs_window_stats(pr, dev2["K"], dev2["V"], dev2["counts"], dq, n_list, list(w.budgets), ws2, mask=mask)
+            step_budget = [plans[b][r][0] - plans[b][r][3] if r < len(plans[b]) else min(n_list[b], w.budgets[b])
+                           for b in range(B)]
+            n_list = kb.kvs_merge_layer(pr, dev2["K"], dev2["V"], dev2["counts"], dq, n_list, step_budget, ws2)
+            gpu_masks.append(mask.cpu().numpy())
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        assert new_len == n_list == [min(c + chunk, bud) for c, bud in zip(cur, w.budgets)]
+        Kg, Vg, Cg = tl.bits_of(dev["K"]), tl.bits_of(dev["V"]), dev["counts"].cpu().numpy()
+        for b in range(B):
+            m = new_len[b]
+            assert np.array_equal(Kg[b, :, :m], tl.bits_of(dev2["K"])[b, :, :m])
+            assert np.array_equal(Vg[b, :, :m], tl.bits_of(dev2["V"])[b, :, :m])
+            assert np.array_equal(Cg[b, :, :m], dev2["counts"].cpu().numpy()[b, :, :m])
+            for h in range(Hkv):
+                Ko, Vo, Co = ora[(b, h)]
+                forced = [gpu_masks[r][b, h, :plans[b][r][2]] for r in range(len(plans[b]))]
+                trace = []
+                Ko, Vo, Co = oc.append_and_merge(Ko, Vo, Co, cK[b, h], cV[b, h], qw[b, h * G:(h + 1) * G],
+                                                 w.budgets[b], forced_masks=forced, trace=trace,
+                                                 **_oracle_kwargs(w))
+                for r, st in enumerate(trace):
+                    ok, nm, nout = tl.mask_band_ok(forced[r], st["mask"], st["score"], st["R"])
+                    assert ok, f"step {step} unit {(b, h)} round {r}: {nm} mismatches, {nout} outside the band"
+                    flips += nm
+                assert np.array_equal(Cg[b, h, :m], Co) and Co.sum() == cur0[b] + (step + 1) * chunk
+                okk, mxk, _, _ = tl.bf16_close(Kg[b, h, :m], Ko)
+                okv, mxv, _, _ = tl.bf16_close(Vg[b, h, :m], Vo)
+                assert okk and okv, (step, b, h, mxk, mxv)
+                # the next step starts from the GPU's state (so that rounding flips do not add up)
+                ora[(b, h)] = (Kg[b, h, :m].copy(), Vg[b, h, :m].copy(), Cg[b, h, :m].astype(np.int64))
+        cur = new_len
+    print(f"band flips followed: {flips}")
+
+
 def test_decode_matches_oracle_and_is_lossless_on_identical_keys(kb):
     import torch
     w = _small(seed=5, seq_lens=(400, 257), budgets=(90, 60), n_decode=5)

@@ -97,3 +97,14 @@ def test_null_pointers_are_rejected_before_any_cuda_call(lib):
     rc = lib.kvs_decode_attn(ctypes.byref(p), None, 0, None, None, None, one, 4096, None, None, None,
                              ctypes.c_size_t(0), None, None)
     assert rc == 1
+
+
+def test_append_and_merge_rejects_bad_arguments_before_any_cuda_call(lib):
+    p = _params()
+    one, zero = (ctypes.c_int32 * 1)(4096), (ctypes.c_int32 * 1)(0)
+    args = lambda chunk_len, cur: (ctypes.byref(p), None, None, None, None, None, chunk_len, None, cur, one, 4096,
+                                   one, None, ctypes.c_size_t(0), None, None)
+    assert lib.kvs_append_and_merge(*args(-1, zero)) == 1          # negative chunk length
+    assert lib.kvs_append_and_merge(*args(16, one)) == 1           # NULL chunk / no room behind 4096 slots
+    assert lib.kvs_append_and_merge(*args(0, None)) == 1           # NULL cur_len
+    assert b"" != lib.kvs_last_error_string()
