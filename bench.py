@@ -221,6 +221,66 @@ def workload_config(w, args):
             "parallelism": f"dp{args.gpus} over sequences, no collective"}
 
 
+def run_stream(args):
+    """Streaming step in the paper's setting (Section 5.1: budget 2048, chunk 512, sink 32): every
+    step appends 512 fresh tokens per sequence to a cache of 2048 slots and merges back to 2048,
+    for all layers of configs[1] in one kvs_append_and_merge call.  Synthetic inputs of the same
+    recipe as the other workloads; CUDA events, cache restored before every step."""
+    import torch
+    from paper_2603_00907_b200 import binding as kb, build as kbuild
+    kbuild.build()
+    kb.lib()
+    budget, chunk = 2048, 512
+    w = wl.config(1).scaled(seq_lens=(budget + chunk,), budgets=(budget,))
+    if args.layers:
+        w = w.scaled(layers=args.layers)
+    L, B, Hq, Hkv, W = w.layers, w.batch, w.n_q_heads, w.n_kv_heads, w.window
+    layers = wl.make_layers_parallel(w, range(L))
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    stack = lambda k, dt: torch.from_numpy(np.stack([d[k] for d in layers]).view(dt)).to(dev)
+    mK, mV = stack("K", np.int16), stack("V", np.int16)                  # [L, B, Hkv, 2560, 128]
+    mC = torch.from_numpy(np.stack([d["counts"] for d in layers])).to(dev)
+    q = stack("q_win", np.int16)
+    fold = lambda t: t.view(L * B, *t.shape[2:])
+    bf = lambda t: t.view(torch.bfloat16)
+    cK = fold(mK)[:, :, budget:].contiguous()
+    cV = fold(mV)[:, :, budget:].contiguous()
+    wK, wV, wC = torch.empty_like(mK), torch.empty_like(mV), torch.empty_like(mC)
+    p = kb.make_params(bf(fold(wK)), bf(fold(wV)), Hq, W, sink=w.sink, round_frac=w.round_frac)
+    ws = torch.empty(kb.kvs_workspace_size(p, budget + chunk, 0), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    cur, bud = [budget] * (L * B), [budget] * (L * B)
+
+    def restore():
+        wK.copy_(mK); wV.copy_(mV); wC.copy_(mC)
+
+    def step():
+        return kb.kvs_append_and_merge(p, bf(fold(wK)), bf(fold(wV)), fold(wC), bf(cK), bf(cV), bf(fold(q)),
+                                       cur, bud, ws, status_dev=status)
+
+    for _ in range(max(3, args.warmup)):
+        restore(); new_len = step()
+    torch.cuda.synchronize()
+    l0 = kb.lib().kvs_launch_count()
+    total = 0.0
+    for _ in range(args.steps):
+        restore()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); step(); b.record(); b.synchronize()
+        total += a.elapsed_time(b)
+    launches = kb.lib().kvs_launch_count() - l0
+    assert status.item() == 0 and new_len == bud
+    ms = total / args.steps
+    print(json.dumps({"metric": "stream_step_ms", "value": ms, "unit": "ms", "higher_is_better": False,
+                      "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup), "data": "synthetic",
+                      "dtype": "bf16", "gpu_launches": int(launches),
+                      "chunk_tokens_per_sec_per_layer": B * chunk / (ms * 1e-3),
+                      "config": {"workload": "streaming step, configs[1] head layout", "layers": L, "batch": B,
+                                 "n_kv_heads": Hkv, "budget": budget, "chunk": chunk, "window": W, "sink": w.sink,
+                                 "calls_per_step": "one kvs_append_and_merge over all layers"}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -235,7 +295,13 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-groups", type=int, default=4,
                     help="end-to-end leg: layer groups whose host copies overlap the other groups' kernels")
+    ap.add_argument("--stream", action="store_true",
+                    help="time the streaming step instead (budget 2048 + chunk 512, all layers of configs[1] "
+                         "in one call); prints its own JSON line, not the headline metric")
     args = ap.parse_args()
+    if args.stream:
+        run_stream(args)
+        return
     w = wl.config(args.config)
     if args.layers:
         w = w.scaled(layers=args.layers)
