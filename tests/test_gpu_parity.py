@@ -481,6 +481,71 @@ def test_streaming_steps_match_the_oracle(kb):
     print(f"band flips followed: {flips}")
 
 
+def test_streaming_edge_cases(kb):
+    """An empty chunk is exactly kvs_merge_layer; a chunk into an empty cache that fits the budget
+    is a plain copy with counts 1; a chunk several times the budget takes several rounds and
+    equals kvs_merge_layer on the concatenation, bit for bit."""
+    import torch
+    w = _small(seed=22, batch=2, n_q_heads=8, n_kv_heads=2, window=8, seq_lens=(400, 260), budgets=(90, 70))
+    B, Hkv = w.batch, w.n_kv_heads
+    data = wl.make_layer(w)
+    # (1) empty chunk
+    dev, p, ws = _setup(kb, w, data)
+    dev2, _, ws2 = _setup(kb, w, data)
+    empty = torch.zeros((B, Hkv, 0, 128), dtype=torch.bfloat16, device="cuda")
+    n1 = kb.kvs_append_and_merge(p, dev["K"], dev["V"], dev["counts"], empty, empty, dev["q_win"],
+                                 list(w.seq_lens), list(w.budgets), ws)
+    n2 = kb.kvs_merge_layer(p, dev2["K"], dev2["V"], dev2["counts"], dev2["q_win"], list(w.seq_lens),
+                            list(w.budgets), ws2)
+    torch.cuda.synchronize()
+    assert n1 == n2 == list(w.budgets)
+    for b in range(B):
+        m = n1[b]
+        assert torch.equal(dev["K"][b, :, :m], dev2["K"][b, :, :m]) and torch.equal(dev["V"][b, :, :m], dev2["V"][b, :, :m])
+        assert torch.equal(dev["counts"][b, :, :m], dev2["counts"][b, :, :m])
+    # (2) a chunk into an empty cache, below the budget: a copy
+    dev, p, ws = _setup(kb, w, data)
+    chunk = 60
+    cK = dev2["K"][:, :, :chunk].contiguous() * 0 + 1.5          # any bf16 payload
+    cV = tl.to_dev_bf16(data["V"][:, :, 100:100 + chunk].copy())
+    dev["counts"].fill_(7)
+    n3 = kb.kvs_append_and_merge(p, dev["K"], dev["V"], dev["counts"], cK, cV, dev["q_win"], [0, 0],
+                                 list(w.budgets), ws)
+    torch.cuda.synchronize()
+    assert n3 == [60, 60]
+    assert torch.equal(dev["K"][:, :, :chunk], cK) and torch.equal(dev["V"][:, :, :chunk], cV)
+    assert torch.all(dev["counts"][:, :, :chunk] == 1) and torch.all(dev["counts"][:, :, chunk:] == 7)
+    # (3) a large chunk behind a short cache: several rounds, equal to the pass on the concatenation
+    dev, p, ws = _setup(kb, w, data)
+    dev2, _, ws2 = _setup(kb, w, data)
+    cur, chunk = [100, 40], 220
+    cK = tl.to_dev_bf16(np.ascontiguousarray(data["K"][:, :, 30:30 + chunk]))
+    cV = tl.to_dev_bf16(np.ascontiguousarray(data["V"][:, :, 30:30 + chunk]))
+    for b in range(B):
+        dev2["K"][b, :, cur[b]:cur[b] + chunk] = cK[b]
+        dev2["V"][b, :, cur[b]:cur[b] + chunk] = cV[b]
+        dev2["counts"][b, :, cur[b]:cur[b] + chunk] = 1
+    n4 = kb.kvs_append_and_merge(p, dev["K"], dev["V"], dev["counts"], cK, cV, dev["q_win"], cur,
+                                 list(w.budgets), ws)
+    n5 = kb.kvs_merge_layer(p, dev2["K"], dev2["V"], dev2["counts"], dev2["q_win"], [c + chunk for c in cur],
+                            list(w.budgets), ws2)
+    torch.cuda.synchronize()
+    assert n4 == n5 == list(w.budgets)
+    assert len(oc.full_plan(cur[0] + chunk, w.budgets[0], w.sink, w.window, w.round_frac)) >= 3
+    for b in range(B):
+        m = n4[b]
+        assert torch.equal(dev["K"][b, :, :m], dev2["K"][b, :, :m]) and torch.equal(dev["V"][b, :, :m], dev2["V"][b, :, :m])
+        assert torch.equal(dev["counts"][b, :, :m], dev2["counts"][b, :, :m])
+        assert int(dev["counts"][b, 0, :m].sum()) == cur[b] + chunk
+    # (4) no room behind the slots in use: rejected on the host, nothing is touched
+    before = dev["K"].clone()
+    with pytest.raises(kb.KvsError):
+        kb.kvs_append_and_merge(p, dev["K"], dev["V"], dev["counts"], cK, cV, dev["q_win"],
+                                [w.n_max - 10, 0], list(w.budgets), ws)
+    torch.cuda.synchronize()
+    assert torch.equal(before, dev["K"])
+
+
 def test_decode_matches_oracle_and_is_lossless_on_identical_keys(kb):
     import torch
     w = _small(seed=5, seq_lens=(400, 257), budgets=(90, 60), n_decode=5)
