@@ -8,7 +8,7 @@
 // Two teams of eight softmax warps take alternate tiles, so that one team's arithmetic overlaps
 // the other team's waits.  Inside a team the two warps of a TMEM lane quarter own the same 32
 // query rows and 64 slot columns each.  A thread reads its logits twice: once for the maximum
-// (the two threads of a row agree on the row maximum through a shared-memory atomic maximum),
+// (the two threads of a row show each other their maxima through shared memory),
 // once to form P' = exp(s - m), split into two bf16 terms and stored back into the very columns
 // the thread's logits came from (32 logits make 16 columns of hi and 16 of lo terms), keeping
 // its part of l = sum_j c_j exp(s_j - m): the count bias ln c_j of a merged slot is just the
@@ -47,24 +47,15 @@ struct Misc {
   uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[2], pready[2][2], ofull[2], stabdone[2], qfull, qready;
   uint32_t tmem_base;
   int abort_flag;
-  uint32_t rowmax[2][3][kTile];            // per team, team tile (mod 3) and query row: maximum logit, as an ordered integer
+  float rowmax[2][2][2][kTile];            // per team, tile parity, column half and query row: that thread's maximum logit
   alignas(16) float cnt[2][2][kTile];      // per team and tile parity: counts of the tile's slots (read as float4)
   float mstab[2][kTile];                   // per tile parity and query row: the stabiliser after that tile (-inf: none yet)
   float lsum[4][kTile];                    // the four parts of every row sum (team x column half)
 };
 constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc);
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
-constexpr uint32_t kColQ = 256, kColO = 384;   // TMEM columns: two logit buffers of 128, Q (64), O (128)
 
-constexpr uint32_t kOrdNegInf = 0x007fffffu;   // ordered-integer image of -infinity
-// monotone map float -> unsigned (so that an integer maximum is the float maximum) and back
-__device__ __forceinline__ uint32_t f2ord(float f) {
-  const uint32_t b = __float_as_uint(f);
-  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-}
-__device__ __forceinline__ float ord2f(uint32_t u) {
-  return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
-}
+constexpr uint32_t kColQ = 256, kColO = 384;   // TMEM columns: two logit buffers of 128, Q (64), O (128)
 
 __device__ __forceinline__ void team_barrier(int team) { asm volatile("bar.sync %0, 256;" ::"r"(team + 1) : "memory"); }
 __device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 3, 512;" ::: "memory"); }
@@ -220,7 +211,6 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     misc->abort_flag = 0;
     mbar_fence_init();
   }
-  for (int i = threadIdx.x; i < 2 * 3 * kTile; i += kThreads) (&misc->rowmax[0][0][0])[i] = kOrdNegInf;
   if (warp == 1) tmem_alloc(&misc->tmem_base, 512);
   tc_fence_before();
   __syncthreads();
@@ -494,7 +484,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       const int tile_row0 = (t_begin + li) * kTile - shift;
       const int jA = tile_row0 + ch * 64, jB = jA + 32;    // first slots of this thread's two column groups
       float* cnt = misc->cnt[team][j & 1];
-      uint32_t* rmax = misc->rowmax[team][j % 3];
+      float (*rmax)[kTile] = misc->rowmax[team][j & 1];   // (the other parity may still be read by a slow partner)
       if (ch == 0) {
         cnt[row] = (float)cnt_next;
         const int jj = tile_row0 + 2 * kTile + row;
@@ -512,12 +502,10 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
           load32(scol + 32 * sub, jA + 32 * sub, x);
           mx = fmaxf(mx, max32(x));
         }
-        atomicMax(&rmax[row], f2ord(mx));
+        rmax[ch][row] = mx;
       }
       // the one barrier of the tile: the row maxima and the staged counts of the team are complete
       team_barrier(team);
-      // the buffer of the team's tile after next was last read one tile ago: every thread is past that read now
-      if (ch == 0) misc->rowmax[team][(j + 2) % 3][row] = kOrdNegInf;
       // ---- the stabiliser after this tile, from the one after the tile before (the other team's decision)
       float m_prev = -INFINITY;
       if (li > 0) {
@@ -526,7 +514,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       }
       // row maximum of the tile: it becomes the stabiliser when the row has none yet or when it
       // has outgrown the stabiliser by more than the gap
-      const float mt = alive ? ord2f(rmax[row]) + m_stab : -INFINITY;
+      const float mt = alive ? fmaxf(rmax[0][row], rmax[1][row]) + m_stab : -INFINITY;
       const bool need = mt > -INFINITY && (m_prev == -INFINITY || mt - m_prev > kRescaleGap);
       const float m_new = need ? mt : m_prev;
       if (ch == 0) misc->mstab[li & 1][row] = m_new;
