@@ -429,9 +429,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       if (jj >= 0 && jj < n) cnt_next = ldg_here(Cb + jj);
     }
     // logits of 32 columns, relative to the stabiliser (one multiply-add), masked where needed
-    auto load32 = [&](uint32_t col, int j0, float* x) {
-      tmem_ld32(col, x);
-      tmem_ld_wait();
+    auto scale32 = [&](int j0, float* x) {
       if (j0 >= 0 && j0 + 31 <= last_free) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) x[i] = fmaf(x[i], a.scale_log2, -m_stab);
@@ -440,6 +438,11 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         for (int i = 0; i < 32; ++i)
           x[i] = (j0 + i >= 0 && j0 + i <= last_vis) ? fmaf(x[i], a.scale_log2, -m_stab) : -INFINITY;
       }
+    };
+    auto load32 = [&](uint32_t col, int j0, float* x) {
+      tmem_ld32(col, x);
+      tmem_ld_wait();
+      scale32(j0, x);
     };
     auto max32 = [&](const float* x) {
       float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one
@@ -495,13 +498,18 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       if (alive) alive = warp_wait(&misc->sfull[b], ph, abort_flag, lane);
       if (alive) {
         tc_fence_after();
-        // (loops that are not unrolled keep the code of the four roles within the instruction cache)
-        float mx = -INFINITY;
-#pragma unroll 1
-        for (int sub = 0; sub < 2; ++sub) {                // the second 32 stay in registers: they are exponentiated first
-          load32(scol + 32 * sub, jA + 32 * sub, x);
-          mx = fmaxf(mx, max32(x));
+        float mx;
+        {
+          float xa[32];
+          tmem_ld32(scol, xa);
+          tmem_ld_wait();
+          tmem_ld32(scol + 32, x);                         // in flight while the first 32 are reduced
+          scale32(jA, xa);
+          mx = max32(xa);
         }
+        tmem_ld_wait();
+        scale32(jB, x);                                    // these stay in registers: they are exponentiated first
+        mx = fmaxf(mx, max32(x));
         rmax[ch][row] = mx;
       }
       // the one barrier of the tile: the row maxima and the staged counts of the team are complete
@@ -561,6 +569,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         fence_proxy_async();                               // the tensor core reads these rows
       }
       // the last 32 slots first (their logits are still in registers), then the first 32 again from TMEM
+      // (one copy of the exponentiation code, run twice, keeps the four roles' code within the instruction cache)
 #pragma unroll 1
       for (int hf = 0; hf < 2; ++hf) {
         const int o32 = hf == 0 ? 32 : 0;
