@@ -9,7 +9,7 @@
 #include "kvs.h"
 
 #define KVS_D 128                 // head dimension
-#define KVS_SEQ_CHUNK 32          // sequences handled by one launch (kernel-parameter table)
+#define KVS_SEQ_CHUNK 128         // sequences handled by one launch (kernel-parameter table of 2 KB)
 #define KVS_MAX_M 1024            // query rows per KV head (group * window or group * n_new)
 #define KVS_MAX_SPLITS 64         // key splits of the attention partials
 #define KVS_MAX_ROUNDS 64

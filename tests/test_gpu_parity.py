@@ -406,6 +406,43 @@ def test_merge_layer_stagewise_and_end_to_end(kb):
     print(f"band flips followed: {flips}")
 
 
+def test_more_sequences_than_one_launch_table_holds(kb):
+    """150 short sequences in one call (the kernels take 128 sequences per launch, so every round
+    is two launches per kernel, of 128 and of 22 sequences) against the same sequences in two
+    calls of 128 and 22 (the same launch shapes, hence the same summation orders): merged caches,
+    lengths and decode outputs must be identical bit for bit; the bookkeeping of a unit of the
+    second table is checked too."""
+    import torch
+    B = 150
+    w = _small(seed=31, batch=B, n_q_heads=4, n_kv_heads=2, window=8,
+               seq_lens=tuple(96 + 3 * (i % 15) for i in range(B)), budgets=(64,) * B, n_decode=2)
+    data = wl.make_layer(w)
+    dev, p, ws = _setup(kb, w, data)
+    out = torch.zeros((B, w.n_q_heads, 2, 128), dtype=torch.bfloat16, device="cuda")
+    n_all = kb.kvs_merge_layer(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], list(w.seq_lens),
+                               list(w.budgets), ws)
+    kb.kvs_decode_attn(p, dev["q_new"], dev["K"], dev["V"], dev["counts"], n_all, out, ws)
+    torch.cuda.synchronize()
+    assert n_all == list(w.budgets)
+    for lo, hi in ((0, 128), (128, B)):
+        sl = slice(lo, hi)
+        part = {k: np.ascontiguousarray(v[sl]) for k, v in data.items()}
+        d2 = tl.upload_layer(part)
+        p2 = kb.make_params(d2["K"], d2["V"], w.n_q_heads, w.window, sink=w.sink, round_frac=w.round_frac)
+        out2 = torch.zeros((hi - lo, w.n_q_heads, 2, 128), dtype=torch.bfloat16, device="cuda")
+        n2 = kb.kvs_merge_layer(p2, d2["K"], d2["V"], d2["counts"], d2["q_win"], list(w.seq_lens[sl]),
+                                list(w.budgets[sl]), ws)
+        kb.kvs_decode_attn(p2, d2["q_new"], d2["K"], d2["V"], d2["counts"], n2, out2, ws)
+        torch.cuda.synchronize()
+        assert n2 == n_all[sl]
+        assert torch.equal(dev["K"][sl, :, :64], d2["K"][:, :, :64]) and torch.equal(dev["V"][sl, :, :64], d2["V"][:, :, :64])
+        assert torch.equal(dev["counts"][sl, :, :64], d2["counts"][:, :, :64])
+        assert torch.equal(out[sl], out2)
+    b = 140                                               # a sequence of the second launch table
+    assert int(dev["counts"][b, 0, :64].sum()) == w.seq_lens[b]
+    assert torch.equal(dev["K"][b, :, :w.sink], tl.to_dev_bf16(data["K"][b:b + 1])[0, :, :w.sink])
+
+
 def test_streaming_steps_match_the_oracle(kb):
     """Three streaming steps (a chunk is appended, the pass merges back to the budget) through
     kvs_append_and_merge: each step must equal, bit for bit, a plain device copy of the chunk
