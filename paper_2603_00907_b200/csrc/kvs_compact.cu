@@ -81,6 +81,18 @@ __device__ __forceinline__ bool consumer_wait(uint64_t* b0, uint64_t* b1, uint32
   return *fail == 0;
 }
 
+// Persistent CTAs per unit: the 2 x 148 CTAs that fit the GPU are shared out in proportion to the
+// units' tile counts (a ragged batch would otherwise wait for its longest sequence, which would
+// have no more CTAs than the shortest), at least one and at most one per tile.
+__host__ __device__ inline int ctas_of_unit(int unit_tiles, long long all_tiles) {
+  if (unit_tiles <= 0) return 0;
+  long long c = all_tiles > 0 ? (2LL * 148 * unit_tiles + all_tiles / 2) / all_tiles : 1;
+  if (c < 1) c = 1;
+  if (c > unit_tiles) c = unit_tiles;
+  return (int)c;
+}
+__host__ __device__ inline int tiles_of(int n, int off) { return n > off ? (n - off + KVS_CTILE - 1) / KVS_CTILE : 0; }
+
 __global__ void __launch_bounds__(kThreads, 2)
 merge_compact_kernel(const CompactArgs a, const RoundTable tab) {
   extern __shared__ __align__(128) uint8_t smem[];
@@ -93,8 +105,11 @@ merge_compact_kernel(const CompactArgs a, const RoundTable tab) {
   const int h = blockIdx.y;
   const int unit = sr.b * a.c.Hkv + h;
   const int off = tab.off;
-  const int ntiles = (n - off + KVS_CTILE - 1) / KVS_CTILE;
-  if ((int)blockIdx.x >= ntiles) return;                   // more CTAs than tiles: nothing to take
+  const int ntiles = tiles_of(n, off);
+  long long all_tiles = 0;
+  for (int i = 0; i < tab.nseq; ++i) all_tiles += tiles_of(tab.s[i].n, off);
+  const int unit_ctas = ctas_of_unit(ntiles, all_tiles * a.c.Hkv);
+  if ((int)blockIdx.x >= unit_ctas) return;                // this unit's share of the CTAs is smaller
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int P = sr.P;
 
@@ -215,7 +230,7 @@ merge_compact_kernel(const CompactArgs a, const RoundTable tab) {
       // the tile's source rows are out of global memory: later tiles may overwrite them
       if (tid == 0) st_release_u32(&a.flags[(size_t)unit * a.tile_stride + t], a.epoch);
       const int moved = E0 + __popc(selbits);
-      if (E0 > 0 && gridDim.x > 1) {
+      if (E0 > 0 && unit_ctas > 1) {
         // earlier tiles whose source rows overlap [j0 - E0, j0); a CTA that owns the whole unit
         // has read them itself, in order, before it gets here
         const int first = (j0 - E0 - off) / KVS_CTILE;
@@ -276,11 +291,15 @@ cudaError_t kvs_launch_compact(const CompactArgs& a, const RoundTable& t, cudaSt
   for (int i = 0; i < t.nseq; ++i) nmax = nmax > t.s[i].n ? nmax : t.s[i].n;
   const int ntiles = (nmax - t.off + KVS_CTILE - 1) / KVS_CTILE;
   if (ntiles <= 0) return cudaSuccess;
-  // persistent CTAs: two per SM over all units of the launch, at most one per tile
-  const int units = a.c.Hkv * t.nseq;
-  int per_unit = (2 * 148) / units;
-  if (per_unit > ntiles) per_unit = ntiles;
-  if (per_unit < 1) per_unit = 1;
+  // persistent CTAs: two per SM over all units of the launch, in proportion to the units' lengths;
+  // the grid is as wide as the longest unit's share, the CTAs beyond a unit's share leave at once
+  long long all_tiles = 0;
+  for (int i = 0; i < t.nseq; ++i) all_tiles += tiles_of(t.s[i].n, t.off);
+  int per_unit = 1;
+  for (int i = 0; i < t.nseq; ++i) {
+    const int c = ctas_of_unit(tiles_of(t.s[i].n, t.off), all_tiles * a.c.Hkv);
+    if (c > per_unit) per_unit = c;
+  }
   dim3 grid(per_unit, a.c.Hkv, t.nseq);
   merge_compact_kernel<<<grid, kThreads, kSmemBytes, st>>>(a, t);
   return cudaGetLastError();
