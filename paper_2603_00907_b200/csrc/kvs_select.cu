@@ -24,7 +24,7 @@ select_pairs_kernel(const SelectArgs a, const RoundTable tab) {
 
   __shared__ uint32_t hist[256];
   __shared__ uint32_t s_digit, s_k;
-  __shared__ uint32_t s_warp_tie[32], s_warp_sel[32];
+  __shared__ uint32_t s_cnt[128], s_pre[128];
   __shared__ uint32_t s_run_tie, s_run_sel;
 
   uint32_t prefix = 0, pmask = 0, k = (uint32_t)R;
@@ -84,53 +84,87 @@ select_pairs_kernel(const SelectArgs a, const RoundTable tab) {
       __syncthreads();
     }
   }
-  // prefix = bit pattern of the cutoff score, k = ties (in index order) still to take
+  // prefix = bit pattern of the cutoff score, k = ties (in index order) still to take.
+  // The sweep takes 4096 pairs per step (four per thread, 128 warp-sized groups): the groups'
+  // tie counts and, after the ranks are known, their selection counts are scanned by the first
+  // warp, which also gives the number of merged pairs in front of every compaction tile.
   if (tid == 0) { s_run_tie = 0; s_run_sel = 0; }
   __syncthreads();
   const int ntiles = (n - tab.off + KVS_CTILE - 1) / KVS_CTILE;
   int32_t* tp = a.tile_prefix + (size_t)unit * a.tile_stride;
-  const int sweep = ((ntiles * 32 + 1023) / 1024) * 1024;
-  // (the value of the chunk after this one is requested before this chunk's barriers)
-  uint32_t v_next = 0;
-  if (tid < P) v_next = a.from_mask ? (uint32_t)mask[tid] : __ldg(key + tid);
-  for (int p0 = 0; p0 < sweep; p0 += 1024) {
-    const int p = p0 + tid;
-    bool tie = false, less = false, sel = false;
-    const uint32_t v = v_next;
-    if (p + 1024 < P) v_next = a.from_mask ? (uint32_t)mask[p + 1024] : __ldg(key + p + 1024);
-    if (p < P) {
-      if (a.from_mask) {
-        sel = v != 0;
-      } else {
-        less = v < prefix;
-        tie = v == prefix;
+  const int sweep = ((ntiles * 32 + 4095) / 4096) * 4096;
+  // exclusive scan of the 128 group counts in s_cnt by warp 0 (lane i owns groups 4 i .. 4 i + 3)
+  auto scan_groups = [&](uint32_t* run_total) {
+    if (warp == 0) {
+      uint32_t c[4], sum = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { c[i] = s_cnt[4 * lane + i]; sum += c[i]; }
+      uint32_t inc = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
       }
+      uint32_t ex = *run_total + inc - sum;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { s_pre[4 * lane + i] = ex; ex += c[i]; }
+      __syncwarp();
+      if (lane == 31) *run_total = ex;
     }
-    const uint32_t run_tie = s_run_tie, run_sel = s_run_sel;
+  };
+  uint32_t v4[4];
+  auto fetch = [&](int p0) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int p = p0 + u * 1024 + tid;
+      v4[u] = 0;
+      if (p < P) v4[u] = a.from_mask ? (uint32_t)mask[p] : __ldg(key + p);
+    }
+  };
+  fetch(0);
+  for (int p0 = 0; p0 < sweep; p0 += 4096) {
+    uint32_t v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) v[u] = v4[u];
+    if (p0 + 4096 < sweep) fetch(p0 + 4096);              // the next step's values travel meanwhile
+    bool sel[4];
     if (!a.from_mask) {
-      const uint32_t tb = __ballot_sync(0xffffffffu, tie);
-      if (lane == 0) s_warp_tie[warp] = __popc(tb);
+      uint32_t tb[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int p = p0 + u * 1024 + tid;
+        tb[u] = __ballot_sync(0xffffffffu, p < P && v[u] == prefix);
+        if (lane == 0) s_cnt[u * 32 + warp] = __popc(tb[u]);
+      }
       __syncthreads();
-      uint32_t wpre = 0;
-      for (int wq = 0; wq < warp; ++wq) wpre += s_warp_tie[wq];
-      const uint32_t rank = run_tie + wpre + __popc(tb & ((1u << lane) - 1u));
-      sel = less || (tie && rank < k);
-      if (p < P) mask[p] = sel ? 1 : 0;
+      scan_groups(&s_run_tie);
+      __syncthreads();
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int p = p0 + u * 1024 + tid;
+        const uint32_t rank = s_pre[u * 32 + warp] + __popc(tb[u] & ((1u << lane) - 1u));
+        sel[u] = p < P && (v[u] < prefix || (v[u] == prefix && rank < k));
+        if (p < P) mask[p] = sel[u] ? 1 : 0;
+      }
+      __syncthreads();                                    // s_pre is reused below
+    } else {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) sel[u] = (p0 + u * 1024 + tid) < P && v[u] != 0;
     }
-    const uint32_t sb = __ballot_sync(0xffffffffu, sel);
-    if (lane == 0) s_warp_sel[warp] = __popc(sb);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t sb = __ballot_sync(0xffffffffu, sel[u]);
+      if (lane == 0) s_cnt[u * 32 + warp] = __popc(sb);
+    }
     __syncthreads();
-    uint32_t spre = 0;
-    for (int wq = 0; wq < warp; ++wq) spre += s_warp_sel[wq];
-    const int tile = (p0 >> 5) + warp;
-    if (lane == 0 && tile < ntiles) tp[tile] = (int32_t)(run_sel + spre);
+    scan_groups(&s_run_sel);
     __syncthreads();
-    if (tid == 1023) {
-      // last warp: totals of this chunk
-      uint32_t tt = 0;
-      if (!a.from_mask) for (int wq = 0; wq < 32; ++wq) tt += s_warp_tie[wq];
-      s_run_tie = run_tie + tt;
-      s_run_sel = run_sel + spre + s_warp_sel[31];
+    if (lane == 0) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int tile = (p0 >> 5) + u * 32 + warp;
+        if (tile < ntiles) tp[tile] = (int32_t)s_pre[u * 32 + warp];
+      }
     }
     __syncthreads();
   }
