@@ -231,10 +231,12 @@ merge_compact_kernel(const CompactArgs a, const RoundTable tab) {
       if (tid == 0) st_release_u32(&a.flags[(size_t)unit * a.tile_stride + t], a.epoch);
       const int moved = E0 + __popc(selbits);
       if (E0 > 0 && unit_ctas > 1) {
-        // earlier tiles whose source rows overlap [j0 - E0, j0); a CTA that owns the whole unit
-        // has read them itself, in order, before it gets here
+        // This tile's rows land in [j0 - E0, j0 - E0 + 64): those are source rows of at most two
+        // earlier tiles (and of this tile itself), which must have been read before they are
+        // overwritten; a CTA that owns the whole unit has read them itself, in order
         const int first = (j0 - E0 - off) / KVS_CTILE;
-        for (int tt = t - 1 - tid; tt >= first; tt -= kConsumers) {
+        const int last = min(t - 1, first + 1);
+        for (int tt = last - tid; tt >= first; tt -= kConsumers) {
           const uint32_t* f = &a.flags[(size_t)unit * a.tile_stride + tt];
           int spins = 0;
           while (ld_acquire_u32(f) < a.epoch) {
