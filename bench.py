@@ -91,7 +91,7 @@ class ClockSampler(threading.Thread):
 NCU_TRAFFIC = {
     "hessian_stats": (1.06, "kvs_stats_tc.cu", "6aa90ad0e6355729"),
     "attn_partials": (1.08, "kvs_flash_tc.cu", "f06c90efce487272"),
-    "merge_compact": (0.98, "kvs_compact.cu", "c28752d898c08b93"),
+    "merge_compact": (0.98, "kvs_compact.cu", "b399e8259464a6e9"),
 }
 
 

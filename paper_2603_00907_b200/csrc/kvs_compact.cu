@@ -86,7 +86,7 @@ __device__ __forceinline__ bool consumer_wait(uint64_t* b0, uint64_t* b1, uint32
 // have no more CTAs than the shortest), at least one and at most one per tile.
 __host__ __device__ inline int ctas_of_unit(int unit_tiles, long long all_tiles) {
   if (unit_tiles <= 0) return 0;
-  long long c = all_tiles > 0 ? (2LL * 148 * unit_tiles + all_tiles / 2) / all_tiles : 1;
+  long long c = all_tiles > 0 ? (2LL * 148 * unit_tiles) / all_tiles : 1;   // rounded down: all of them are resident at once
   if (c < 1) c = 1;
   if (c > unit_tiles) c = unit_tiles;
   return (int)c;
