@@ -500,3 +500,121 @@ def test_streaming_step_in_the_paper_setting_is_one_round():
     which merges exactly 512 of the candidate pairs."""
     plan = oc.full_plan(2048 + 512, 2048, 32, 64, 0.5)
     assert len(plan) == 1 and plan[0][3] == 512 and plan[0][2] >= 2 * 512
+
+
+# ------------------------------------------------------------------ Eq. kstar_final inside the pass
+def _bf16_exact(x):
+    """Round to bf16 and return (bits, float64 values): both sides then see the same numbers."""
+    bits = oc.f64_to_bf16(np.asarray(x, dtype=np.float64))
+    return bits, oc.bf16_to_f64(bits)
+
+
+def _fd_scalar(E, q, K, V, i, j):
+    """g_ij of h^{ij} = (g_ij / d_k) q q^T, read off the finite-difference Hessian block."""
+    qq = np.outer(q, q) / K.shape[1]
+    H = fd_hessian_block(E, q, K, V, i, j, h=2e-4)
+    return float(np.sum(H * qq) / np.sum(qq * qq))
+
+
+def _aligned_tiny_cache(seed):
+    """One query, d_v = 1, every value far above the attention output on one side (so all residuals
+    v - o have one sign), no probability above 1/2, and candidate pairs that are far from symmetric."""
+    r = np.random.default_rng(seed)
+    n, d = 9, 4
+    Kb, Kf = _bf16_exact(r.standard_normal((n, d)) * 0.8)
+    qb, qf = _bf16_exact(r.standard_normal((1, 1, d)))
+    v = r.uniform(-9.0, -7.0, size=(n, 1))                   # the protected slots pull o down
+    v[1:7, 0] = [4.0, 6.0, 7.0, 5.0, 9.0, 6.5]              # the candidate slots, all above o
+    Vb, Vf = _bf16_exact(v)
+    return n, d, Kb, Kf, qb, qf, Vb, Vf
+
+
+@pytest.mark.parametrize("seed", [21, 22, 23])
+def test_round_weights_equal_exact_hessian_weights_in_the_aligned_case(seed):
+    """Where Eq. cos_sign_relation_supp1 holds exactly (d_v = 1, residuals of one sign, alpha < 1/2) the
+    weight that the pass applies must be the exact w_m = (g11 + g12) / gamma of
+    Eq. kstar_weight_final_rewrite, with g_ij taken from a finite-difference Hessian of textbook
+    attention.  Pairs are asymmetric, so a swapped pair, a shifted slot index or a constant 1/2 fails."""
+    n, d, Kb, Kf, qb, qf, Vb, Vf = _aligned_tiny_cache(seed)
+    sink, recent, W = 1, 2, 1
+    st = oc.round_stats(Kb, Vb, np.ones(n, dtype=np.int64), qb, n - 1, 0, window=W, sink=sink,
+                        recent=recent, scale=1.0 / math.sqrt(d), causal=True, round_frac=0.5, score_mode=0)
+    assert st["off"] == 1 and st["P"] == 3
+    out, alpha = ref_attention_output(qf[0, 0], Kf, Vf)
+    assert alpha.max() < 0.5
+    E = np.array([1.0])
+    seen = []
+    for p in range(st["P"]):
+        m = st["off"] + 2 * p
+        assert Vf[m, 0] > out[0] and Vf[m + 1, 0] > out[0]
+        g11, g22, g12 = (_fd_scalar(E, qf[0, 0], Kf, Vf, m, m), _fd_scalar(E, qf[0, 0], Kf, Vf, m + 1, m + 1),
+                         _fd_scalar(E, qf[0, 0], Kf, Vf, m, m + 1))
+        w_exact = (g11 + g12) / (g11 + 2.0 * g12 + g22)
+        assert 0.0 < w_exact < 1.0 and abs(w_exact - 0.5) > 0.03, w_exact
+        assert abs(st["w"][p] - w_exact) < 2e-5, (p, st["w"][p], w_exact)
+        seen.append(w_exact)
+    assert max(seen) - min(seen) > 0.05                       # the pairs really differ from one another
+
+
+def test_round_weights_from_per_query_norms_summed_in_the_test():
+    """Several queries, causal window, merged counts: the weight of pair p must be formed from
+    N1 of slot off+2p (left), N1 of slot off+2p+1 (right) and N12 of pair p, each the sum over the
+    window queries of the norm of the per-query vector, all rebuilt here from textbook attention."""
+    r = np.random.default_rng(31)
+    n, d, dv, G, W, sink, recent = 14, 6, 5, 2, 3, 2, 3
+    Kb, Kf = _bf16_exact(r.standard_normal((n, d)))
+    Vb, Vf = _bf16_exact(r.standard_normal((n, dv)) * np.linspace(0.3, 3.0, n)[:, None])
+    Qb, Qf = _bf16_exact(r.standard_normal((G, W, d)))
+    scale = 1.0 / math.sqrt(d)
+    for rnd in (0, 1):
+        st = oc.round_stats(Kb, Vb, np.ones(n, dtype=np.int64), Qb, n - 2, rnd, window=W, sink=sink,
+                            recent=recent, scale=scale, causal=True, round_frac=0.5, score_mode=0)
+        off, P = st["off"], st["P"]
+        assert off == sink + rnd and P == (n - off - recent) // 2
+        n1 = np.zeros(n)
+        n12 = np.zeros(P)
+        for g in range(G):
+            for i in range(W):
+                vis = n - W + i + 1
+                out, a = ref_attention_output(Qf[g, i], Kf[:vis], Vf[:vis])
+                for j in range(vis):
+                    n1[j] += a[j] * abs(1.0 - 2.0 * a[j]) * math.sqrt(float(np.sum((Vf[j] - out) ** 2)))
+                for p in range(P):
+                    j = off + 2 * p
+                    n12[p] += a[j] * a[j + 1] * math.sqrt(float(np.sum((Vf[j] + Vf[j + 1] - 2.0 * out) ** 2)))
+        ws = []
+        for p in range(P):
+            j = off + 2 * p
+            D = n1[j] - 2.0 * n12[p] + n1[j + 1]
+            assert D > 1e-3 * (n1[j] + n1[j + 1])            # well away from the guard
+            want = min(1.0, max(0.0, (n1[j] - n12[p]) / D))
+            assert abs(st["w"][p] - want) < 1e-12, (rnd, p, st["w"][p], want)
+            ws.append(want)
+        assert np.ptp(ws) > 0.02 and np.max(np.abs(np.array(ws) - 0.5)) > 0.02
+
+
+def test_merge_unit_applies_the_exact_weight_to_the_left_key():
+    """One round of the whole pass on the aligned tiny cache with the middle pair forced: the merged
+    row must be bf16(w K_m + (1 - w) K_{m+1}) with w the finite-difference weight of the LEFT key,
+    the value the sum, and everything else shifted by one slot."""
+    n, d, Kb, Kf, qb, qf, Vb, Vf = _aligned_tiny_cache(22)
+    sink, recent, W = 1, 2, 1
+    forced = np.array([0, 1, 0], dtype=np.uint8)
+    K1, V1, c1 = oc.merge_unit(Kb, Vb, np.ones(n, dtype=np.int64), qb, n - 1, window=W, sink=sink,
+                               recent=recent, causal=True, round_frac=0.5, max_rounds=1,
+                               forced_masks=[forced])
+    m = 3
+    E = np.array([1.0])
+    g11, g22, g12 = (_fd_scalar(E, qf[0, 0], Kf, Vf, m, m), _fd_scalar(E, qf[0, 0], Kf, Vf, m + 1, m + 1),
+                     _fd_scalar(E, qf[0, 0], Kf, Vf, m, m + 1))
+    w = (g11 + g12) / (g11 + 2.0 * g12 + g22)
+    want = w * Kf[m] + (1.0 - w) * Kf[m + 1]
+    got = oc.bf16_to_f64(K1[m])
+    assert K1.shape[0] == n - 1 and c1[m] == 2 and c1.sum() == n
+    # the finite-difference weight is good to ~1e-5: allow that on top of half a bf16 ulp
+    assert np.all(np.abs(got - want) <= np.abs(want) * 2.0 ** -8 + 3e-5 * np.abs(Kf[m] - Kf[m + 1]))
+    # a weight of 1/2, or the weight given to the other key, would be off by many ulps on some channel
+    far = np.abs(Kf[m] - Kf[m + 1]) * abs(w - 0.5)
+    assert np.max(far / (np.abs(want) * 2.0 ** -8)) > 3.0
+    assert np.array_equal(V1[m], oc.f64_to_bf16(Vf[m] + Vf[m + 1]))
+    assert np.array_equal(K1[m + 1:], Kb[m + 2:]) and np.array_equal(K1[:m], Kb[:m])
