@@ -206,6 +206,48 @@ def rank_tokens_per_step(w, n_layers):
     return n_layers * sum(w.seq_lens)
 
 
+def free_port():
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(n):
+    """`python bench.py --gpus N` without a launcher around it: start the N ranks here (one process
+    per GPU, rendezvous on 127.0.0.1) and hand back their exit code."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def run_shard_check(args):
+    """The N > 1 plumbing without a GPU (`gloo`): every rank draws its own shard of a small workload
+    (seeds shifted by the rank), the ranks exchange a digest of it, and the step time is the slowest
+    rank's.  Prints one JSON line from rank 0.  Used by the CPU tests."""
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    w = wl.small_case(3, batch=2, seq_lens=(200, 150), budgets=(80, 60))
+    data = wl.make_layer(w, 0, seq_offset=rank)
+    digest = torch.tensor([float(data["K"].astype(np.int64).sum() % 1000003)], dtype=torch.float64)
+    gathered = [torch.zeros_like(digest) for _ in range(world)]
+    if world > 1:
+        dist.all_gather(gathered, digest)
+    else:
+        gathered = [digest]
+    ms = max_over_ranks(10.0 + 5.0 * rank, world, torch.device("cpu"))
+    if rank == 0:
+        print(json.dumps({"shard_check": True, "n_gpus": world, "ms_per_step": ms,
+                          "tokens_per_step": world * rank_tokens_per_step(w, 1),
+                          "digests": [float(g.item()) for g in gathered]}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def workload_config(w, args):
     return {"workload": f"configs[{w.config_id}] {w.name}", "layers": w.layers, "batch": w.batch,
             "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": 128,
@@ -218,7 +260,7 @@ def workload_config(w, args):
                                if args.per_layer_calls else
                                "one kvs_merge_layer + one kvs_decode_attn over all layers "
                                "(layers folded into the batch dimension)"),
-            "parallelism": f"dp{args.gpus} over sequences, no collective"}
+            "parallelism": f"dp{int(os.environ.get('WORLD_SIZE', '1'))} over sequences, no collective"}
 
 
 def run_stream(args):
@@ -298,6 +340,8 @@ def main():
     ap.add_argument("--stream", action="store_true",
                     help="time the streaming step instead (budget 2048 + chunk 512, all layers of configs[1] "
                          "in one call); prints its own JSON line, not the headline metric")
+    ap.add_argument("--shard-check", action="store_true",
+                    help="CPU only: exercise the multi-rank plumbing (gloo) on a small workload and exit")
     args = ap.parse_args()
     if args.stream:
         run_stream(args)
@@ -308,6 +352,11 @@ def main():
     if args.impl == "reference":
         run_reference(args, w)
         return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args.gpus))
+    if args.shard_check:
+        run_shard_check(args)
+        return
 
     import torch
     import torch.distributed as dist
@@ -316,6 +365,8 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but {world} rank(s) were started")
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))

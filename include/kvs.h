@@ -88,9 +88,11 @@ kvs_status_t kvs_round_plan(const kvs_params_t* params, int32_t n, int32_t budge
                             int32_t* R_r, int32_t* n_rounds);
 
 /*
- * Bytes of DEVICE workspace that kvs_merge_layer / kvs_compact / kvs_window_stats need for
- * caches of up to max_seq_len slots, and kvs_decode_attn for up to max_new query tokens
- * (pass 0 if decode is not used).  Host only.
+ * Bytes of DEVICE workspace that kvs_merge_layer / kvs_append_and_merge / kvs_compact /
+ * kvs_window_stats need for caches whose slot capacity (the n_max argument of those calls) is
+ * max_seq_len, and kvs_decode_attn for up to max_new query tokens (pass 0 if decode is not
+ * used).  The workspace layout depends on the capacity, so a call with another n_max needs the
+ * size asked for that n_max.  Host only.
  */
 kvs_status_t kvs_workspace_size(const kvs_params_t* params, int32_t max_seq_len,
                                 int32_t max_new, size_t* bytes);
@@ -103,9 +105,11 @@ kvs_status_t kvs_workspace_size(const kvs_params_t* params, int32_t max_seq_len,
  *   q_win      DEVICE bf16 [B,Hq,W,128] contiguous: queries of the last W positions
  *   seq_len    HOST int32[B]: slots in use per sequence (<= n_max)
  *   budget     HOST int32[B]: target slot count per sequence
- *   n_max      Nmax, the slot capacity that the counts layout uses
+ *   n_max      Nmax, the slot capacity that the counts layout uses (an odd capacity needs
+ *              recent >= 1: KVS_ERR_UNSUPPORTED otherwise)
  *   new_len    HOST int32[B] out: min(seq_len, budget); written before the call returns
- *   workspace  DEVICE, >= kvs_workspace_size(params, max seq_len, 0); 256-byte aligned
+ *   workspace  DEVICE, >= kvs_workspace_size(params, n_max, 0) (the layout follows the capacity
+ *              n_max, not the longest sequence); 256-byte aligned
  * A sequence with seq_len <= budget is left untouched.  Slots at index >= new_len[b] are
  * unspecified afterwards.  Rounds run back to back on the stream with no host sync.
  */
@@ -125,7 +129,7 @@ kvs_status_t kvs_merge_layer(const kvs_params_t* params, void* K, void* V, int32
  *   chunk_len         tokens appended to every sequence (>= 0)
  *   cur_len           HOST int32[B]: slots in use before the call; cur_len[b] + chunk_len <= n_max
  *   new_len           HOST int32[B] out: min(cur_len[b] + chunk_len, budget[b])
- * The workspace must cover kvs_workspace_size(params, max(cur_len) + chunk_len, 0).
+ * The workspace must cover kvs_workspace_size(params, n_max, 0).
  * Errors that the host can detect (ranges, an unreachable budget) are returned before anything
  * is enqueued, the append included.  Asynchronous on the stream; the caller owns all buffers.
  */
@@ -146,8 +150,9 @@ kvs_status_t kvs_append_and_merge(const kvs_params_t* params, void* K, void* V, 
  *              computed here: the caller passes n_merge HOST int32[B], the number of ones in
  *              each sequence's mask (per head, equal for all heads), and gets
  *              new_len = seq_len - n_merge
- *   new_index  optional DEVICE int32 [B,Hkv,Nmax] out: old slot -> new slot (the right
- *              member of a merged pair maps to its partner's new slot)
+ *   new_index  optional DEVICE int32 [B,Hkv,Nmax] out: old slot -> new slot for every slot in use
+ *              (the right member of a merged pair maps to its partner's new slot; a sequence
+ *              without a merge gets the identity)
  * Compaction indices and counts are exact integer work: the same mask gives the same
  * result bit for bit.
  */
@@ -170,10 +175,12 @@ kvs_status_t kvs_compact(const kvs_params_t* params, void* K, void* V, int32_t* 
  *
  * The scratch memory of the compaction (per-tile merge counts, tile tickets, "tile loaded" flags)
  * lives in a fixed device array inside the library, kvs_static_scratch_bytes() = 4 MiB, which
- * every GPU that loads the library holds until the process exits.  The call needs
- *   batch * n_kv_heads * (n_max / 64 + 2) * 8 bytes (+ 512)
- * of it and returns KVS_ERR_WORKSPACE, before anything is enqueued, if that exceeds the array
- * (for example 8 KV heads x 131072 slots need 131 KiB; 256 units x 32768 slots need 1.03 MiB).
+ * every GPU that loads the library holds until the process exits.  With U = batch * n_kv_heads
+ * units and T = n_max / 64 + 2 tile entries per unit the call needs
+ *   round256(U * T * 4) + round256((U + U * T) * 4) bytes
+ * (per-tile merge counts; then one ticket per unit and one flag per tile; round256 rounds up to a
+ * multiple of 256) and returns KVS_ERR_WORKSPACE, before anything is enqueued, if that exceeds the
+ * array (for example 8 KV heads x 131072 slots need 128.5 KiB; 256 units x 32768 slots need 1.005 MiB).
  * All other arguments, results and error behaviour are those of kvs_compact.
  *
  * The function calls no cudaMalloc, cudaFree or other allocating routine.  The first call on each
@@ -226,6 +233,19 @@ kvs_status_t kvs_window_stats(const kvs_params_t* params, const void* K, const v
                               float* N12, float* cosv, float* score, float* w, uint8_t* mask,
                               float* o_win, float* lse_win, void* workspace,
                               size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
+
+/*
+ * Time limit of the device-side waits, and a test hook that makes one of them run out.
+ * Every wait inside the kernels (on a tile that a copy engine delivers, on a tensor-core product,
+ * on another CTA's "tile loaded" flag) gives up after limit_us microseconds; the kernel then sets
+ * *status_dev = KVS_ERR_TIMEOUT, lets its copies in flight land, frees its tensor memory and
+ * returns, and the CUDA context stays usable.  limit_us = 0 restores the default of one second.
+ * `withhold` is for tests of that path and must be 0 in production: bit 0 makes the attention
+ * kernel's producer request no K tiles, bit 1 does the same in the statistics kernel, bit 2 keeps
+ * the compaction from publishing its "tile loaded" flags, so that the waits for them run out after
+ * limit_us without any real stall.  Applies to calls made afterwards, process wide.  Host only.
+ */
+kvs_status_t kvs_debug_set_wait(uint32_t limit_us, uint32_t withhold);
 
 /*
  * Per-kernel device timing for benchmarks.  Between kvs_profile_begin() and

@@ -22,7 +22,8 @@ STATUS_NAMES = {0: "KVS_OK", 1: "KVS_ERR_INVALID_ARG", 2: "KVS_ERR_UNSUPPORTED",
 EXPORTS = ["kvs_version", "kvs_last_error_string", "kvs_launch_count", "kvs_round_plan",
            "kvs_workspace_size", "kvs_merge_layer", "kvs_compact", "kvs_decode_attn",
            "kvs_window_stats", "kvs_profile_begin", "kvs_profile_end", "kvs_profile_kind_name",
-           "kvs_compact_static", "kvs_static_scratch_bytes", "kvs_append_and_merge"]
+           "kvs_compact_static", "kvs_static_scratch_bytes", "kvs_append_and_merge",
+           "kvs_debug_set_wait"]
 
 
 class KvsError(RuntimeError):
@@ -59,7 +60,7 @@ def lib() -> ctypes.CDLL:
         L.kvs_static_scratch_bytes.restype = ctypes.c_size_t
         for name in ("kvs_round_plan", "kvs_workspace_size", "kvs_merge_layer", "kvs_compact",
                      "kvs_decode_attn", "kvs_window_stats", "kvs_profile_begin", "kvs_profile_end",
-                     "kvs_compact_static"):
+                     "kvs_compact_static", "kvs_append_and_merge", "kvs_debug_set_wait"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -206,6 +207,12 @@ def kvs_window_stats(params: kvs_params_t, K, V, counts, q_win, seq_len: Sequenc
                                   _ptr(mask), _ptr(o_win), _ptr(lse_win), _ptr(workspace),
                                   ctypes.c_size_t(workspace.numel() * workspace.element_size()),
                                   _ptr(status_dev), _stream()))
+
+
+def kvs_debug_set_wait(limit_us: int = 0, withhold: int = 0) -> None:
+    """Time limit of the device-side waits (0: the default of one second) and the test hook that
+    makes one kind of wait run out (see kvs.h)."""
+    _check(lib().kvs_debug_set_wait(ctypes.c_uint32(limit_us), ctypes.c_uint32(withhold)))
 
 
 def kvs_profile_begin() -> None:

@@ -16,6 +16,9 @@ namespace {
 
 thread_local char g_err[256] = "";
 std::atomic<uint64_t> g_launches{0};
+constexpr uint32_t kDefaultWaitUs = 1000000;       // one second per device-side wait
+std::atomic<uint32_t> g_wait_us{kDefaultWaitUs};
+std::atomic<uint32_t> g_debug_stall{0};
 
 kvs_status_t fail(kvs_status_t code, const char* fmt, ...) {
   va_list ap;
@@ -269,20 +272,6 @@ CacheView make_view(const kvs_params_t* p, void* K, void* V, int32_t* counts, in
   return c;
 }
 
-int choose_splits(int M, int Hkv, int nseq, int nmax_slots, int* split_len) {
-  const int nqblk = (M + 127) / 128;
-  int s = (2 * 148 + nqblk * Hkv * nseq - 1) / (nqblk * Hkv * nseq);
-  const int cap = (nmax_slots + 255) / 256;
-  if (s > cap) s = cap;
-  const int bound = splits_bound(M, Hkv);
-  if (s > bound) s = bound;
-  if (s < 1) s = 1;
-  int len = (nmax_slots + s - 1) / s;
-  len = (len + 15) / 16 * 16;
-  *split_len = len;
-  return s;
-}
-
 #define CUDA_TRY(expr)                                                                   \
   do {                                                                                   \
     cudaError_t e_ = (expr);                                                             \
@@ -296,42 +285,17 @@ struct Common {
   cudaStream_t st;
   int G, Mw;
   int32_t* status_dev;
-  bool simt_stats;           // debugging aid: statistics on the CUDA cores
-  bool simt_flash;           // debugging aid: attention partials on the CUDA cores
   CUtensorMap tmK, tmV, tmQ, tmOhi, tmOlo, tmKp, tmVp;
 };
 
-int choose_splits(int M, int Hkv, int nseq, int nmax_slots, int* split_len);
-
-bool env_simt_flash() {
-  static int v = -1;
-  if (v < 0) { const char* e = getenv("KVS_DEBUG_SIMT_FLASH"); v = (e && e[0] == '1') ? 1 : 0; }
-  return v == 1;
-}
-
-// Attention partials of the rows in `q` (a [U, M, 128] view) over the caches in `view`.
+// Attention partials of the query rows behind `tmQ` (a [U, M, 128] view) over the caches in `view`.
 // Returns the number of partials per row through *n_part.
 template <class LaunchFn>
 kvs_status_t enqueue_flash(const kvs_params_t* p, char* ws, const WsLayout& L, cudaStream_t st,
-                           const CacheView& view, const void* q, int G, int Wq, int M, int causal,
-                           const RoundTable& tab, int nmax_slots, bool simt, const CUtensorMap& tmK,
+                           const CacheView& view, int Wq, int M, int causal,
+                           const RoundTable& tab, int nmax_slots, const CUtensorMap& tmK,
                            const CUtensorMap& tmV, const CUtensorMap& tmQ, int32_t* status_dev,
                            bool pair_norms, LaunchFn&& launch_fn, int* n_part) {
-  float2* part_ml = reinterpret_cast<float2*>(ws + L.part_ml);
-  float* part_o = reinterpret_cast<float*>(ws + L.part_o);
-  const float scale_log2 = p->softmax_scale * 1.4426950408889634f;
-  if (simt) {
-    FlashArgs fa;
-    fa.c = view;
-    fa.q = static_cast<const __nv_bfloat16*>(q);
-    fa.Hq = p->n_q_heads; fa.G = G; fa.Wq = Wq; fa.M = M;
-    fa.causal = causal;
-    fa.scale_log2 = scale_log2;
-    fa.splits = choose_splits(M, p->n_kv_heads, tab.nseq, nmax_slots, &fa.split_len);
-    fa.part_ml = part_ml; fa.part_o = part_o;
-    *n_part = fa.splits;
-    return launch_fn([&] { return kvs_launch_flash_simt(fa, tab, st); });
-  }
   FlashTcArgs ta;
   ta.Hkv = p->n_kv_heads; ta.M = M; ta.nqblk = (M + 127) / 128;
   // with pair norms the tiles start at -(off & 1), so that candidate pairs never straddle a tile
@@ -339,23 +303,23 @@ kvs_status_t enqueue_flash(const kvs_params_t* p, char* ws, const WsLayout& L, c
   ta.pair_norms = pair_norms ? reinterpret_cast<float4*>(ws + L.norms) : nullptr;
   ta.pair_stride = L.pair_stride;
   ta.splits = tc_splits(M, p->n_kv_heads, tab.nseq, ntiles, &ta.tiles_per_split);
-  ta.Wq = Wq; ta.causal = causal; ta.scale_log2 = scale_log2;
+  ta.Wq = Wq; ta.causal = causal; ta.scale_log2 = p->softmax_scale * 1.4426950408889634f;
   ta.n_max = view.n_max; ta.counts = view.counts;
-  ta.part_ml = part_ml; ta.part_o = part_o; ta.status_dev = status_dev;
+  ta.part_ml = reinterpret_cast<float2*>(ws + L.part_ml);
+  ta.part_o = reinterpret_cast<float*>(ws + L.part_o);
+  ta.status_dev = status_dev;
+  ta.wait_us = g_wait_us.load(); ta.debug_stall = g_debug_stall.load();
   *n_part = ta.splits;
   return launch_fn([&] { return kvs_launch_flash_tc(ta, tab, tmK, tmV, tmQ, st); });
-}
-
-bool env_simt_stats() {
-  static int v = -1;
-  if (v < 0) { const char* e = getenv("KVS_DEBUG_SIMT_STATS"); v = (e && e[0] == '1') ? 1 : 0; }
-  return v == 1;
 }
 
 // Tensor maps of one call: K and V caches [B,Hkv,n_max,128] with the caller's strides, the
 // window queries and the two bf16 terms of the attention output as [U, M, 128].
 kvs_status_t make_call_tmaps(Common* c, const void* K, const void* V, const void* q_win, int n_max) {
   const kvs_params_t* p = c->p;
+  // the pair view covers floor(n_max / 2) slot pairs: with an odd capacity and no protected suffix
+  // the last slot could be the right member of a candidate pair and lie outside the view
+  if ((n_max & 1) && p->recent == 0) return fail(KVS_ERR_UNSUPPORTED, "an odd n_max needs recent >= 1");
   const uint64_t kd[4] = {KVS_D, (uint64_t)n_max, (uint64_t)p->n_kv_heads, (uint64_t)p->batch};
   const uint64_t ks[3] = {(uint64_t)p->k_stride_t * 2, (uint64_t)p->k_stride_h * 2, (uint64_t)p->k_stride_b * 2};
   const uint64_t vs[3] = {(uint64_t)p->v_stride_t * 2, (uint64_t)p->v_stride_h * 2, (uint64_t)p->v_stride_b * 2};
@@ -381,8 +345,8 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
   const float scale_log2 = p->softmax_scale * 1.4426950408889634f;
   int n_part = 0;
   {
-    kvs_status_t fs = enqueue_flash(p, c.ws, c.L, c.st, view, q_win, c.G, p->window, c.Mw, p->causal, tab,
-                                    nmax_slots, c.simt_flash, c.tmK, c.tmV, c.tmQ, c.status_dev, !c.simt_stats,
+    kvs_status_t fs = enqueue_flash(p, c.ws, c.L, c.st, view, p->window, c.Mw, p->causal, tab, nmax_slots,
+                                    c.tmK, c.tmV, c.tmQ, c.status_dev, true,
                                     [&](auto&& f) -> kvs_status_t {
                                       CUDA_TRY(launch(KVS_K_FLASH, c.st, f));
                                       return KVS_OK;
@@ -402,43 +366,33 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
   ca.out_bf16 = nullptr; ca.lse_out = lse_out; ca.o_out = o_out;
   CUDA_TRY(launch(KVS_K_COMBINE, c.st, [&] { return kvs_launch_combine(ca, tab, c.st); }));
 
-  StatsArgs sa;
-  sa.c = view;
-  sa.q = static_cast<const __nv_bfloat16*>(q_win); sa.Hq = p->n_q_heads; sa.G = c.G; sa.Wq = p->window; sa.M = c.Mw;
-  sa.causal = p->causal; sa.scale_log2 = scale_log2; sa.score_mode = p->score_mode;
-  sa.qstat = ca.qstat; sa.o = ca.o;
-  sa.pair_stride = c.L.pair_stride;
-  sa.score = score_out ? score_out : reinterpret_cast<float*>(c.ws + c.L.score);
-  sa.w = w_out ? w_out : reinterpret_cast<float*>(c.ws + c.L.w);
-  sa.A = A; sa.N1 = N1; sa.N12 = N12; sa.cosv = cosv;
-  if (c.simt_stats) {
-    CUDA_TRY(launch(KVS_K_STATS, c.st, [&] { return kvs_launch_stats_simt(sa, tab, c.st); }));
-  } else {
-    StatsTcArgs ta;
-    ta.Hkv = p->n_kv_heads; ta.M = c.Mw; ta.nqblk = (c.Mw + 127) / 128;
-    int pmax = 0;
-    for (int i = 0; i < tab.nseq; ++i) pmax = pmax > tab.s[i].P ? pmax : tab.s[i].P;
-    const int ntiles = (pmax + 127) / 128;               // tiles of 128 candidate pairs
-    ta.splits = balanced_splits(ta.nqblk * ta.Hkv * tab.nseq, ntiles, &ta.tiles_per_split);
-    ta.n_max = view.n_max; ta.pair_stride = c.L.pair_stride;
-    ta.scale_log2 = scale_log2; ta.score_mode = p->score_mode;
-    ta.counts = view.counts; ta.qc2 = ca.qc2; ta.M_pad = ca.M_pad;
-    ta.pair_norms = reinterpret_cast<const float4*>(c.ws + c.L.norms); ta.norm_stride = c.L.pair_stride;
-    ta.score = sa.score; ta.w = sa.w; ta.A = A; ta.N1 = N1; ta.N12 = N12; ta.cosv = cosv;
-    ta.partA = reinterpret_cast<float*>(c.ws + c.L.partA);
-    ta.partN1 = reinterpret_cast<float*>(c.ws + c.L.partN1);
-    ta.partN12 = reinterpret_cast<float*>(c.ws + c.L.partN12);
-    ta.status_dev = c.status_dev;
-    CUDA_TRY(launch(KVS_K_STATS, c.st, [&] {
-      return kvs_launch_stats_tc(ta, tab, c.tmKp, c.tmVp, c.tmQ, c.tmOhi, c.tmOlo, c.st);
-    }));
-  }
+  StatsTcArgs ta;
+  ta.Hkv = p->n_kv_heads; ta.M = c.Mw; ta.nqblk = (c.Mw + 127) / 128;
+  int pmax = 0;
+  for (int i = 0; i < tab.nseq; ++i) pmax = pmax > tab.s[i].P ? pmax : tab.s[i].P;
+  const int ntiles = (pmax + 127) / 128;               // tiles of 128 candidate pairs
+  ta.splits = balanced_splits(ta.nqblk * ta.Hkv * tab.nseq, ntiles, &ta.tiles_per_split);
+  ta.n_max = view.n_max; ta.pair_stride = c.L.pair_stride;
+  ta.scale_log2 = scale_log2; ta.score_mode = p->score_mode;
+  ta.counts = view.counts; ta.qc2 = ca.qc2; ta.M_pad = ca.M_pad;
+  ta.pair_norms = reinterpret_cast<const float4*>(c.ws + c.L.norms); ta.norm_stride = c.L.pair_stride;
+  ta.score = score_out ? score_out : reinterpret_cast<float*>(c.ws + c.L.score);
+  ta.w = w_out ? w_out : reinterpret_cast<float*>(c.ws + c.L.w);
+  ta.A = A; ta.N1 = N1; ta.N12 = N12; ta.cosv = cosv;
+  ta.partA = reinterpret_cast<float*>(c.ws + c.L.partA);
+  ta.partN1 = reinterpret_cast<float*>(c.ws + c.L.partN1);
+  ta.partN12 = reinterpret_cast<float*>(c.ws + c.L.partN12);
+  ta.status_dev = c.status_dev;
+  ta.wait_us = g_wait_us.load(); ta.debug_stall = g_debug_stall.load();
+  CUDA_TRY(launch(KVS_K_STATS, c.st, [&] {
+    return kvs_launch_stats_tc(ta, tab, c.tmKp, c.tmVp, c.tmQ, c.tmOhi, c.tmOlo, c.st);
+  }));
 
   if (do_select) {
     SelectArgs se;
     se.Hkv = p->n_kv_heads;
     se.pair_stride = c.L.pair_stride; se.tile_stride = c.L.tile_stride;
-    se.score = sa.score;
+    se.score = ta.score;
     se.mask = mask_out ? mask_out : reinterpret_cast<uint8_t*>(c.ws + c.L.mask);
     se.tile_prefix = reinterpret_cast<int32_t*>(c.ws + c.L.tile_prefix);
     se.from_mask = 0;
@@ -469,9 +423,6 @@ kvs_status_t check_common(const kvs_params_t* p, const void* K, const void* V, c
   c->G = p->n_q_heads / p->n_kv_heads;
   c->Mw = c->G * p->window;
   c->status_dev = nullptr;
-  c->simt_flash = env_simt_flash();
-  // the tensor-core statistics need the pair norms that the tensor-core attention pass writes
-  c->simt_stats = env_simt_stats() || c->simt_flash;
   return KVS_OK;
 }
 
@@ -554,6 +505,7 @@ kvs_status_t kvs_detail_compact_scratch(const kvs_params_t* p, void* K, void* V,
     ka.epoch = 1;
     ka.new_index = new_index;
     ka.status_dev = status_dev;
+    ka.wait_us = g_wait_us.load(); ka.debug_stall = g_debug_stall.load();
     CUDA_TRY(launch(KVS_K_COMPACT, st, [&] { return kvs_launch_compact(ka, tab, st); }));
   }
   return KVS_OK;
@@ -567,6 +519,13 @@ int kvs_version(void) { return 100; }
 const char* kvs_last_error_string(void) { return g_err; }
 
 uint64_t kvs_launch_count(void) { return g_launches.load(); }
+
+kvs_status_t kvs_debug_set_wait(uint32_t limit_us, uint32_t withhold) {
+  if (withhold > 7u) return fail(KVS_ERR_INVALID_ARG, "withhold has three bits");
+  g_wait_us.store(limit_us ? limit_us : kDefaultWaitUs);
+  g_debug_stall.store(withhold);
+  return KVS_OK;
+}
 
 kvs_status_t kvs_round_plan(const kvs_params_t* p, int32_t n, int32_t budget, int32_t max_rounds,
                             int32_t* n_r, int32_t* off_r, int32_t* P_r, int32_t* R_r,
@@ -694,6 +653,8 @@ kvs_status_t merge_layer_impl(const kvs_params_t* p, void* K, void* V, int32_t* 
       ka.epoch = (uint32_t)(i + 1);
       ka.new_index = nullptr;
       ka.status_dev = status_dev;
+      ka.wait_us = g_wait_us.load(); ka.debug_stall = g_debug_stall.load();
+    ka.wait_us = g_wait_us.load(); ka.debug_stall = g_debug_stall.load();
       CUDA_TRY(launch(KVS_K_COMPACT, c.st, [&] { return kvs_launch_compact(ka, tab, c.st); }));
     }
   }
@@ -790,6 +751,7 @@ kvs_status_t kvs_compact(const kvs_params_t* p, void* K, void* V, int32_t* count
     ka.epoch = 1;
     ka.new_index = new_index;
     ka.status_dev = status_dev;
+    ka.wait_us = g_wait_us.load(); ka.debug_stall = g_debug_stall.load();
     CUDA_TRY(launch(KVS_K_COMPACT, c.st, [&] { return kvs_launch_compact(ka, tab, c.st); }));
   }
   return KVS_OK;
@@ -799,7 +761,6 @@ kvs_status_t kvs_decode_attn(const kvs_params_t* p, const void* q_new, int32_t n
                              const void* V, const int32_t* counts, const int32_t* seq_len,
                              int32_t n_max, void* out, float* lse, void* workspace,
                              size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
-  (void)status_dev;
   if (n_new <= 0) return fail(KVS_ERR_INVALID_ARG, "n_new must be positive");
   if (p && p->n_kv_heads > 0 && (int64_t)(p->n_q_heads / p->n_kv_heads) * n_new > KVS_MAX_M)
     return fail(KVS_ERR_UNSUPPORTED, "group * n_new must be <= %d", KVS_MAX_M);
@@ -818,8 +779,8 @@ kvs_status_t kvs_decode_attn(const kvs_params_t* p, const void* q_new, int32_t n
     const uint64_t vs[3] = {(uint64_t)p->v_stride_t * 2, (uint64_t)p->v_stride_h * 2, (uint64_t)p->v_stride_b * 2};
     const uint64_t qd[3] = {KVS_D, (uint64_t)M, (uint64_t)c.L.U};
     const uint64_t qs[2] = {KVS_D * 2, (uint64_t)M * KVS_D * 2};
-    if (!c.simt_flash && !(make_tmap(&tmK, K, 4, kd, ks, 128) && make_tmap(&tmV, V, 4, kd, vs, 128) &&
-                           make_tmap(&tmQ, q_new, 3, qd, qs, 128)))
+    if (!(make_tmap(&tmK, K, 4, kd, ks, 128) && make_tmap(&tmV, V, 4, kd, vs, 128) &&
+          make_tmap(&tmQ, q_new, 3, qd, qs, 128)))
       return fail(KVS_ERR_CUDA, "cuTensorMapEncodeTiled failed or is unavailable");
   }
   for (int b0 = 0; b0 < B; b0 += KVS_SEQ_CHUNK) {
@@ -833,8 +794,7 @@ kvs_status_t kvs_decode_attn(const kvs_params_t* p, const void* q_new, int32_t n
     }
     if (tab.nseq == 0) continue;
     int n_part = 0;
-    s = enqueue_flash(p, c.ws, c.L, c.st, view, q_new, c.G, n_new, M, 0, tab, nmax_slots, c.simt_flash, tmK,
-                      tmV, tmQ, status_dev, false,
+    s = enqueue_flash(p, c.ws, c.L, c.st, view, n_new, M, 0, tab, nmax_slots, tmK, tmV, tmQ, status_dev, false,
                       [&](auto&& f) -> kvs_status_t {
                         CUDA_TRY(launch(KVS_K_FLASH, c.st, f));
                         return KVS_OK;

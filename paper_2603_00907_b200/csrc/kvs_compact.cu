@@ -57,7 +57,7 @@ struct TileMeta {
 };
 struct Shared {
   uint64_t full[kStages], meta_full[kStages], empty[kStages];
-  int abort_flag;
+  int abort_flag, wait_us;       // (adjacent: the bounded waits read both through one pointer)
   int fail;
   TileMeta meta[kStages];
 };
@@ -106,6 +106,14 @@ merge_compact_kernel(const CompactArgs a, const RoundTable tab) {
   const int unit = sr.b * a.c.Hkv + h;
   const int off = tab.off;
   const int ntiles = tiles_of(n, off);
+  if (ntiles == 0) {
+    // a unit that ends inside the protected prefix has nothing to move; its slot map is the identity
+    if (a.new_index && blockIdx.x == 0) {
+      int32_t* ni = a.new_index + (size_t)unit * a.c.n_max;
+      for (int j = threadIdx.x; j < n; j += kThreads) ni[j] = j;
+    }
+    return;
+  }
   long long all_tiles = 0;
   for (int i = 0; i < tab.nseq; ++i) all_tiles += tiles_of(tab.s[i].n, off);
   const int unit_ctas = ctas_of_unit(ntiles, all_tiles * a.c.Hkv);
@@ -120,6 +128,7 @@ merge_compact_kernel(const CompactArgs a, const RoundTable tab) {
       mbar_init(&sh->empty[s], kConsumers / 32);
     }
     sh->abort_flag = 0;
+    sh->wait_us = (int)a.wait_us;
     sh->fail = 0;
     mbar_fence_init();
   }
@@ -136,13 +145,19 @@ merge_compact_kernel(const CompactArgs a, const RoundTable tab) {
     const float* wl = a.w + (size_t)unit * a.pair_stride;
     uint32_t next_ticket = 0;
     if (lane == 0) next_ticket = atomicAdd(&a.tickets[unit], 1u);
+    int issued = 0;                  // tiles whose copies were requested
     for (int k = 0;; ++k) {
       const int s = k % kStages;
       const uint32_t ph = (uint32_t)(k / kStages) & 1u;
       int ok = 1;
       if (lane == 0) ok = mbar_wait(&sh->empty[s], ph ^ 1u, abort_flag) ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
+      if (!ok) {
+        // give the copies of the last stages a bounded time to land before the CTA leaves
+        if (lane == 0)
+          for (int kk = max(0, issued - kStages); kk < issued; ++kk) mbar_drain(&sh->full[kk % kStages], (uint32_t)(kk / kStages) & 1u);
+        break;
+      }
       const int t = (int)__shfl_sync(0xffffffffu, next_ticket, 0);
       TileMeta* m = &sh->meta[s];
       if (t >= ntiles) {
@@ -155,6 +170,7 @@ merge_compact_kernel(const CompactArgs a, const RoundTable tab) {
       uint8_t* sk = smem + s * kStageBytes;
       uint8_t* sv = sk + kOperandBytes;
       if (lane == 0) mbar_expect_tx(&sh->full[s], (uint32_t)rows * 2u * kRowBytes);
+      issued = k + 1;
       __syncwarp();
       if (a.c.kst == KVS_D && a.c.vst == KVS_D) {
         if (lane == 0) bulk_load(sk, Kb + (int64_t)j0 * KVS_D, (uint32_t)rows * kRowBytes, &sh->full[s]);
@@ -228,7 +244,8 @@ merge_compact_kernel(const CompactArgs a, const RoundTable tab) {
         cl += cr;
       }
       // the tile's source rows are out of global memory: later tiles may overwrite them
-      if (tid == 0) st_release_u32(&a.flags[(size_t)unit * a.tile_stride + t], a.epoch);
+      // (test hook: with bit 2 of debug_stall the flag stays unset, so that the waits on it run out)
+      if (tid == 0 && !(a.debug_stall & 4u)) st_release_u32(&a.flags[(size_t)unit * a.tile_stride + t], a.epoch);
       const int moved = E0 + __popc(selbits);
       if (E0 > 0 && unit_ctas > 1) {
         // This tile's rows land in [j0 - E0, j0 - E0 + 64): those are source rows of at most two
@@ -239,8 +256,10 @@ merge_compact_kernel(const CompactArgs a, const RoundTable tab) {
         for (int tt = last - tid; tt >= first; tt -= kConsumers) {
           const uint32_t* f = &a.flags[(size_t)unit * a.tile_stride + tt];
           int spins = 0;
+          const uint64_t t0 = globaltimer_ns();
           while (ld_acquire_u32(f) < a.epoch) {
-            if (++spins > KVS_SPIN_LIMIT || *abort_flag) { *fail = 1; *abort_flag = 1; break; }
+            const bool late = (++spins & 255) == 0 && globaltimer_ns() - t0 > (uint64_t)(uint32_t)sh->wait_us * 1000ull;
+            if (late || spins > KVS_SPIN_LIMIT || *abort_flag) { *fail = 1; *abort_flag = 1; break; }
             __nanosleep(20);
           }
         }
@@ -283,16 +302,16 @@ merge_compact_kernel(const CompactArgs a, const RoundTable tab) {
 }  // namespace
 
 cudaError_t kvs_launch_compact(const CompactArgs& a, const RoundTable& t, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(merge_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static KvsPerDeviceOnce configured;
+  cudaError_t ce = configured.run([] {
+    return cudaFuncSetAttribute(merge_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  });
+  if (ce != cudaSuccess) return ce;
   int nmax = 0;
   for (int i = 0; i < t.nseq; ++i) nmax = nmax > t.s[i].n ? nmax : t.s[i].n;
   const int ntiles = (nmax - t.off + KVS_CTILE - 1) / KVS_CTILE;
-  if (ntiles <= 0) return cudaSuccess;
+  // (units that end inside the protected prefix still get their identity slot map)
+  if (nmax <= 0 || (ntiles <= 0 && !a.new_index)) return cudaSuccess;
   // persistent CTAs: two per SM over all units of the launch, in proportion to the units' lengths;
   // the grid is as wide as the longest unit's share, the CTAs beyond a unit's share leave at once
   long long all_tiles = 0;

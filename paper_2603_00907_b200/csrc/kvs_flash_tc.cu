@@ -46,7 +46,7 @@ constexpr float kRescaleGap = 8.f;         // log2 units
 struct Misc {
   uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[2], pready[2][2], ofull[2], stabdone[2], qfull, qready;
   uint32_t tmem_base;
-  int abort_flag;
+  int abort_flag, wait_us;                 // (adjacent: the bounded waits read both through one pointer)
   float rowmax[2][2][2][kTile];            // per team, tile parity, column half and query row: that thread's maximum logit
   alignas(16) float cnt[2][2][kTile];      // per team and tile parity: counts of the tile's slots (read as float4)
   float mstab[2][kTile];                   // per tile parity and query row: the stabiliser after that tile (-inf: none yet)
@@ -209,6 +209,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     mbar_init(&misc->qfull, 1);
     mbar_init(&misc->qready, kSoftmaxWarps);
     misc->abort_flag = 0;
+    misc->wait_us = (int)a.wait_us;
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc(&misc->tmem_base, 512);
@@ -217,6 +218,8 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
   tc_fence_after();
   const uint32_t tmem = __shfl_sync(0xffffffffu, misc->tmem_base, 0);   // (uniform for the compiler too)
   volatile int* abort_flag = &misc->abort_flag;
+  // test hook: the producer requests no K tile, so that the waits on them run out
+  const bool withhold_k = (a.debug_stall & 1u) != 0;
 
   if (warp == 0) {
     // ================================================================ TMA producer
@@ -234,8 +237,10 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         if (!mbar_wait(&misc->kfree[s], ((kli >> 1) & 1) ^ 1, abort_flag)) return false;
         uint8_t* st = smem + kSmemStage + s * kStage;
         const int row = (t_begin + kli) * kTile - shift;
-        mbar_expect_tx(&misc->kfull[s], kOperand);
-        for (int hf = 0; hf < 2; ++hf) tma_load_4d(st + hf * kHalf, &tmK, &misc->kfull[s], hf * 64, row, h, sr.b);
+        if (!withhold_k) {
+          mbar_expect_tx(&misc->kfull[s], kOperand);
+          for (int hf = 0; hf < 2; ++hf) tma_load_4d(st + hf * kHalf, &tmK, &misc->kfull[s], hf * 64, row, h, sr.b);
+        }
         ++kli;
         return true;
       };
@@ -256,14 +261,8 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       }
       if (*abort_flag) {
         // drain: give the copies already issued a bounded time to land before the CTA leaves
-        for (int li = max(0, kli - 2); li < kli; ++li) {
-          const uint64_t t1 = globaltimer_ns();
-          while (!mbar_try_wait(&misc->kfull[li & 1], (li >> 1) & 1) && globaltimer_ns() - t1 < 200000000ull) {}
-        }
-        for (int li = max(0, vli - 2); li < vli; ++li) {
-          const uint64_t t1 = globaltimer_ns();
-          while (!mbar_try_wait(&misc->vfull[li & 1], (li >> 1) & 1) && globaltimer_ns() - t1 < 200000000ull) {}
-        }
+        for (int li = max(0, kli - 2); li < kli && !withhold_k; ++li) mbar_drain(&misc->kfull[li & 1], (li >> 1) & 1);
+        for (int li = max(0, vli - 2); li < vli; ++li) mbar_drain(&misc->vfull[li & 1], (li >> 1) & 1);
       }
     }
   } else if (warp == 1) {
@@ -616,12 +615,11 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
 
 cudaError_t kvs_launch_flash_tc(const FlashTcArgs& a, const RoundTable& t, const CUtensorMap& tmK,
                                 const CUtensorMap& tmV, const CUtensorMap& tmQ, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(flash_partial_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static KvsPerDeviceOnce configured;
+  cudaError_t ce = configured.run([] {
+    return cudaFuncSetAttribute(flash_partial_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  });
+  if (ce != cudaSuccess) return ce;
   dim3 grid(a.nqblk * a.splits, a.Hkv, t.nseq);
   flash_partial_tc<<<grid, kThreads, kSmemBytes, st>>>(a, t, tmK, tmV, tmQ);
   return cudaGetLastError();

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "kvs.h"
 
 #define KVS_D 128                 // head dimension
@@ -50,18 +52,6 @@ struct CacheView {
   int32_t Hkv;
 };
 
-struct FlashArgs {
-  CacheView c;
-  const __nv_bfloat16* q;  // [B, Hq, Wq, 128]
-  int32_t Hq, G, Wq, M;    // M = G * Wq rows per KV head
-  int32_t causal;
-  float scale_log2;        // softmax_scale * log2(e)
-  int32_t splits;
-  int32_t split_len;       // keys per split (multiple of the key tile)
-  float2* part_ml;         // [U, splits, M]  (running max in log2 units, sum)
-  float* part_o;           // [U, splits, M, 128]
-};
-
 struct FlashTcArgs {
   int32_t Hkv, M, nqblk, splits, tiles_per_split;
   int32_t Wq, causal;
@@ -73,6 +63,8 @@ struct FlashTcArgs {
   float4* pair_norms;      // optional [U, pair_stride]: (|vbar_l|^2, |vbar_r|^2, |vbar_l + vbar_r|^2, cos(K_l, K_r))
   int32_t pair_stride;     //   of the round's candidate pairs; tiles are then aligned with the pairs
   int32_t* status_dev;
+  uint32_t wait_us;        // time limit of one device-side wait, microseconds
+  uint32_t debug_stall;    // test hook (kvs_debug_set_wait): bit 0 = the producer withholds the K tiles
 };
 
 struct CombineArgs {
@@ -88,24 +80,6 @@ struct CombineArgs {
   __nv_bfloat16* out_bf16; // decode: [B, Hq, n_new, 128] == [U, M, 128] (may be NULL)
   float* lse_out;          // optional [U, M]
   float* o_out;            // optional diagnostic copy [U, M, 128]
-};
-
-struct StatsArgs {
-  CacheView c;
-  const __nv_bfloat16* q;
-  int32_t Hq, G, Wq, M;
-  int32_t causal;
-  float scale_log2;
-  int32_t score_mode;
-  const float4* qstat;
-  const float* o;
-  int32_t pair_stride;     // row length of the per-pair arrays (n_max / 2)
-  float* score;            // [U, pair_stride]
-  float* w;                // [U, pair_stride]
-  float* A;                // optional diagnostics [U, n_max]
-  float* N1;
-  float* N12;              // [U, pair_stride]
-  float* cosv;
 };
 
 struct StatsTcArgs {
@@ -128,6 +102,8 @@ struct StatsTcArgs {
   const float4* pair_norms; // [U, norm_stride] from the attention pass
   int32_t norm_stride;
   int32_t* status_dev;
+  uint32_t wait_us;        // time limit of one device-side wait, microseconds
+  uint32_t debug_stall;    // test hook: bit 1 = the producer withholds the K tiles
 };
 
 struct SelectArgs {
@@ -151,13 +127,13 @@ struct CompactArgs {
   uint32_t epoch;
   int32_t* new_index;      // optional [U, n_max]
   int32_t* status_dev;
+  uint32_t wait_us;        // time limit of one device-side wait, microseconds
+  uint32_t debug_stall;    // test hook: bit 2 = "tile loaded" flags are not published
 };
 
 // ----------------------------------------------------------------------------- launchers
 // Each returns the cudaError_t of its launch.  `nseq_units` = table.nseq * Hkv.
-cudaError_t kvs_launch_flash_simt(const FlashArgs& a, const RoundTable& t, cudaStream_t st);
 cudaError_t kvs_launch_combine(const CombineArgs& a, const RoundTable& t, cudaStream_t st);
-cudaError_t kvs_launch_stats_simt(const StatsArgs& a, const RoundTable& t, cudaStream_t st);
 // tmKp / tmVp: 5-D pair views [128, parity, slot / 2, head, sequence] of the caches
 cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const CUtensorMap& tmKp,
                                 const CUtensorMap& tmVp, const CUtensorMap& tmQ, const CUtensorMap& tmOhi,
@@ -174,6 +150,23 @@ struct AppendArgs {
 cudaError_t kvs_launch_append(const AppendArgs& a, const RoundTable& t, cudaStream_t st);
 cudaError_t kvs_launch_select(const SelectArgs& a, const RoundTable& t, cudaStream_t st);
 cudaError_t kvs_launch_compact(const CompactArgs& a, const RoundTable& t, cudaStream_t st);
+
+// Runs a per-device set-up call (raising a kernel's dynamic shared-memory limit) once for every
+// device ordinal that launches through it: the attribute belongs to the device's copy of the kernel.
+struct KvsPerDeviceOnce {
+  std::atomic<unsigned char> done[64] = {};
+  template <class F>
+  cudaError_t run(F&& f) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return f();      // beyond the table: set up on every launch
+    if (done[dev].load(std::memory_order_acquire)) return cudaSuccess;
+    e = f();
+    if (e == cudaSuccess) done[dev].store(1, std::memory_order_release);
+    return e;
+  }
+};
 
 // ----------------------------------------------------------------------------- device helpers
 #ifdef __CUDACC__

@@ -77,20 +77,26 @@ __device__ __forceinline__ bool mbar_poll(uint64_t* bar, uint32_t parity, uint32
       : "memory");
   return ok != 0;
 }
-// Bounded wait: false after ~1 s (or when another role already flagged an abort).
+// Bounded wait: false once the time limit has passed (or when another role already flagged an
+// abort).  `ctl` points at two ints in shared memory: ctl[0] is the CTA's abort flag, ctl[1] the
+// time limit of one wait in microseconds (one second unless the host asked otherwise).
 // These kernels are chains of hand-offs, so the wake-up latency of a wait counts for more than
 // the issue slots its polling takes: a wait on the critical path (`eager`) polls in a tight
 // loop and looks at the clock only between bursts; a role that runs ahead of the others anyway
 // lets the hardware suspend it between attempts.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          bool eager = false) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* ctl, bool eager = false) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   while (!(eager ? mbar_poll(bar, parity, 256) : mbar_try_wait_hint(bar, parity, 10000u))) {
-    if (*abort_flag) return false;
-    if (globaltimer_ns() - t0 > 1000000000ull) { *abort_flag = 1; return false; }
+    if (ctl[0]) return false;
+    if (globaltimer_ns() - t0 > (uint64_t)(uint32_t)ctl[1] * 1000ull) { ctl[0] = 1; return false; }
   }
   return true;
+}
+// Time a role gives copies already in flight to land before its CTA leaves after an abort.
+__device__ __forceinline__ void mbar_drain(uint64_t* bar, uint32_t parity) {
+  const uint64_t t1 = globaltimer_ns();
+  while (!mbar_try_wait(bar, parity) && globaltimer_ns() - t1 < 200000000ull) {}
 }
 
 // Loads that stay where they are written: the compiler may move a plain load of a value that is

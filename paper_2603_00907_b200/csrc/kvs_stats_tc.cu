@@ -43,7 +43,7 @@ constexpr int kThreads = (2 + kStatWarps) * 32;   // warp 0: TMA, warp 1: MMA, w
 struct Misc {
   uint64_t kfull, vfull, kfree, vfree, tfull[2], tfree[2], qfull, xhand[kGroups - 1][4], xfree[4];
   uint32_t tmem_base;
-  int abort_flag;
+  int abort_flag, wait_us;                 // (adjacent: the bounded waits read both through one pointer)
   float xbuf[kPairs * 5];                  // partial sums of a pair on their way from the last group down to group 0
 };
 constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc);
@@ -137,6 +137,7 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
       mbar_init(&misc->xfree[q], 1);
     }
     misc->abort_flag = 0;
+    misc->wait_us = (int)a.wait_us;
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc(&misc->tmem_base, 512);
@@ -145,6 +146,8 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
   tc_fence_after();
   const uint32_t tmem = __shfl_sync(0xffffffffu, misc->tmem_base, 0);   // (uniform for the compiler too)
   volatile int* abort_flag = &misc->abort_flag;
+  // test hook: the producer requests no K tile, so that the waits on them run out
+  const bool withhold_k = (a.debug_stall & 2u) != 0;
 
   // tensor-map coordinates of the pair members: slot = 2 * rho + parity
   const int par_l = off & 1, par_r = par_l ^ 1;
@@ -176,10 +179,12 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
         bool progress = false;
         if (kli < my_tiles && mbar_try_wait(&misc->kfree, (kli & 1) ^ 1)) {
           const int p0 = (t_begin + kli) * kPairs;
-          mbar_expect_tx(&misc->kfull, 2 * kOperand);
-          for (int hf = 0; hf < 2; ++hf) {
-            tma_load_5d(smem + kSmemKl + hf * kHalf, &tmKp, &misc->kfull, hf * 64, par_l, rho_l0 + p0, h, sr.b);
-            tma_load_5d(smem + kSmemKr + hf * kHalf, &tmKp, &misc->kfull, hf * 64, par_r, rho_r0 + p0, h, sr.b);
+          if (!withhold_k) {
+            mbar_expect_tx(&misc->kfull, 2 * kOperand);
+            for (int hf = 0; hf < 2; ++hf) {
+              tma_load_5d(smem + kSmemKl + hf * kHalf, &tmKp, &misc->kfull, hf * 64, par_l, rho_l0 + p0, h, sr.b);
+              tma_load_5d(smem + kSmemKr + hf * kHalf, &tmKp, &misc->kfull, hf * 64, par_r, rho_r0 + p0, h, sr.b);
+            }
           }
           if (kli + 1 < my_tiles) prefetch(kli + 1, false);
           ++kli;
@@ -200,14 +205,13 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
           t0 = globaltimer_ns();
         } else {
           if (*abort_flag) break;
-          if (globaltimer_ns() - t0 > 1000000000ull) { *abort_flag = 1; break; }
+          if (globaltimer_ns() - t0 > (uint64_t)(uint32_t)misc->wait_us * 1000ull) { *abort_flag = 1; break; }
         }
       }
       if (*abort_flag) {
         // drain: give the copies already issued a bounded time to land before the CTA leaves
-        const uint64_t t1 = globaltimer_ns();
-        while (kli > 0 && !mbar_try_wait(&misc->kfull, (kli - 1) & 1) && globaltimer_ns() - t1 < 200000000ull) {}
-        while (vli > 0 && !mbar_try_wait(&misc->vfull, (vli - 1) & 1) && globaltimer_ns() - t1 < 200000000ull) {}
+        if (kli > 0 && !withhold_k) mbar_drain(&misc->kfull, (kli - 1) & 1);
+        if (vli > 0) mbar_drain(&misc->vfull, (vli - 1) & 1);
       }
     }
   } else if (warp == 1) {
@@ -417,12 +421,11 @@ stats_finalize_kernel(const StatsTcArgs a, const RoundTable tab) {
 cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const CUtensorMap& tmKp,
                                 const CUtensorMap& tmVp, const CUtensorMap& tmQ, const CUtensorMap& tmOhi,
                                 const CUtensorMap& tmOlo, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(hessian_stats_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static KvsPerDeviceOnce configured;
+  cudaError_t ce = configured.run([] {
+    return cudaFuncSetAttribute(hessian_stats_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  });
+  if (ce != cudaSuccess) return ce;
   dim3 grid(a.nqblk * a.splits, a.Hkv, t.nseq);
   hessian_stats_tc<<<grid, kThreads, kSmemBytes, st>>>(a, t, tmKp, tmVp, tmQ, tmOhi, tmOlo);
   cudaError_t e = cudaGetLastError();

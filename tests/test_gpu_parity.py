@@ -67,25 +67,14 @@ def _check_round_stats(kb, w, K, V, C, q_win, n_list, r, score_mode=0, causal=Tr
                                 q_win[b, h * G:(h + 1) * G], w.budgets[b], r,
                                 **_oracle_kwargs(w, score_mode=score_mode, causal=causal))
             refs[(b, h)] = st
-            off, P, R = st["off"], st["P"], st["R"]
-            sl = slice(off, off + 2 * P)
-            for name, g, ref in (("A", A[b, h, sl], st["A"][sl]), ("N1", N1[b, h, sl], st["N1"][sl]),
-                                 ("N12", N12[b, h, :P], st["N12"]), ("score", score[b, h, :P], st["score"]),
-                                 ("o", o_win[b, h], st["o"])):
-                # o is an intermediate formed on the tensor cores from a two-term bf16 split of the
-                # probabilities: held to 1e-4; the statistics that the method uses to 1e-5
-                ok, ratio, plain = tl.stat_close(g, ref, rtol=tl.O_RTOL if name == "o" else tl.STAT_RTOL)
-                report.append((b, h, name, ratio, plain))
-                assert ok, f"{name} unit {(b, h)} round {r}: err/allowed {ratio:.3g} plain rel {plain:.3g}"
-            # cosine: compared through 1 - cos (what the score uses), absolute 1e-6
-            assert np.max(np.abs(cosv[b, h, :P] - st["cos"])) < 2e-6
-            # weights: compare where the denominator is well conditioned
-            D = st["N1"][off:off + 2 * P:2] - 2 * st["N12"] + st["N1"][off + 1:off + 2 * P:2]
-            good = D > 1e-3 * (st["N1"][off:off + 2 * P:2] + st["N1"][off + 1:off + 2 * P:2])
-            assert np.max(np.abs(wgt[b, h, :P][good] - st["w"][good])) < 2e-3
-            assert np.all((wgt[b, h, :P] >= 0) & (wgt[b, h, :P] <= 1))
-            ok, nm, nout = tl.mask_band_ok(mask[b, h, :P], st["mask"], st["score"], R)
-            assert ok, f"mask unit {(b, h)} round {r}: {nm} mismatches, {nout} outside the band"
+            got = {"A": A[b, h], "N1": N1[b, h], "N12": N12[b, h], "cos": cosv[b, h], "score": score[b, h],
+                   "w": wgt[b, h], "mask": mask[b, h]}
+            worst = tl.check_unit_stats(got, st, label=f"unit {(b, h)} round {r}")
+            # o is an intermediate formed on the tensor cores from a two-term bf16 split of the
+            # probabilities: held to 1e-4 of max(|ref|, mean |ref|) (its elements cross zero)
+            ok, ratio, plain = tl.stat_close(o_win[b, h], st["o"], rtol=tl.O_RTOL)
+            assert ok, f"o unit {(b, h)} round {r}: err/allowed {ratio:.3g}"
+            report.append((b, h, worst))
     return refs, {"mask": mask, "w": wgt, "report": report}
 
 
@@ -149,7 +138,7 @@ def test_attention_partials_with_late_spikes(kb):
         ok, ratio, plain = tl.stat_close(o_win[0, h].cpu().numpy(), o, rtol=tl.O_RTOL)
         assert ok, (h, ratio, plain)
         off, P, _ = oc.round_plan(4000, 1500, w.sink, w.window, 0.5, 0)
-        ok, ratio, plain = tl.stat_close(A[0, h, off:off + 2 * P].cpu().numpy(), alpha.sum(0)[off:off + 2 * P])
+        ok, ratio, plain = tl.rel_close(A[0, h, off:off + 2 * P].cpu().numpy(), alpha.sum(0)[off:off + 2 * P])
         assert ok, (h, ratio, plain)
         s = (Qf.reshape(M, 128) @ Kf.T) / math.sqrt(128)
         i = np.tile(np.arange(w.window), w.group)
@@ -193,7 +182,7 @@ def test_attention_partials_with_spikes_in_consecutive_tiles(kb):
         ok, ratio, plain = tl.stat_close(o_win[0, h].cpu().numpy(), o, rtol=tl.O_RTOL)
         assert ok, (h, ratio, plain)
         off, P, _ = oc.round_plan(4000, 1500, w.sink, w.window, 0.5, 0)
-        ok, ratio, plain = tl.stat_close(A[0, h, off:off + 2 * P].cpu().numpy(), alpha.sum(0)[off:off + 2 * P])
+        ok, ratio, plain = tl.rel_close(A[0, h, off:off + 2 * P].cpu().numpy(), alpha.sum(0)[off:off + 2 * P])
         assert ok, (h, ratio, plain)
         i = np.tile(np.arange(w.window), w.group)
         s = np.where(np.arange(4000)[None, :] > (4000 - w.window + i)[:, None], -np.inf, s)
@@ -338,71 +327,88 @@ def test_compact_one_cta_per_unit_and_strided_rows(kb):
             n_list = got
 
 
-def test_merge_layer_stagewise_and_end_to_end(kb):
-    """Round by round from the oracle's state (statistics, mask modulo the cutoff band, merge),
-    then the whole pass in one call: it must equal the composition of single-round calls bit
-    for bit, and the oracle that follows the GPU's near-cutoff choices."""
+def full_pass_vs_oracle(kb, w, data, units=None, seq_len=None, budgets=None):
+    """The whole pass in one call; the same pass as single-round calls (it must equal their
+    composition bit for bit); and, for the (sequence, KV head) `units` (all when None), the oracle
+    that follows the GPU's near-cutoff choices: every deviation of the GPU's mask from the oracle's
+    own must lie in the cutoff band, counts must be identical and K / value sums within the bf16
+    tolerance.  Returns the merged caches (numpy) and the number of band flips followed."""
     import torch
-    w = _small(seed=4, seq_lens=(700, 333), budgets=(128, 64))
-    data = wl.make_layer(w)
     B, Hkv, Nmax = data["K"].shape[:3]
     G = w.group
-    plans = [oc.full_plan(n, bud, w.sink, w.window, w.round_frac) for n, bud in zip(w.seq_lens, w.budgets)]
+    seq_len = list(w.seq_lens) if seq_len is None else list(seq_len)
+    budgets = list(w.budgets) if budgets is None else list(budgets)
+    plans = [oc.full_plan(n, bud, w.sink, w.window, w.round_frac) if n > bud else []
+             for n, bud in zip(seq_len, budgets)]
     rounds = max(len(pl) for pl in plans)
 
     # (1) full pass in one call
     dev, p, ws = _setup(kb, w, data)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    new_len = kb.kvs_merge_layer(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], list(w.seq_lens),
-                                 list(w.budgets), ws, status_dev=status)
+    new_len = kb.kvs_merge_layer(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], seq_len, budgets, ws,
+                                 status_dev=status)
     torch.cuda.synchronize()
-    assert status.item() == 0 and new_len == list(w.budgets)
+    assert status.item() == 0 and new_len == [min(n, b) for n, b in zip(seq_len, budgets)]
     K_full, V_full, C_full = tl.bits_of(dev["K"]), tl.bits_of(dev["V"]), dev["counts"].cpu().numpy()
+    del dev
 
     # (2) the same pass as single-round calls, recording the GPU's masks
     dev2, _, ws2 = _setup(kb, w, data)
-    n_list = list(w.seq_lens)
+    n_list = list(seq_len)
     gpu_masks = []
     for r in range(rounds):
         pr = kb.make_params(dev2["K"], dev2["V"], w.n_q_heads, w.window, sink=w.sink,
                             round_frac=w.round_frac, first_round=r)
         mask = torch.zeros((B, Hkv, Nmax // 2), dtype=torch.uint8, device="cuda")
-        kb.kvs_window_stats(pr, dev2["K"], dev2["V"], dev2["counts"], dev2["q_win"], n_list,
-                            list(w.budgets), ws2, mask=mask)
-        step_budget = [plans[b][r][0] - plans[b][r][3] if r < len(plans[b]) else w.budgets[b]
+        kb.kvs_window_stats(pr, dev2["K"], dev2["V"], dev2["counts"], dev2["q_win"], n_list, budgets, ws2, mask=mask)
+        step_budget = [plans[b][r][0] - plans[b][r][3] if r < len(plans[b]) else min(seq_len[b], budgets[b])
                        for b in range(B)]
         n_list = kb.kvs_merge_layer(pr, dev2["K"], dev2["V"], dev2["counts"], dev2["q_win"], n_list,
                                     step_budget, ws2)
-        gpu_masks.append(mask.cpu().numpy())
+        gpu_masks.append(mask.cpu().numpy() if units is None else
+                         {(b, h): mask[b, h].cpu().numpy() for (b, h) in units})
     torch.cuda.synchronize()
-    assert n_list == list(w.budgets)
+    assert n_list == new_len
+    K2, V2, C2 = tl.bits_of(dev2["K"]), tl.bits_of(dev2["V"]), dev2["counts"].cpu().numpy()
     for b in range(B):
-        m = w.budgets[b]
-        assert np.array_equal(tl.bits_of(dev2["K"])[b, :, :m], K_full[b, :, :m])
-        assert np.array_equal(tl.bits_of(dev2["V"])[b, :, :m], V_full[b, :, :m])
-        assert np.array_equal(dev2["counts"].cpu().numpy()[b, :, :m], C_full[b, :, :m])
+        m = new_len[b]
+        assert np.array_equal(K2[b, :, :m], K_full[b, :, :m])
+        assert np.array_equal(V2[b, :, :m], V_full[b, :, :m])
+        assert np.array_equal(C2[b, :, :m], C_full[b, :, :m])
 
     # (3) oracle following the GPU's masks; every deviation from its own mask must be in the band
     flips = 0
-    for b in range(B):
-        n0 = w.seq_lens[b]
-        for h in range(Hkv):
-            forced = [gpu_masks[r][b, h, :plans[b][r][2]] for r in range(len(plans[b]))]
-            trace = []
-            Ko, Vo, Co = oc.merge_unit(data["K"][b, h, :n0], data["V"][b, h, :n0],
-                                       data["counts"][b, h, :n0], data["q_win"][b, h * G:(h + 1) * G],
-                                       w.budgets[b], forced_masks=forced, trace=trace,
-                                       **_oracle_kwargs(w))
-            for r, st in enumerate(trace):
-                ok, nm, nout = tl.mask_band_ok(forced[r], st["mask"], st["score"], st["R"])
-                assert ok, f"unit {(b, h)} round {r}: {nm} mask mismatches, {nout} outside the band"
-                flips += nm
-            m = w.budgets[b]
-            assert np.array_equal(C_full[b, h, :m], Co)
-            assert Co.sum() == n0
-            okk, mxk, nulpk, _ = tl.bf16_close(K_full[b, h, :m], Ko)
-            okv, mxv, nulpv, _ = tl.bf16_close(V_full[b, h, :m], Vo)
-            assert okk and okv, (mxk, mxv)
+    todo = [(b, h) for b in range(B) for h in range(Hkv)] if units is None else list(units)
+    for (b, h) in todo:
+        n0 = seq_len[b]
+        if n0 <= budgets[b]:
+            continue
+        gm = (lambda r: gpu_masks[r][b, h]) if units is None else (lambda r: gpu_masks[r][(b, h)])
+        forced = [gm(r)[:plans[b][r][2]] for r in range(len(plans[b]))]
+        trace = []
+        Ko, Vo, Co = oc.merge_unit(data["K"][b, h, :n0], data["V"][b, h, :n0],
+                                   data["counts"][b, h, :n0], data["q_win"][b, h * G:(h + 1) * G],
+                                   budgets[b], forced_masks=forced, trace=trace, **_oracle_kwargs(w))
+        for r, st in enumerate(trace):
+            ok, nm, nout = tl.mask_band_ok(forced[r], st["mask"], st["score"], st["R"])
+            assert ok, f"unit {(b, h)} round {r}: {nm} mask mismatches, {nout} outside the band"
+            flips += nm
+        m = budgets[b]
+        assert np.array_equal(C_full[b, h, :m], Co)
+        assert Co.sum() == n0
+        okk, mxk, nulpk, _ = tl.bf16_close(K_full[b, h, :m], Ko)
+        okv, mxv, nulpv, _ = tl.bf16_close(V_full[b, h, :m], Vo)
+        assert okk and okv, (b, h, mxk, mxv)
+    return K_full, V_full, C_full, new_len, flips
+
+
+def test_merge_layer_stagewise_and_end_to_end(kb):
+    """Round by round from the oracle's state (statistics, mask modulo the cutoff band, merge),
+    then the whole pass in one call: it must equal the composition of single-round calls bit
+    for bit, and the oracle that follows the GPU's near-cutoff choices."""
+    w = _small(seed=4, seq_lens=(700, 333), budgets=(128, 64))
+    data = wl.make_layer(w)
+    *_, flips = full_pass_vs_oracle(kb, w, data)
     print(f"band flips followed: {flips}")
 
 

@@ -56,3 +56,27 @@ def test_rank_shards_are_reproducible_and_rank0_is_the_single_gpu_batch():
     assert np.array_equal(a["K"], b["K"]) and np.array_equal(a["V"], b["V"])
     assert np.array_equal(wl.make_layer(w, 0)["K"], wl.make_layer(w, 0, seq_offset=0)["K"])
     assert not np.array_equal(a["K"], wl.make_layer(w, 0)["K"])
+
+
+def test_bench_starts_its_own_ranks():
+    """`python bench.py --gpus 2` with no launcher around it starts two ranks itself; in its CPU
+    self-check mode they run the sharding arithmetic over gloo: rank -> its own shard, tokens x
+    world, time = the slowest rank's."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--shard-check"],
+                       capture_output=True, text=True, timeout=300, env=env, cwd=root)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                  # rank 0 alone prints
+    d = lines[0]
+    assert d["n_gpus"] == 2 and d["ms_per_step"] == 15.0 and d["tokens_per_step"] == 2 * (200 + 150)
+    assert len(d["digests"]) == 2 and d["digests"][0] != d["digests"][1]
+    # one rank, no launcher: the same path without a process group
+    r1 = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "1", "--shard-check"],
+                        capture_output=True, text=True, timeout=300, env=env, cwd=root)
+    d1 = json.loads([l for l in r1.stdout.splitlines() if l.startswith("{")][0])
+    assert d1["n_gpus"] == 1 and d1["tokens_per_step"] == 350 and d1["digests"] == d["digests"][:1]
