@@ -235,6 +235,46 @@ kvs_status_t kvs_window_stats(const kvs_params_t* params, const void* K, const v
                               size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
 
 /*
+ * Non-uniform budgets: the merge pass and the decode check with a length and a budget per
+ * (sequence, KV head) instead of per sequence  [Section 6 (discussion): one compression ratio for
+ * every layer and head is the method's stated limitation; the heads of a sequence may now end at
+ * different lengths].  Everything else is kvs_merge_layer / kvs_decode_attn: each (sequence, head)
+ * is treated as a sequence of its own with one KV head and its n_q_heads / n_kv_heads query heads.
+ *   seq_len, budget   HOST int32[B*Hkv], index b * Hkv + h
+ *   new_len           HOST int32[B*Hkv] out: min(seq_len, budget) per head
+ *   workspace         >= kvs_workspace_size_per_head(params, n_max, max_new)
+ * The caches must have k/v_stride_b == n_kv_heads * k/v_stride_h (the usual contiguous
+ * [B,Hkv,Nmax,128] layout, or any layout whose heads tile the sequence stride); otherwise
+ * KVS_ERR_UNSUPPORTED.  Slots at index >= new_len[b * Hkv + h] of a head are unspecified afterwards.
+ */
+kvs_status_t kvs_workspace_size_per_head(const kvs_params_t* params, int32_t n_max, int32_t max_new,
+                                         size_t* bytes);
+kvs_status_t kvs_merge_layer_per_head(const kvs_params_t* params, void* K, void* V, int32_t* counts,
+                                      const void* q_win, const int32_t* seq_len, const int32_t* budget,
+                                      int32_t n_max, int32_t* new_len, void* workspace,
+                                      size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
+kvs_status_t kvs_decode_attn_per_head(const kvs_params_t* params, const void* q_new, int32_t n_new,
+                                      const void* K, const void* V, const int32_t* counts,
+                                      const int32_t* seq_len, int32_t n_max, void* out, float* lse,
+                                      void* workspace, size_t workspace_bytes, int32_t* status_dev,
+                                      void* cuda_stream);
+
+/*
+ * Adjacent-token cosine similarity of a bf16 tensor along its token axis  [Section 3.2,
+ * Eq. cosine_raw]:  cos_out[b,h,t] = <x_t, x_t+1> / max(|x_t| |x_t+1|, 1e-30)  for t < seq_len[b] - 1.
+ * A diagnostic for the queries, keys and values of a layer (the method rests on adjacent keys
+ * being nearly parallel and adjacent values not); independent of the merge pass.
+ *   x          DEVICE bf16 [B,H,Nmax,128], element strides stride_b / stride_h / stride_t
+ *              (multiples of 8, stride_t >= 128), 16-byte aligned; read only
+ *   seq_len    HOST int32[B]: rows in use per sequence (<= n_max)
+ *   cos_out    DEVICE fp32 [B,H,Nmax] contiguous; entries t >= seq_len[b] - 1 are not written
+ * No workspace.  Asynchronous on the stream.
+ */
+kvs_status_t kvs_adjacent_cosine(const void* x, int32_t batch, int32_t n_heads, int32_t n_max,
+                                 int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                                 const int32_t* seq_len, float* cos_out, void* cuda_stream);
+
+/*
  * Time limit of the device-side waits, and a test hook that makes one of them run out.
  * Every wait inside the kernels (on a tile that a copy engine delivers, on a tensor-core product,
  * on another CTA's "tile loaded" flag) gives up after limit_us microseconds; the kernel then sets

@@ -17,7 +17,9 @@ What is computed (paper passages in brackets):
   linear system M k* = N and its weight-form solution [Eqs. H_gamma_rank1_rewrite,
   u_rank1_rewrite, kstar_weight_final_rewrite];
 * the gradient-free merged key [Eq. kstar_final] with the norms of the c-vectors
-  summed over the window queries;
+  summed over the window queries; and, as variants of the weight only, the exact weights from a
+  supplied loss gradient E [Eq. kstar_weight_final_rewrite with g_ij = E^T c_ij] and the
+  diagonal-only merge that drops the coupling [Section 3.1, Eq. simplified_k];
 * the value merge v* = v_m + v_{m+1} [Section 3.1] and the count bookkeeping;
 * the chunk schedule "merge R adjacent pairs in parallel" [Section 3.1], repeated in
   rounds until the budget is met; the first `sink` tokens are never merged
@@ -25,7 +27,8 @@ What is computed (paper passages in brackets):
 * attention over the merged cache for new queries (numerator uses value sums,
   denominator weights each slot by its count);
 * the streaming step: a chunk of fresh tokens is appended and the pass brings the cache
-  back to the budget [Section 3.1; Section 5.1: budget 2048, chunk 512].
+  back to the budget [Section 3.1; Section 5.1: budget 2048, chunk 512];
+* the adjacent-token cosine similarity of queries, keys or values [Section 3.2, Eq. cosine_raw].
 
 Readings where the paper is silent are fixed here and listed in the design notes:
 aligned candidate pairs with alternating parity, pair score = attention mass times
@@ -271,6 +274,40 @@ def pair_weights(N1: np.ndarray, N12: np.ndarray, off: int, P: int) -> np.ndarra
     return w
 
 
+def exact_pair_sums(alpha: np.ndarray, o: np.ndarray, vbar: np.ndarray, E: np.ndarray, off: int,
+                    P: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
+    """Scalar sensitivities of every candidate pair with a supplied loss gradient E [M, d_v] (one row
+    per window query, E_q = dL/do_q): g_ij^(q) = E_q^T c_ij^(q) [Section 4.2, text before
+    Eq. h_rank1_unified], summed over the window queries (the Hessian of the summed loss is the sum
+    of the per-query Hessians).  Returns G11, G22, G12 [P] and, for tolerances, the sum of the
+    absolute values of all terms that entered each pair."""
+    G11, G22, G12, Gabs = np.zeros(P), np.zeros(P), np.zeros(P), np.zeros(P)
+    for p in range(P):
+        j = off + 2 * p
+        for q in range(alpha.shape[0]):
+            c11, c22, c12 = c_vectors(alpha[q, j], alpha[q, j + 1], vbar[j], vbar[j + 1], o[q])
+            g11, g22, g12 = float(E[q] @ c11), float(E[q] @ c22), float(E[q] @ c12)
+            G11[p] += g11
+            G22[p] += g22
+            G12[p] += g12
+            Gabs[p] += abs(g11) + abs(g22) + 2.0 * abs(g12)
+    return G11, G22, G12, Gabs
+
+
+def exact_form_weight(g11: float, g22: float, g12: float, diagonal_only: bool = False) -> float:
+    """Weight of k_m from the scalar sensitivities: (g11 + g12) / (g11 + 2 g12 + g22)
+    [Eq. kstar_weight_final_rewrite]; with `diagonal_only` the coupling g12 is dropped, which is
+    the diagonal-Hessian merge that the paper starts from [Section 3.1, Eq. simplified_k].
+    Guard (reading, paper silent): the quadratic model has a minimum only for gamma > 0; if gamma
+    is not safely positive the weight is 1/2; the result is clipped to [0, 1]."""
+    if diagonal_only:
+        g12 = 0.0
+    gamma = g11 + 2.0 * g12 + g22
+    if not (math.isfinite(gamma) and gamma > 1e-6 * (abs(g11) + abs(g22))):
+        return 0.5
+    return min(1.0, max(0.0, (g11 + g12) / gamma))
+
+
 def apply_merge(K_bits: np.ndarray, V_bits: np.ndarray, c: np.ndarray, off: int,
                 mask: np.ndarray, w: np.ndarray
                 ) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
@@ -300,8 +337,14 @@ def apply_merge(K_bits: np.ndarray, V_bits: np.ndarray, c: np.ndarray, off: int,
 
 def round_stats(K_bits: np.ndarray, V_bits: np.ndarray, c: np.ndarray, Q_bits: np.ndarray,
                 budget: int, r: int, *, window: int, sink: int, recent: int, scale: float,
-                causal: bool, round_frac: float, score_mode: int) -> Dict[str, np.ndarray]:
-    """Everything round r decides on the current cache of one unit (nothing is modified)."""
+                causal: bool, round_frac: float, score_mode: int, weight_mode: int = 0,
+                E_bits: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+    """Everything round r decides on the current cache of one unit (nothing is modified).
+
+    weight_mode 0: gradient-free weights from the summed norms [Eq. kstar_final];
+    1: exact weights from a supplied loss gradient E_bits (bf16 [G, W, d_v], one row per window
+    query) [Eq. kstar_weight_final_rewrite]; 2: the same with the coupling term dropped
+    [Eq. simplified_k].  Scores and selection do not depend on the mode."""
     n = K_bits.shape[0]
     Kf = bf16_to_f64(K_bits)
     Vs = bf16_to_f64(V_bits)
@@ -314,16 +357,24 @@ def round_stats(K_bits: np.ndarray, V_bits: np.ndarray, c: np.ndarray, Q_bits: n
     A, N1 = slot_stats(alpha, o, vbar)
     N12, cosv, score = pair_stats(Kf, alpha, o, vbar, A, off, P, score_mode)
     mask = select_pairs(score, R)
-    w = pair_weights(N1, N12, off, P)
-    return {"off": off, "P": P, "R": R, "A": A, "N1": N1, "N12": N12, "cos": cosv,
-            "score": score, "mask": mask, "w": w, "o": o, "alpha": alpha}
+    out = {"off": off, "P": P, "R": R, "A": A, "N1": N1, "N12": N12, "cos": cosv,
+           "score": score, "mask": mask, "o": o, "alpha": alpha}
+    if weight_mode == 0:
+        out["w"] = pair_weights(N1, N12, off, P)
+    else:
+        E = bf16_to_f64(E_bits).reshape(alpha.shape[0], -1)
+        G11, G22, G12, Gabs = exact_pair_sums(alpha, o, vbar, E, off, P)
+        out.update(G11=G11, G22=G22, G12=G12, Gabs=Gabs)
+        out["w"] = np.array([exact_form_weight(G11[p], G22[p], G12[p], weight_mode == 2) for p in range(P)])
+    return out
 
 
 def merge_unit(K_bits: np.ndarray, V_bits: np.ndarray, c: np.ndarray, Q_bits: np.ndarray,
                budget: int, *, window: int, sink: int = 32, recent: Optional[int] = None,
                scale: Optional[float] = None, causal: bool = True, round_frac: float = 0.5,
                score_mode: int = 0, first_round: int = 0, max_rounds: Optional[int] = None,
-               forced_masks: Optional[List[np.ndarray]] = None, trace: Optional[list] = None
+               forced_masks: Optional[List[np.ndarray]] = None, trace: Optional[list] = None,
+               weight_mode: int = 0, E_bits: Optional[np.ndarray] = None
                ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
     """The whole pass on one (sequence, KV head): rounds until n == budget.
 
@@ -339,7 +390,7 @@ def merge_unit(K_bits: np.ndarray, V_bits: np.ndarray, c: np.ndarray, Q_bits: np
     while K_bits.shape[0] > budget and (max_rounds is None or done < max_rounds):
         st = round_stats(K_bits, V_bits, c, Q_bits, budget, r, window=window, sink=sink,
                          recent=recent, scale=scale, causal=causal, round_frac=round_frac,
-                         score_mode=score_mode)
+                         score_mode=score_mode, weight_mode=weight_mode, E_bits=E_bits)
         mask = st["mask"] if forced_masks is None else np.asarray(forced_masks[done], dtype=np.uint8)
         assert int(mask.sum()) == st["R"]
         if trace is not None:
@@ -386,20 +437,35 @@ def decode_attention(q_bits: np.ndarray, K_bits: np.ndarray, V_bits: np.ndarray,
     return out.reshape(G, T, -1), lse.reshape(G, T)
 
 
+def adjacent_cosine(X_bits: np.ndarray) -> np.ndarray:
+    """cos(y_t, y_t+1) = <y_t, y_t+1> / (|y_t| |y_t+1|) of consecutive rows of a bf16 matrix [n, d]
+    [Section 3.2, Eq. cosine_raw]; returns float64 [n - 1] (denominator floored at 1e-30)."""
+    X = bf16_to_f64(X_bits)
+    out = np.zeros(max(0, X.shape[0] - 1))
+    for t in range(out.shape[0]):
+        den = max(np.linalg.norm(X[t]) * np.linalg.norm(X[t + 1]), 1e-30)
+        out[t] = float(X[t] @ X[t + 1]) / den
+    return out
+
+
 def merge_layer(inputs: Dict[str, np.ndarray], *, window: int, sink: int = 32,
                 recent: Optional[int] = None, causal: bool = True, round_frac: float = 0.5,
                 score_mode: int = 0, heads: Optional[List[int]] = None,
                 sequences: Optional[List[int]] = None) -> Dict[Tuple[int, int], tuple]:
-    """All (sequence, KV head) units of one layer; returns {(b, h): (K_bits, V_bits, counts)}."""
+    """All (sequence, KV head) units of one layer; returns {(b, h): (K_bits, V_bits, counts)}.
+    `seq_len` and `budget` are per sequence ([B]) or, for non-uniform budgets, per (sequence,
+    KV head) ([B, Hkv]): units are independent, so a head simply runs to its own budget."""
     K, V, counts, q_win = inputs["K"], inputs["V"], inputs["counts"], inputs["q_win"]
     B, Hkv = K.shape[0], K.shape[1]
     G = q_win.shape[1] // Hkv
+    seq_len = np.broadcast_to(np.asarray(inputs["seq_len"]).reshape(B, -1), (B, Hkv))
+    budget = np.broadcast_to(np.asarray(inputs["budget"]).reshape(B, -1), (B, Hkv))
     out = {}
     for b in (range(B) if sequences is None else sequences):
-        n = int(inputs["seq_len"][b])
         for h in (range(Hkv) if heads is None else heads):
+            n = int(seq_len[b, h])
             out[(b, h)] = merge_unit(K[b, h, :n], V[b, h, :n], counts[b, h, :n],
-                                     q_win[b, h * G:(h + 1) * G], int(inputs["budget"][b]),
+                                     q_win[b, h * G:(h + 1) * G], int(budget[b, h]),
                                      window=window, sink=sink, recent=recent, causal=causal,
                                      round_frac=round_frac, score_mode=score_mode)
     return out

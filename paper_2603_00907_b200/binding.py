@@ -23,7 +23,8 @@ EXPORTS = ["kvs_version", "kvs_last_error_string", "kvs_launch_count", "kvs_roun
            "kvs_workspace_size", "kvs_merge_layer", "kvs_compact", "kvs_decode_attn",
            "kvs_window_stats", "kvs_profile_begin", "kvs_profile_end", "kvs_profile_kind_name",
            "kvs_compact_static", "kvs_static_scratch_bytes", "kvs_append_and_merge",
-           "kvs_debug_set_wait"]
+           "kvs_debug_set_wait", "kvs_adjacent_cosine",
+           "kvs_workspace_size_per_head", "kvs_merge_layer_per_head", "kvs_decode_attn_per_head"]
 
 
 class KvsError(RuntimeError):
@@ -60,7 +61,8 @@ def lib() -> ctypes.CDLL:
         L.kvs_static_scratch_bytes.restype = ctypes.c_size_t
         for name in ("kvs_round_plan", "kvs_workspace_size", "kvs_merge_layer", "kvs_compact",
                      "kvs_decode_attn", "kvs_window_stats", "kvs_profile_begin", "kvs_profile_end",
-                     "kvs_compact_static", "kvs_append_and_merge", "kvs_debug_set_wait"):
+                     "kvs_compact_static", "kvs_append_and_merge", "kvs_debug_set_wait", "kvs_adjacent_cosine",
+                     "kvs_workspace_size_per_head", "kvs_merge_layer_per_head", "kvs_decode_attn_per_head"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -207,6 +209,45 @@ def kvs_window_stats(params: kvs_params_t, K, V, counts, q_win, seq_len: Sequenc
                                   _ptr(mask), _ptr(o_win), _ptr(lse_win), _ptr(workspace),
                                   ctypes.c_size_t(workspace.numel() * workspace.element_size()),
                                   _ptr(status_dev), _stream()))
+
+
+def kvs_workspace_size_per_head(params: kvs_params_t, n_max: int, max_new: int = 0) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().kvs_workspace_size_per_head(ctypes.byref(params), n_max, max_new, ctypes.byref(out)))
+    return int(out.value)
+
+
+def kvs_merge_layer_per_head(params: kvs_params_t, K, V, counts, q_win, seq_len: Sequence[int],
+                             budget: Sequence[int], workspace, status_dev=None) -> List[int]:
+    """kvs_merge_layer with a length and a budget per (sequence, KV head): flat lists of B * Hkv
+    entries, index b * Hkv + h.  Returns new_len in the same order."""
+    U = params.batch * params.n_kv_heads
+    new_len = (ctypes.c_int32 * U)()
+    _check(lib().kvs_merge_layer_per_head(ctypes.byref(params), _ptr(K), _ptr(V), _ptr(counts), _ptr(q_win),
+                                          _i32(seq_len), _i32(budget), ctypes.c_int32(counts.shape[-1]),
+                                          new_len, _ptr(workspace),
+                                          ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+                                          _ptr(status_dev), _stream()))
+    return list(new_len)
+
+
+def kvs_decode_attn_per_head(params: kvs_params_t, q_new, K, V, counts, seq_len: Sequence[int], out,
+                             workspace, lse=None, status_dev=None) -> None:
+    n_new = q_new.shape[2]
+    _check(lib().kvs_decode_attn_per_head(ctypes.byref(params), _ptr(q_new), ctypes.c_int32(n_new), _ptr(K),
+                                          _ptr(V), _ptr(counts), _i32(seq_len),
+                                          ctypes.c_int32(counts.shape[-1]), _ptr(out), _ptr(lse),
+                                          _ptr(workspace),
+                                          ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+                                          _ptr(status_dev), _stream()))
+
+
+def kvs_adjacent_cosine(x, seq_len: Sequence[int], cos_out) -> None:
+    """cos_out[b,h,t] = cosine of rows t and t+1 of the bf16 tensor x [B,H,Nmax,128], t < seq_len[b]-1."""
+    B, H, Nmax, _ = x.shape
+    _check(lib().kvs_adjacent_cosine(_ptr(x), ctypes.c_int32(B), ctypes.c_int32(H), ctypes.c_int32(Nmax),
+                                     ctypes.c_int64(x.stride(0)), ctypes.c_int64(x.stride(1)),
+                                     ctypes.c_int64(x.stride(2)), _i32(seq_len), _ptr(cos_out), _stream()))
 
 
 def kvs_debug_set_wait(limit_us: int = 0, withhold: int = 0) -> None:

@@ -1,6 +1,7 @@
 // C ABI of libkvs.so: argument checks, the host round scheduler, the workspace layout and
 // the launch sequence of each entry point.  No device memory is allocated here and the
 // stream is never synchronised.
+#include <limits.h>
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
@@ -856,6 +857,83 @@ kvs_status_t kvs_window_stats(const kvs_params_t* p, const void* K, const void* 
     s = enqueue_round_stats(cc, view, q_win, tab, nmax_slots, mask != nullptr, A, N1, N12, cosv,
                             score, w, mask, o_win, lse_win);
     if (s != KVS_OK) return s;
+  }
+  return KVS_OK;
+}
+
+namespace {
+
+// Per-head lengths: every (sequence, KV head) becomes a sequence of its own with one KV head and
+// the G query heads of its group.  The caches, counts and queries keep their memory layout; only
+// the way it is indexed changes, which needs the head stride to tile the sequence stride.
+kvs_status_t remap_per_head(const kvs_params_t* p, kvs_params_t* q) {
+  kvs_status_t s = check_params(p);
+  if (s != KVS_OK) return s;
+  if ((int64_t)p->batch * p->n_kv_heads > INT32_MAX) return fail(KVS_ERR_UNSUPPORTED, "too many (sequence, head) units");
+  if (p->batch > 1 && (p->k_stride_b != p->k_stride_h * p->n_kv_heads || p->v_stride_b != p->v_stride_h * p->n_kv_heads))
+    return fail(KVS_ERR_UNSUPPORTED, "per-head lengths need stride_b == n_kv_heads * stride_h");
+  *q = *p;
+  q->batch = p->batch * p->n_kv_heads;
+  q->n_q_heads = p->n_q_heads / p->n_kv_heads;
+  q->n_kv_heads = 1;
+  q->k_stride_b = p->k_stride_h; q->v_stride_b = p->v_stride_h;
+  return KVS_OK;
+}
+
+}  // namespace
+
+kvs_status_t kvs_workspace_size_per_head(const kvs_params_t* p, int32_t n_max, int32_t max_new, size_t* bytes) {
+  kvs_params_t q;
+  kvs_status_t s = remap_per_head(p, &q);
+  if (s != KVS_OK) return s;
+  return kvs_workspace_size(&q, n_max, max_new, bytes);
+}
+
+kvs_status_t kvs_merge_layer_per_head(const kvs_params_t* p, void* K, void* V, int32_t* counts,
+                                      const void* q_win, const int32_t* seq_len, const int32_t* budget,
+                                      int32_t n_max, int32_t* new_len, void* workspace,
+                                      size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+  kvs_params_t q;
+  kvs_status_t s = remap_per_head(p, &q);
+  if (s != KVS_OK) return s;
+  return kvs_merge_layer(&q, K, V, counts, q_win, seq_len, budget, n_max, new_len, workspace, workspace_bytes,
+                         status_dev, cuda_stream);
+}
+
+kvs_status_t kvs_decode_attn_per_head(const kvs_params_t* p, const void* q_new, int32_t n_new, const void* K,
+                                      const void* V, const int32_t* counts, const int32_t* seq_len,
+                                      int32_t n_max, void* out, float* lse, void* workspace,
+                                      size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+  kvs_params_t q;
+  kvs_status_t s = remap_per_head(p, &q);
+  if (s != KVS_OK) return s;
+  return kvs_decode_attn(&q, q_new, n_new, K, V, counts, seq_len, n_max, out, lse, workspace, workspace_bytes,
+                         status_dev, cuda_stream);
+}
+
+kvs_status_t kvs_adjacent_cosine(const void* x, int32_t batch, int32_t n_heads, int32_t n_max,
+                                 int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                                 const int32_t* seq_len, float* cos_out, void* cuda_stream) {
+  if (!x || !seq_len || !cos_out) return fail(KVS_ERR_INVALID_ARG, "NULL pointer argument");
+  if (batch <= 0 || n_heads <= 0 || n_max <= 0) return fail(KVS_ERR_INVALID_ARG, "sizes must be positive");
+  if (n_heads > 65535) return fail(KVS_ERR_UNSUPPORTED, "more than 65535 heads");
+  if (!aligned16(x)) return fail(KVS_ERR_INVALID_ARG, "x must be 16-byte aligned");
+  const int64_t s[3] = {stride_b, stride_h, stride_t};
+  for (int i = 0; i < 3; ++i)
+    if (s[i] < 0 || (s[i] % 8)) return fail(KVS_ERR_INVALID_ARG, "strides must be non-negative multiples of 8 elements");
+  if (stride_t < KVS_D) return fail(KVS_ERR_INVALID_ARG, "row stride must be >= 128");
+  for (int b = 0; b < batch; ++b)
+    if (seq_len[b] < 0 || seq_len[b] > n_max) return fail(KVS_ERR_INVALID_ARG, "seq_len[%d] out of range", b);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  for (int b0 = 0; b0 < batch; b0 += KVS_SEQ_CHUNK) {
+    RoundTable tab;
+    tab.nseq = 0; tab.off = 0;
+    for (int b = b0; b < batch && tab.nseq < KVS_SEQ_CHUNK; ++b)
+      if (seq_len[b] >= 2) tab.s[tab.nseq++] = {seq_len[b], 0, 0, b};
+    if (tab.nseq == 0) continue;
+    CUDA_TRY(launch(KVS_K_MISC, st, [&] {
+      return kvs_launch_adjacent_cosine(x, stride_b, stride_h, stride_t, n_heads, n_max, cos_out, tab, st);
+    }));
   }
   return KVS_OK;
 }

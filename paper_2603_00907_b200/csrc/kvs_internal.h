@@ -25,7 +25,7 @@ enum KvsKernelKind {
   KVS_K_STATS = 2,     // Hessian statistics + cosine + score + weight
   KVS_K_SELECT = 3,    // exact R-smallest selection + tile prefix
   KVS_K_COMPACT = 4,   // merge + in-place compaction
-  KVS_K_MISC = 5,      // mask scan for kvs_compact, copies of diagnostics
+  KVS_K_MISC = 5,      // mask scan for kvs_compact, chunk append, similarity diagnostics
   KVS_K_COUNT = 6
 };
 
@@ -149,6 +149,9 @@ struct AppendArgs {
 };
 cudaError_t kvs_launch_append(const AppendArgs& a, const RoundTable& t, cudaStream_t st);
 cudaError_t kvs_launch_select(const SelectArgs& a, const RoundTable& t, cudaStream_t st);
+// Adjacent-row cosine of a bf16 tensor [B, H, n_max, 128] (element strides sb, sh, st); table entry n = rows in use.
+cudaError_t kvs_launch_adjacent_cosine(const void* x, int64_t sb, int64_t sh, int64_t st, int H, int n_max,
+                                       float* out, const RoundTable& t, cudaStream_t stream);
 cudaError_t kvs_launch_compact(const CompactArgs& a, const RoundTable& t, cudaStream_t st);
 
 // Runs a per-device set-up call (raising a kernel's dynamic shared-memory limit) once for every

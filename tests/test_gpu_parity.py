@@ -726,3 +726,86 @@ def test_merged_counts_statistics(kb):
     data["counts"][:] = rng.integers(1, 5, size=data["counts"].shape)
     _check_round_stats(kb, w, data["K"], data["V"], data["counts"], data["q_win"], list(w.seq_lens), 0)
     _check_round_stats(kb, w, data["K"], data["V"], data["counts"], data["q_win"], list(w.seq_lens), 1)
+
+
+def test_adjacent_cosine_of_queries_keys_and_values(kb):
+    """kvs_adjacent_cosine on the keys, values and (decode) queries of a ragged batch against the
+    oracle, on a strided view too; entries at and behind seq_len - 1 stay untouched.  The synthetic
+    keys are an AR(1) drift (homogeneous neighbours), values and queries are i.i.d."""
+    import torch
+    w = _small(seed=51, batch=3, n_q_heads=8, n_kv_heads=2, window=8, seq_lens=(700, 1, 333), budgets=(700, 1, 333),
+               n_decode=40)
+    data = wl.make_layer(w)
+    dev = tl.upload_layer(data)
+    B, Hkv, Nmax = w.batch, w.n_kv_heads, w.n_max
+    means = {}
+    for name, x, lens in (("K", dev["K"], list(w.seq_lens)), ("V", dev["V"], list(w.seq_lens)),
+                          ("Q", dev["q_new"], [40, 40, 40])):
+        out = torch.full(x.shape[:3], -7.0, dtype=torch.float32, device="cuda")
+        kb.kvs_adjacent_cosine(x, lens, out)
+        torch.cuda.synchronize()
+        g = out.cpu().numpy()
+        xb = tl.bits_of(x)
+        acc = []
+        for b in range(B):
+            for h in range(x.shape[1]):
+                ref = oc.adjacent_cosine(xb[b, h, :lens[b]])
+                assert np.max(np.abs(g[b, h, :len(ref)] - ref), initial=0.0) < 1e-6
+                assert np.all(g[b, h, len(ref):] == -7.0)
+                acc.append(ref)
+        means[name] = float(np.mean(np.concatenate(acc)))
+    assert means["K"] > 0.8 and abs(means["V"]) < 0.05 and abs(means["Q"]) < 0.1
+    # a strided view (row stride 160 elements)
+    xs = torch.zeros((B, Hkv, Nmax, 160), dtype=torch.bfloat16, device="cuda")[..., :128]
+    xs.copy_(dev["K"])
+    out = torch.zeros((B, Hkv, Nmax), dtype=torch.float32, device="cuda")
+    kb.kvs_adjacent_cosine(xs, list(w.seq_lens), out)
+    torch.cuda.synchronize()
+    ref = oc.adjacent_cosine(data["K"][2, 1, :333])
+    assert np.max(np.abs(out[2, 1, :332].cpu().numpy() - ref)) < 1e-6
+
+
+def test_per_head_budgets(kb):
+    """kvs_merge_layer_per_head / kvs_decode_attn_per_head: every (sequence, KV head) runs to its own
+    budget.  The same memory viewed as a batch of one-head sequences goes through the ordinary entry
+    points against the oracle (band flips followed); the per-head entry points must then give those
+    results bit for bit on the original layout."""
+    import torch
+    w = _small(seed=61, batch=2, n_q_heads=12, n_kv_heads=3, window=8, seq_lens=(600, 410), budgets=(1, 1), n_decode=2)
+    data = wl.make_layer(w)
+    B, Hkv, G, Nmax = w.batch, w.n_kv_heads, w.group, w.n_max
+    seq_len = [600, 600, 600, 410, 410, 410]
+    budget = [90, 600, 300, 64, 200, 51]
+    # (1) as a batch of B * Hkv one-head sequences through the ordinary calls, against the oracle
+    wu = w.scaled(batch=B * Hkv, n_q_heads=G, n_kv_heads=1, seq_lens=tuple(seq_len), budgets=tuple(budget))
+    du = {"K": data["K"].reshape(B * Hkv, 1, Nmax, 128), "V": data["V"].reshape(B * Hkv, 1, Nmax, 128),
+          "counts": data["counts"].reshape(B * Hkv, 1, Nmax), "q_win": data["q_win"].reshape(B * Hkv, G, w.window, 128),
+          "q_new": data["q_new"].reshape(B * Hkv, G, 2, 128)}
+    K_ref, V_ref, C_ref, len_ref, flips = full_pass_vs_oracle(kb, wu, du)
+    assert len_ref == [min(n, b) for n, b in zip(seq_len, budget)]
+    # (2) the per-head entry points on the original [B, Hkv, ...] layout
+    dev = tl.upload_layer(data)
+    p = kb.make_params(dev["K"], dev["V"], w.n_q_heads, w.window, sink=w.sink, round_frac=w.round_frac)
+    ws = torch.empty(kb.kvs_workspace_size_per_head(p, Nmax, 2), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    new_len = kb.kvs_merge_layer_per_head(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], seq_len, budget, ws,
+                                          status_dev=status)
+    out = torch.zeros((B, w.n_q_heads, 2, 128), dtype=torch.bfloat16, device="cuda")
+    kb.kvs_decode_attn_per_head(p, dev["q_new"], dev["K"], dev["V"], dev["counts"], new_len, out, ws)
+    torch.cuda.synchronize()
+    assert status.item() == 0 and new_len == len_ref
+    Kg, Vg, Cg, og = tl.bits_of(dev["K"]), tl.bits_of(dev["V"]), dev["counts"].cpu().numpy(), tl.bits_of(out)
+    for b in range(B):
+        for h in range(Hkv):
+            u, m = b * Hkv + h, new_len[b * Hkv + h]
+            assert np.array_equal(Kg[b, h, :m], K_ref[u, 0, :m]) and np.array_equal(Vg[b, h, :m], V_ref[u, 0, :m])
+            assert np.array_equal(Cg[b, h, :m], C_ref[u, 0, :m]) and int(Cg[b, h, :m].sum()) == seq_len[u]
+            ref, _ = oc.decode_attention(data["q_new"][b, h * G:(h + 1) * G], Kg[b, h, :m], Vg[b, h, :m], Cg[b, h, :m])
+            ok, mx, _, _ = tl.bf16_close(og[b, h * G:(h + 1) * G], oc.f64_to_bf16(ref))
+            assert ok, ((b, h), mx)
+    # a layout whose heads do not tile the sequence stride is refused
+    Kbad = torch.zeros((B, Hkv + 1, Nmax, 128), dtype=torch.bfloat16, device="cuda")[:, :Hkv]
+    pbad = kb.make_params(Kbad, Kbad, w.n_q_heads, w.window, sink=w.sink)
+    with pytest.raises(kb.KvsError) as e:
+        kb.kvs_merge_layer_per_head(pbad, Kbad, Kbad, dev["counts"], dev["q_win"], seq_len, budget, ws)
+    assert e.value.code == 2

@@ -618,3 +618,48 @@ def test_merge_unit_applies_the_exact_weight_to_the_left_key():
     assert np.max(far / (np.abs(want) * 2.0 ** -8)) > 3.0
     assert np.array_equal(V1[m], oc.f64_to_bf16(Vf[m] + Vf[m + 1]))
     assert np.array_equal(K1[m + 1:], Kb[m + 2:]) and np.array_equal(K1[:m], Kb[:m])
+
+
+# ------------------------------------------------------------------ Section 3.2: adjacent similarity
+def test_adjacent_cosine_closed_forms():
+    """Eq. cosine_raw on rows whose angles are known in closed form (all entries are small integers,
+    exact in bf16): (3,4)/(4,3) -> 24/25, orthogonal -> 0, a negative multiple -> -1, a positive
+    multiple -> 1, (1,1,1,1)/(1,1,0,0) -> 1/sqrt(2); the result does not depend on row scale."""
+    rows = np.zeros((7, 8))
+    rows[0, :2] = (3, 4)
+    rows[1, :2] = (4, 3)
+    rows[2, :2] = (-6, 8)            # orthogonal to (4, 3)
+    rows[3, :2] = (12, -16)          # -2 x the row before
+    rows[4, :2] = (48, -64)          # 4 x the row before
+    rows[5, :4] = (1, 1, 1, 1)
+    rows[6, :4] = (1, 1, 0, 0)
+    want = np.array([24 / 25, 0.0, -1.0, 1.0, (48 - 64) / (80 * 2), 1 / math.sqrt(2)])
+    got = oc.adjacent_cosine(oc.f64_to_bf16(rows))
+    assert np.allclose(got, want, atol=1e-15)
+    scaled = rows * np.array([1, 2, 0.5, 8, 0.25, 4, 16])[:, None]
+    assert np.allclose(oc.adjacent_cosine(oc.f64_to_bf16(scaled)), want, atol=1e-15)
+    assert oc.adjacent_cosine(oc.f64_to_bf16(rows[:1])).shape == (0,)
+    assert oc.adjacent_cosine(oc.f64_to_bf16(np.zeros((2, 8))))[0] == 0.0      # floored denominator
+
+
+def test_per_head_budgets_run_every_head_to_its_own_length():
+    """Non-uniform budgets: each (sequence, KV head) ends exactly at its own budget with all of its
+    tokens still counted; a head whose budget is not below its length is returned unchanged; a head
+    given the sequence-wide budget gives what the per-sequence call gives."""
+    r = np.random.default_rng(17)
+    B, Hkv, G, W, n, d, sink = 2, 3, 2, 4, 90, 8, 4
+    inputs = {"K": _rand_bf16((B, Hkv, n, d), r), "V": _rand_bf16((B, Hkv, n, d), r),
+              "counts": np.ones((B, Hkv, n), dtype=np.int64), "q_win": _rand_bf16((B, Hkv * G, W, d), r),
+              "seq_len": np.array([[90, 70, 90], [60, 90, 33]]), "budget": np.array([[40, 70, 25], [30, 61, 33]])}
+    out = oc.merge_layer(inputs, window=W, sink=sink)
+    for b in range(B):
+        for h in range(Hkv):
+            Kn, Vn, cn = out[(b, h)]
+            n_bh, bud = inputs["seq_len"][b, h], inputs["budget"][b, h]
+            assert Kn.shape[0] == min(n_bh, bud) and int(cn.sum()) == n_bh
+            if bud >= n_bh:
+                assert np.array_equal(Kn, inputs["K"][b, h, :n_bh])
+    same = dict(inputs, seq_len=np.array([90, 60]), budget=np.array([40, 30]))
+    ref = oc.merge_layer(same, window=W, sink=sink, heads=[0])
+    for b in range(B):
+        assert all(np.array_equal(x, y) for x, y in zip(out[(b, 0)], ref[(b, 0)]))
