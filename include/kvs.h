@@ -235,6 +235,33 @@ kvs_status_t kvs_window_stats(const kvs_params_t* params, const void* K, const v
                               size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
 
 /*
+ * The merge pass and its diagnostic export with EXACT merge weights from a supplied loss gradient
+ * [Section 4.2: g_ij = E^T c_ij, Eqs. c11_def-c12_def, H_gamma_rank1_rewrite,
+ * kstar_weight_final_rewrite].  Everything but the weight is as in kvs_merge_layer /
+ * kvs_window_stats (scores and the selection do not use E).
+ *   e_win        DEVICE bf16 [B,Hq,W,128] contiguous, 16-byte aligned: E = dL/do of every window
+ *                query (the backward pass the gradient-free form avoids); read only
+ *   weight_mode  1: w = (G11 + G12) / (G11 + 2 G12 + G22), G_ij = sum over the window queries of
+ *                   E_q^T c_ij  [Eq. kstar_weight_final_rewrite]
+ *                2: the same with the coupling dropped, w = G11 / (G11 + G22): the diagonal-Hessian
+ *                   merge the paper starts from  [Section 3.1, Eq. simplified_k]
+ *                A denominator that is not safely positive gives w = 1/2; w is clipped to [0, 1].
+ *   g_self       optional DEVICE fp32 [B,Hkv,Nmax]: sum over queries of E^T c_jj per candidate slot
+ *   g_pair       optional DEVICE fp32 [B,Hkv,Nmax/2]: sum over queries of E^T c_12 per candidate pair
+ */
+kvs_status_t kvs_merge_layer_exact(const kvs_params_t* params, void* K, void* V, int32_t* counts,
+                                   const void* q_win, const void* e_win, int32_t weight_mode,
+                                   const int32_t* seq_len, const int32_t* budget, int32_t n_max,
+                                   int32_t* new_len, void* workspace, size_t workspace_bytes,
+                                   int32_t* status_dev, void* cuda_stream);
+kvs_status_t kvs_window_stats_exact(const kvs_params_t* params, const void* K, const void* V,
+                                    const int32_t* counts, const void* q_win, const void* e_win,
+                                    int32_t weight_mode, const int32_t* seq_len, const int32_t* budget,
+                                    int32_t n_max, float* A, float* g_self, float* g_pair, float* cosv,
+                                    float* score, float* w, uint8_t* mask, void* workspace,
+                                    size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
+
+/*
  * Non-uniform budgets: the merge pass and the decode check with a length and a budget per
  * (sequence, KV head) instead of per sequence  [Section 6 (discussion): one compression ratio for
  * every layer and head is the method's stated limitation; the heads of a sequence may now end at

@@ -279,9 +279,9 @@ def exact_pair_sums(alpha: np.ndarray, o: np.ndarray, vbar: np.ndarray, E: np.nd
     """Scalar sensitivities of every candidate pair with a supplied loss gradient E [M, d_v] (one row
     per window query, E_q = dL/do_q): g_ij^(q) = E_q^T c_ij^(q) [Section 4.2, text before
     Eq. h_rank1_unified], summed over the window queries (the Hessian of the summed loss is the sum
-    of the per-query Hessians).  Returns G11, G22, G12 [P] and, for tolerances, the sum of the
-    absolute values of all terms that entered each pair."""
-    G11, G22, G12, Gabs = np.zeros(P), np.zeros(P), np.zeros(P), np.zeros(P)
+    of the per-query Hessians).  Returns G11, G22, G12 [P] and, for tolerances, Gabs [3, P]: the sums
+    of the absolute values of the terms of each."""
+    G11, G22, G12, Gabs = np.zeros(P), np.zeros(P), np.zeros(P), np.zeros((3, P))
     for p in range(P):
         j = off + 2 * p
         for q in range(alpha.shape[0]):
@@ -290,7 +290,7 @@ def exact_pair_sums(alpha: np.ndarray, o: np.ndarray, vbar: np.ndarray, E: np.nd
             G11[p] += g11
             G22[p] += g22
             G12[p] += g12
-            Gabs[p] += abs(g11) + abs(g22) + 2.0 * abs(g12)
+            Gabs[:, p] += (abs(g11), abs(g22), abs(g12))
     return G11, G22, G12, Gabs
 
 

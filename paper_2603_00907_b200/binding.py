@@ -24,7 +24,8 @@ EXPORTS = ["kvs_version", "kvs_last_error_string", "kvs_launch_count", "kvs_roun
            "kvs_window_stats", "kvs_profile_begin", "kvs_profile_end", "kvs_profile_kind_name",
            "kvs_compact_static", "kvs_static_scratch_bytes", "kvs_append_and_merge",
            "kvs_debug_set_wait", "kvs_adjacent_cosine",
-           "kvs_workspace_size_per_head", "kvs_merge_layer_per_head", "kvs_decode_attn_per_head"]
+           "kvs_workspace_size_per_head", "kvs_merge_layer_per_head", "kvs_decode_attn_per_head",
+           "kvs_merge_layer_exact", "kvs_window_stats_exact"]
 
 
 class KvsError(RuntimeError):
@@ -62,7 +63,8 @@ def lib() -> ctypes.CDLL:
         for name in ("kvs_round_plan", "kvs_workspace_size", "kvs_merge_layer", "kvs_compact",
                      "kvs_decode_attn", "kvs_window_stats", "kvs_profile_begin", "kvs_profile_end",
                      "kvs_compact_static", "kvs_append_and_merge", "kvs_debug_set_wait", "kvs_adjacent_cosine",
-                     "kvs_workspace_size_per_head", "kvs_merge_layer_per_head", "kvs_decode_attn_per_head"):
+                     "kvs_workspace_size_per_head", "kvs_merge_layer_per_head", "kvs_decode_attn_per_head",
+                     "kvs_merge_layer_exact", "kvs_window_stats_exact"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -209,6 +211,31 @@ def kvs_window_stats(params: kvs_params_t, K, V, counts, q_win, seq_len: Sequenc
                                   _ptr(mask), _ptr(o_win), _ptr(lse_win), _ptr(workspace),
                                   ctypes.c_size_t(workspace.numel() * workspace.element_size()),
                                   _ptr(status_dev), _stream()))
+
+
+def kvs_merge_layer_exact(params: kvs_params_t, K, V, counts, q_win, e_win, weight_mode: int,
+                          seq_len: Sequence[int], budget: Sequence[int], workspace, status_dev=None) -> List[int]:
+    """kvs_merge_layer with exact weights from the loss gradient rows e_win [B,Hq,W,128]
+    (weight_mode 1) or their diagonal-only form (2)."""
+    B = params.batch
+    new_len = (ctypes.c_int32 * B)()
+    _check(lib().kvs_merge_layer_exact(ctypes.byref(params), _ptr(K), _ptr(V), _ptr(counts), _ptr(q_win),
+                                       _ptr(e_win), ctypes.c_int32(weight_mode), _i32(seq_len), _i32(budget),
+                                       ctypes.c_int32(counts.shape[-1]), new_len, _ptr(workspace),
+                                       ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+                                       _ptr(status_dev), _stream()))
+    return list(new_len)
+
+
+def kvs_window_stats_exact(params: kvs_params_t, K, V, counts, q_win, e_win, weight_mode: int,
+                           seq_len: Sequence[int], budget: Sequence[int], workspace, *, A=None, g_self=None,
+                           g_pair=None, cosv=None, score=None, w=None, mask=None, status_dev=None) -> None:
+    _check(lib().kvs_window_stats_exact(ctypes.byref(params), _ptr(K), _ptr(V), _ptr(counts), _ptr(q_win),
+                                        _ptr(e_win), ctypes.c_int32(weight_mode), _i32(seq_len), _i32(budget),
+                                        ctypes.c_int32(counts.shape[-1]), _ptr(A), _ptr(g_self), _ptr(g_pair),
+                                        _ptr(cosv), _ptr(score), _ptr(w), _ptr(mask), _ptr(workspace),
+                                        ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+                                        _ptr(status_dev), _stream()))
 
 
 def kvs_workspace_size_per_head(params: kvs_params_t, n_max: int, max_new: int = 0) -> int:

@@ -286,7 +286,9 @@ struct Common {
   cudaStream_t st;
   int G, Mw;
   int32_t* status_dev;
-  CUtensorMap tmK, tmV, tmQ, tmOhi, tmOlo, tmKp, tmVp;
+  const void* e_win;         // supplied loss gradient rows [B,Hq,W,128] (exact weight modes), else NULL
+  int weight_mode;           // 0: summed norms; 1: exact with E; 2: exact without the coupling
+  CUtensorMap tmK, tmV, tmQ, tmOhi, tmOlo, tmKp, tmVp, tmE;
 };
 
 // Attention partials of the query rows behind `tmQ` (a [U, M, 128] view) over the caches in `view`.
@@ -332,6 +334,7 @@ kvs_status_t make_call_tmaps(Common* c, const void* K, const void* V, const void
             make_tmap(&c->tmOlo, c->ws + c->L.o_lo, 3, qd, qs, 128) &&
             make_tmap_pairs(&c->tmKp, K, n_max, p->n_kv_heads, p->batch, p->k_stride_t, p->k_stride_h, p->k_stride_b) &&
             make_tmap_pairs(&c->tmVp, V, n_max, p->n_kv_heads, p->batch, p->v_stride_t, p->v_stride_h, p->v_stride_b);
+  if (ok && c->e_win) ok = make_tmap(&c->tmE, c->e_win, 3, qd, qs, 128);
   if (!ok) return fail(KVS_ERR_CUDA, "cuTensorMapEncodeTiled failed or is unavailable");
   return KVS_OK;
 }
@@ -365,6 +368,7 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
   ca.qc2 = reinterpret_cast<float2*>(c.ws + c.L.qc2);
   ca.M_pad = (c.Mw + 127) / 128 * 128;
   ca.out_bf16 = nullptr; ca.lse_out = lse_out; ca.o_out = o_out;
+  ca.e = c.weight_mode ? static_cast<const __nv_bfloat16*>(c.e_win) : nullptr;
   CUDA_TRY(launch(KVS_K_COMBINE, c.st, [&] { return kvs_launch_combine(ca, tab, c.st); }));
 
   StatsTcArgs ta;
@@ -374,7 +378,7 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
   const int ntiles = (pmax + 127) / 128;               // tiles of 128 candidate pairs
   ta.splits = balanced_splits(ta.nqblk * ta.Hkv * tab.nseq, ntiles, &ta.tiles_per_split);
   ta.n_max = view.n_max; ta.pair_stride = c.L.pair_stride;
-  ta.scale_log2 = scale_log2; ta.score_mode = p->score_mode;
+  ta.scale_log2 = scale_log2; ta.score_mode = p->score_mode; ta.weight_mode = c.weight_mode;
   ta.counts = view.counts; ta.qc2 = ca.qc2; ta.M_pad = ca.M_pad;
   ta.pair_norms = reinterpret_cast<const float4*>(c.ws + c.L.norms); ta.norm_stride = c.L.pair_stride;
   ta.score = score_out ? score_out : reinterpret_cast<float*>(c.ws + c.L.score);
@@ -386,7 +390,7 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
   ta.status_dev = c.status_dev;
   ta.wait_us = g_wait_us.load(); ta.debug_stall = g_debug_stall.load();
   CUDA_TRY(launch(KVS_K_STATS, c.st, [&] {
-    return kvs_launch_stats_tc(ta, tab, c.tmKp, c.tmVp, c.tmQ, c.tmOhi, c.tmOlo, c.st);
+    return kvs_launch_stats_tc(ta, tab, c.tmKp, c.tmVp, c.tmQ, c.weight_mode ? c.tmE : c.tmOhi, c.tmOlo, c.st);
   }));
 
   if (do_select) {
@@ -424,6 +428,17 @@ kvs_status_t check_common(const kvs_params_t* p, const void* K, const void* V, c
   c->G = p->n_q_heads / p->n_kv_heads;
   c->Mw = c->G * p->window;
   c->status_dev = nullptr;
+  c->e_win = nullptr;
+  c->weight_mode = 0;
+  return KVS_OK;
+}
+
+// The exact weight modes take a loss gradient row per window query, laid out like q_win.
+kvs_status_t check_exact(const void* e_win, int weight_mode) {
+  if (weight_mode == 0) return KVS_OK;
+  if (weight_mode != 1 && weight_mode != 2) return fail(KVS_ERR_INVALID_ARG, "weight_mode must be 1 or 2");
+  if (!e_win) return fail(KVS_ERR_INVALID_ARG, "e_win is NULL");
+  if (!aligned16(e_win)) return fail(KVS_ERR_INVALID_ARG, "e_win must be 16-byte aligned");
   return KVS_OK;
 }
 
@@ -574,10 +589,13 @@ kvs_status_t merge_layer_impl(const kvs_params_t* p, void* K, void* V, int32_t* 
                               int32_t n_max, int32_t* new_len, void* workspace,
                               size_t workspace_bytes, int32_t* status_dev, void* cuda_stream,
                               const void* chunk_k, const void* chunk_v, int32_t chunk_len,
-                              const int32_t* cur_len) {
+                              const int32_t* cur_len, const void* e_win = nullptr, int weight_mode = 0) {
   Common c;
   kvs_status_t s = check_common(p, K, V, counts, seq_len, n_max, workspace, workspace_bytes, 0, &c, cuda_stream);
   if (s != KVS_OK) return s;
+  s = check_exact(e_win, weight_mode);
+  if (s != KVS_OK) return s;
+  c.e_win = e_win; c.weight_mode = weight_mode;
   if (!q_win || !budget || !new_len) return fail(KVS_ERR_INVALID_ARG, "NULL pointer argument");
   if (!aligned16(q_win)) return fail(KVS_ERR_INVALID_ARG, "q_win must be 16-byte aligned");
   const int B = p->batch;
@@ -670,6 +688,16 @@ kvs_status_t kvs_merge_layer(const kvs_params_t* p, void* K, void* V, int32_t* c
                              size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
   return merge_layer_impl(p, K, V, counts, q_win, seq_len, budget, n_max, new_len, workspace, workspace_bytes,
                           status_dev, cuda_stream, nullptr, nullptr, 0, nullptr);
+}
+
+kvs_status_t kvs_merge_layer_exact(const kvs_params_t* p, void* K, void* V, int32_t* counts,
+                                   const void* q_win, const void* e_win, int32_t weight_mode,
+                                   const int32_t* seq_len, const int32_t* budget, int32_t n_max,
+                                   int32_t* new_len, void* workspace, size_t workspace_bytes,
+                                   int32_t* status_dev, void* cuda_stream) {
+  if (weight_mode != 1 && weight_mode != 2) return fail(KVS_ERR_INVALID_ARG, "weight_mode must be 1 or 2");
+  return merge_layer_impl(p, K, V, counts, q_win, seq_len, budget, n_max, new_len, workspace, workspace_bytes,
+                          status_dev, cuda_stream, nullptr, nullptr, 0, nullptr, e_win, weight_mode);
 }
 
 kvs_status_t kvs_append_and_merge(const kvs_params_t* p, void* K, void* V, int32_t* counts,
@@ -807,21 +835,26 @@ kvs_status_t kvs_decode_attn(const kvs_params_t* p, const void* q_new, int32_t n
     ca.part_o = reinterpret_cast<float*>(c.ws + c.L.part_o);
     ca.qstat = nullptr; ca.qc2 = nullptr; ca.M_pad = 0; ca.o = nullptr; ca.o_hi = nullptr; ca.o_lo = nullptr;
     ca.out_bf16 = static_cast<__nv_bfloat16*>(out);
-    ca.lse_out = lse; ca.o_out = nullptr;
+    ca.lse_out = lse; ca.o_out = nullptr; ca.e = nullptr;
     CUDA_TRY(launch(KVS_K_COMBINE, c.st, [&] { return kvs_launch_combine(ca, tab, c.st); }));
   }
   return KVS_OK;
 }
 
-kvs_status_t kvs_window_stats(const kvs_params_t* p, const void* K, const void* V,
-                              const int32_t* counts, const void* q_win, const int32_t* seq_len,
-                              const int32_t* budget, int32_t n_max, float* A, float* N1, float* N12,
-                              float* cosv, float* score, float* w, uint8_t* mask, float* o_win,
-                              float* lse_win, void* workspace, size_t workspace_bytes,
-                              int32_t* status_dev, void* cuda_stream) {
+namespace {
+
+kvs_status_t window_stats_impl(const kvs_params_t* p, const void* K, const void* V,
+                               const int32_t* counts, const void* q_win, const int32_t* seq_len,
+                               const int32_t* budget, int32_t n_max, float* A, float* N1, float* N12,
+                               float* cosv, float* score, float* w, uint8_t* mask, float* o_win,
+                               float* lse_win, void* workspace, size_t workspace_bytes,
+                               int32_t* status_dev, void* cuda_stream, const void* e_win, int weight_mode) {
   Common c;
   kvs_status_t s = check_common(p, K, V, counts, seq_len, n_max, workspace, workspace_bytes, 0, &c, cuda_stream);
   if (s != KVS_OK) return s;
+  s = check_exact(e_win, weight_mode);
+  if (s != KVS_OK) return s;
+  c.e_win = e_win; c.weight_mode = weight_mode;
   if (!q_win || !budget) return fail(KVS_ERR_INVALID_ARG, "NULL pointer argument");
   const int B = p->batch;
   const int r = p->first_round;
@@ -859,6 +892,29 @@ kvs_status_t kvs_window_stats(const kvs_params_t* p, const void* K, const void* 
     if (s != KVS_OK) return s;
   }
   return KVS_OK;
+}
+
+}  // namespace
+
+kvs_status_t kvs_window_stats(const kvs_params_t* p, const void* K, const void* V,
+                              const int32_t* counts, const void* q_win, const int32_t* seq_len,
+                              const int32_t* budget, int32_t n_max, float* A, float* N1, float* N12,
+                              float* cosv, float* score, float* w, uint8_t* mask, float* o_win,
+                              float* lse_win, void* workspace, size_t workspace_bytes,
+                              int32_t* status_dev, void* cuda_stream) {
+  return window_stats_impl(p, K, V, counts, q_win, seq_len, budget, n_max, A, N1, N12, cosv, score, w, mask, o_win,
+                           lse_win, workspace, workspace_bytes, status_dev, cuda_stream, nullptr, 0);
+}
+
+kvs_status_t kvs_window_stats_exact(const kvs_params_t* p, const void* K, const void* V,
+                                    const int32_t* counts, const void* q_win, const void* e_win,
+                                    int32_t weight_mode, const int32_t* seq_len, const int32_t* budget,
+                                    int32_t n_max, float* A, float* g_self, float* g_pair, float* cosv,
+                                    float* score, float* w, uint8_t* mask, void* workspace,
+                                    size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+  if (weight_mode != 1 && weight_mode != 2) return fail(KVS_ERR_INVALID_ARG, "weight_mode must be 1 or 2");
+  return window_stats_impl(p, K, V, counts, q_win, seq_len, budget, n_max, A, g_self, g_pair, cosv, score, w, mask,
+                           nullptr, nullptr, workspace, workspace_bytes, status_dev, cuda_stream, e_win, weight_mode);
 }
 
 namespace {

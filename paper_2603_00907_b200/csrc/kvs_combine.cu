@@ -45,9 +45,18 @@ combine_partials(const CombineArgs a, const RoundTable tab) {
   for (int k = 16; k > 0; k >>= 1) on2 += __shfl_xor_sync(0xffffffffu, on2, k);
   const size_t row = (size_t)unit * a.M + m;
   const float lse = (mstar + log2f(Z)) * 0.6931471805599453f;
+  // with a supplied loss gradient the statistics need <E_q, o_q> in place of |o_q|^2
+  float qconst = on2;
+  if (a.e) {
+    const uint2 er = *reinterpret_cast<const uint2*>(a.e + row * KVS_D + 4 * lane);
+    float eo = fmaf(bf16lo(er.x), od.x, bf16hi(er.x) * od.y) + fmaf(bf16lo(er.y), od.z, bf16hi(er.y) * od.w);
+#pragma unroll
+    for (int k = 16; k > 0; k >>= 1) eo += __shfl_xor_sync(0xffffffffu, eo, k);
+    qconst = eo;
+  }
   if (lane == 0) {
     if (a.qstat) a.qstat[row] = make_float4(mstar, Z, on2, lse);
-    if (a.qc2) a.qc2[(size_t)unit * a.M_pad + m] = make_float2(-(mstar + log2f(Z)), on2);
+    if (a.qc2) a.qc2[(size_t)unit * a.M_pad + m] = make_float2(-(mstar + log2f(Z)), qconst);
     if (a.lse_out) a.lse_out[row] = lse;
   }
   const float v[4] = {od.x, od.y, od.z, od.w};

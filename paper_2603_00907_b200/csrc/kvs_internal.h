@@ -80,6 +80,7 @@ struct CombineArgs {
   __nv_bfloat16* out_bf16; // decode: [B, Hq, n_new, 128] == [U, M, 128] (may be NULL)
   float* lse_out;          // optional [U, M]
   float* o_out;            // optional diagnostic copy [U, M, 128]
+  const __nv_bfloat16* e;  // optional loss gradient rows [U, M, 128]: qc2.y then holds <E_q, o_q> instead of |o_q|^2
 };
 
 struct StatsTcArgs {
@@ -87,8 +88,9 @@ struct StatsTcArgs {
   int32_t n_max, pair_stride;
   float scale_log2;
   int32_t score_mode;
+  int32_t weight_mode;     // 0: summed norms (Eq. kstar_final); 1: exact, supplied E; 2: exact without the coupling
   const int32_t* counts;   // [U, n_max]
-  const float2* qc2;       // [U, M_pad]: (-(max + log2 Z), |o|^2)
+  const float2* qc2;       // [U, M_pad]: (-(max + log2 Z), |o|^2), or (-(max + log2 Z), <E, o>) with a supplied E
   int32_t M_pad;
   float* score;            // [U, pair_stride]
   float* w;
@@ -134,7 +136,8 @@ struct CompactArgs {
 // ----------------------------------------------------------------------------- launchers
 // Each returns the cudaError_t of its launch.  `nseq_units` = table.nseq * Hkv.
 cudaError_t kvs_launch_combine(const CombineArgs& a, const RoundTable& t, cudaStream_t st);
-// tmKp / tmVp: 5-D pair views [128, parity, slot / 2, head, sequence] of the caches
+// tmKp / tmVp: 5-D pair views [128, parity, slot / 2, head, sequence] of the caches; with
+// weight_mode != 0, tmOhi is the map of the supplied gradient rows E and tmOlo is not used
 cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const CUtensorMap& tmKp,
                                 const CUtensorMap& tmVp, const CUtensorMap& tmQ, const CUtensorMap& tmOhi,
                                 const CUtensorMap& tmOlo, cudaStream_t st);

@@ -18,6 +18,10 @@
 // every pair come from the attention pass that precedes this kernel (it streams the same rows).
 // With one query block the kernel forms score and the merge weight of Eq. kstar_final itself;
 // with several, each block writes its partial sums and a small kernel adds them in block order.
+// A second instantiation serves the exact weight modes: a supplied loss gradient E (one row per
+// window query) takes the place of the attention output in the T products, and the statistics
+// warps sum the signed scalars g_ij = E^T c_ij instead of the norms [Section 4.2, text before
+// Eq. h_rank1_unified; Eq. kstar_weight_final_rewrite].
 // Every synchronisation is an mbarrier with a bounded wait, so a warp that gives up can never
 // leave another one stuck.
 #include "kvs_internal.h"
@@ -77,19 +81,35 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
   for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// Score and left-key weight of a pair from its sums over the window queries.  Weight modes:
+//   0: N1j / N1p / N12 are summed norms; w = (N1j - N12) / (N1j - 2 N12 + N1p)            [Eq. kstar_final]
+//   1: they are the signed sums G11, G22, G12 of g_ij = E^T c_ij; w = (G11 + G12) / (G11 + 2 G12 + G22)
+//                                                                            [Eq. kstar_weight_final_rewrite]
+//   2: as 1 with the coupling dropped, w = G11 / (G11 + G22)                              [Eq. simplified_k]
+// A denominator that is not safely positive gives 1/2; the weight is clipped to [0, 1].
 __device__ __forceinline__ void finalize_pair(const StatsTcArgs& a, size_t pi, float Aj, float Ap, float N1j,
                                               float N1p, float N12, float cosv) {
   const float mass = Aj + Ap;
   const float score = (a.score_mode == 0) ? mass * fmaxf(0.f, 1.f - cosv) : mass;
-  const float D = N1j - 2.f * N12 + N1p;
   float w = 0.5f;
-  if (D > 1e-6f * (N1j + N1p) && D < INFINITY) w = fminf(1.f, fmaxf(0.f, (N1j - N12) / D));
+  if (a.weight_mode == 0) {
+    const float D = N1j - 2.f * N12 + N1p;
+    if (D > 1e-6f * (N1j + N1p) && D < INFINITY) w = fminf(1.f, fmaxf(0.f, (N1j - N12) / D));
+  } else {
+    const float g12 = (a.weight_mode == 2) ? 0.f : N12;
+    const float gamma = N1j + 2.f * g12 + N1p;
+    if (gamma > 1e-6f * (fabsf(N1j) + fabsf(N1p)) && gamma < INFINITY) w = fminf(1.f, fmaxf(0.f, (N1j + g12) / gamma));
+  }
   a.score[pi] = fabsf(score);
   a.w[pi] = w;
   if (a.N12) a.N12[pi] = N12;
   if (a.cosv) a.cosv[pi] = cosv;
 }
 
+// kExact: a loss gradient E (one bf16 row per window query) takes the place of the attention
+// output: T = Vsum E^T needs one product chain instead of two, and the statistics warps form the
+// signed sums of g_ij = E^T c_ij instead of the norms (no square roots).
+template <bool kExact>
 __global__ void __launch_bounds__(kThreads, 1)
 hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constant__ CUtensorMap tmKp,
                  const __grid_constant__ CUtensorMap tmVp, const __grid_constant__ CUtensorMap tmQ,
@@ -157,11 +177,11 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
     // ================================================================ TMA producer
     if (lane == 0) {
       prefetch_tmap(&tmKp); prefetch_tmap(&tmVp); prefetch_tmap(&tmQ); prefetch_tmap(&tmOhi); prefetch_tmap(&tmOlo);
-      mbar_expect_tx(&misc->qfull, 3 * kOperand);
+      mbar_expect_tx(&misc->qfull, (kExact ? 2 : 3) * kOperand);
       for (int hf = 0; hf < 2; ++hf) {
         tma_load_3d(smem + kSmemQ + hf * kHalf, &tmQ, &misc->qfull, hf * 64, qblk * kQB, unit);
         tma_load_3d(smem + kSmemOhi + hf * kHalf, &tmOhi, &misc->qfull, hf * 64, qblk * kQB, unit);
-        tma_load_3d(smem + kSmemOlo + hf * kHalf, &tmOlo, &misc->qfull, hf * 64, qblk * kQB, unit);
+        if (!kExact) tma_load_3d(smem + kSmemOlo + hf * kHalf, &tmOlo, &misc->qfull, hf * 64, qblk * kQB, unit);
       }
       // one thread streams both operands; every tile is first requested into L2 one tile ahead,
       // so that the load that fills the (single) stage finds it there
@@ -247,15 +267,16 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
           }
           if (hq == nh - 1) tc_commit(&misc->kfree);
           if (hq == 0 && !mbar_wait(&misc->vfull, li & 1, abort_flag)) { ok = false; break; }
+          constexpr int kTSteps = kExact ? 8 : 16;           // E is one bf16 term, o is two
 #pragma unroll
-          for (int kk = 0; kk < 16; ++kk) {
+          for (int kk = 0; kk < kTSteps; ++kk) {
             const uint32_t o = (((kk & 7) >> 2) * kHalf + (kk & 3) * 32) >> 4;
             const uint32_t ob = (kk < 8 ? oh : ol) + o;
             if (kk == 0) umma_ss<false>(d0 + 128, vl_lo, dhi, ob, dhi, idesc);
             else umma_ss<true>(d0 + 128, vl_lo + o, dhi, ob, dhi, idesc);
           }
 #pragma unroll
-          for (int kk = 0; kk < 16; ++kk) {
+          for (int kk = 0; kk < kTSteps; ++kk) {
             const uint32_t o = (((kk & 7) >> 2) * kHalf + (kk & 3) * 32) >> 4;
             const uint32_t ob = (kk < 8 ? oh : ol) + o;
             if (kk == 0) umma_ss<false>(d0 + 192, vr_lo, dhi, ob, dhi, idesc);
@@ -330,15 +351,27 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
             const float br = fast_exp2(fmaf(buf[b][1][i], a.scale_log2, ncq));
             sAl += bl;
             sAr += br;
-            const float gl = bl * fabsf(fmaf(bl, n2cl, 1.f));              // beta |1 - 2 alpha|
-            const float gr = br * fabsf(fmaf(br, n2cr, 1.f));
-            const float dl = fmaf(buf[b][2][i], n2il, r2l + hq2);          // |vbar_l - o|^2
-            const float dr = fmaf(buf[b][3][i], n2ir, r2r + hq2);
-            sN1l = fmaf(gl, fast_sqrt(fabsf(dl)), sN1l);
-            sN1r = fmaf(gr, fast_sqrt(fabsf(dr)), sN1r);
-            const float u = fmaf(buf[b][2][i], icl, buf[b][3][i] * icr) - hq2;   // <vbar_l + vbar_r, o> - |o|^2
-            const float d12 = fmaf(u, -4.f, pc);                           // |vbar_l + vbar_r - 2 o|^2
-            sN12 = fmaf(bl * br, fast_sqrt(fabsf(d12)), sN12);
+            if constexpr (kExact) {
+              // g11 = alpha (1 - 2 alpha) E^T (vbar_l - o), g12 = -alpha_l alpha_r E^T (vbar_l + vbar_r - 2 o);
+              // hq2 holds <E_q, o_q> here (the sign of g12 is applied after the loop)
+              const float gl = bl * fmaf(bl, n2cl, 1.f);                   // beta (1 - 2 alpha)
+              const float gr = br * fmaf(br, n2cr, 1.f);
+              const float hl = fmaf(buf[b][2][i], icl, -hq2);              // E^T (vbar_l - o)
+              const float hr = fmaf(buf[b][3][i], icr, -hq2);
+              sN1l = fmaf(gl, hl, sN1l);
+              sN1r = fmaf(gr, hr, sN1r);
+              sN12 = fmaf(bl * br, hl + hr, sN12);
+            } else {
+              const float gl = bl * fabsf(fmaf(bl, n2cl, 1.f));            // beta |1 - 2 alpha|
+              const float gr = br * fabsf(fmaf(br, n2cr, 1.f));
+              const float dl = fmaf(buf[b][2][i], n2il, r2l + hq2);        // |vbar_l - o|^2
+              const float dr = fmaf(buf[b][3][i], n2ir, r2r + hq2);
+              sN1l = fmaf(gl, fast_sqrt(fabsf(dl)), sN1l);
+              sN1r = fmaf(gr, fast_sqrt(fabsf(dr)), sN1r);
+              const float u = fmaf(buf[b][2][i], icl, buf[b][3][i] * icr) - hq2;   // <vbar_l + vbar_r, o> - |o|^2
+              const float d12 = fmaf(u, -4.f, pc);                         // |vbar_l + vbar_r - 2 o|^2
+              sN12 = fmaf(bl * br, fast_sqrt(fabsf(d12)), sN12);
+            }
           }
         }
         tc_fence_before();
@@ -363,7 +396,7 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
         warp_arrive(&misc->xfree[quarter], lane);                          // the buffer may be rewritten
         const float Al = cl * sAl, Ar = cr * sAr;
         const float N1l = cl * sN1l, N1r = cr * sN1r;
-        const float N12 = cl * cr * sN12;
+        const float N12 = (kExact ? -1.f : 1.f) * cl * cr * sN12;
         if (pair_ok) {
           if (a.nqblk == 1) {
             const size_t pi = (size_t)unit * a.pair_stride + p;
@@ -423,11 +456,14 @@ cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const
                                 const CUtensorMap& tmOlo, cudaStream_t st) {
   static KvsPerDeviceOnce configured;
   cudaError_t ce = configured.run([] {
-    return cudaFuncSetAttribute(hessian_stats_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(hessian_stats_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(hessian_stats_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   });
   if (ce != cudaSuccess) return ce;
   dim3 grid(a.nqblk * a.splits, a.Hkv, t.nseq);
-  hessian_stats_tc<<<grid, kThreads, kSmemBytes, st>>>(a, t, tmKp, tmVp, tmQ, tmOhi, tmOlo);
+  if (a.weight_mode == 0) hessian_stats_tc<false><<<grid, kThreads, kSmemBytes, st>>>(a, t, tmKp, tmVp, tmQ, tmOhi, tmOlo);
+  else hessian_stats_tc<true><<<grid, kThreads, kSmemBytes, st>>>(a, t, tmKp, tmVp, tmQ, tmOhi, tmOlo);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess || a.nqblk == 1) return e;
   int pmax = 0;

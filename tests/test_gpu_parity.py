@@ -327,12 +327,13 @@ def test_compact_one_cta_per_unit_and_strided_rows(kb):
             n_list = got
 
 
-def full_pass_vs_oracle(kb, w, data, units=None, seq_len=None, budgets=None):
+def full_pass_vs_oracle(kb, w, data, units=None, seq_len=None, budgets=None, exact=None):
     """The whole pass in one call; the same pass as single-round calls (it must equal their
     composition bit for bit); and, for the (sequence, KV head) `units` (all when None), the oracle
     that follows the GPU's near-cutoff choices: every deviation of the GPU's mask from the oracle's
     own must lie in the cutoff band, counts must be identical and K / value sums within the bf16
-    tolerance.  Returns the merged caches (numpy) and the number of band flips followed."""
+    tolerance.  `exact` = (E bits [B,Hq,W,128], weight_mode) runs the exact-weight variant.
+    Returns the merged caches (numpy) and the number of band flips followed."""
     import torch
     B, Hkv, Nmax = data["K"].shape[:3]
     G = w.group
@@ -342,11 +343,20 @@ def full_pass_vs_oracle(kb, w, data, units=None, seq_len=None, budgets=None):
              for n, bud in zip(seq_len, budgets)]
     rounds = max(len(pl) for pl in plans)
 
+    if exact is None:
+        merge = lambda pp, d, lens, buds, wsp, **kw: kb.kvs_merge_layer(pp, d["K"], d["V"], d["counts"], d["q_win"],
+                                                                        lens, buds, wsp, **kw)
+        okw = {}
+    else:
+        e_dev = tl.to_dev_bf16(exact[0])
+        merge = lambda pp, d, lens, buds, wsp, **kw: kb.kvs_merge_layer_exact(pp, d["K"], d["V"], d["counts"], d["q_win"],
+                                                                              e_dev, exact[1], lens, buds, wsp, **kw)
+        okw = {"weight_mode": exact[1]}
+
     # (1) full pass in one call
     dev, p, ws = _setup(kb, w, data)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    new_len = kb.kvs_merge_layer(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], seq_len, budgets, ws,
-                                 status_dev=status)
+    new_len = merge(p, dev, seq_len, budgets, ws, status_dev=status)
     torch.cuda.synchronize()
     assert status.item() == 0 and new_len == [min(n, b) for n, b in zip(seq_len, budgets)]
     K_full, V_full, C_full = tl.bits_of(dev["K"]), tl.bits_of(dev["V"]), dev["counts"].cpu().numpy()
@@ -363,8 +373,7 @@ def full_pass_vs_oracle(kb, w, data, units=None, seq_len=None, budgets=None):
         kb.kvs_window_stats(pr, dev2["K"], dev2["V"], dev2["counts"], dev2["q_win"], n_list, budgets, ws2, mask=mask)
         step_budget = [plans[b][r][0] - plans[b][r][3] if r < len(plans[b]) else min(seq_len[b], budgets[b])
                        for b in range(B)]
-        n_list = kb.kvs_merge_layer(pr, dev2["K"], dev2["V"], dev2["counts"], dev2["q_win"], n_list,
-                                    step_budget, ws2)
+        n_list = merge(pr, dev2, n_list, step_budget, ws2)
         gpu_masks.append(mask.cpu().numpy() if units is None else
                          {(b, h): mask[b, h].cpu().numpy() for (b, h) in units})
     torch.cuda.synchronize()
@@ -388,8 +397,17 @@ def full_pass_vs_oracle(kb, w, data, units=None, seq_len=None, budgets=None):
         trace = []
         Ko, Vo, Co = oc.merge_unit(data["K"][b, h, :n0], data["V"][b, h, :n0],
                                    data["counts"][b, h, :n0], data["q_win"][b, h * G:(h + 1) * G],
-                                   budgets[b], forced_masks=forced, trace=trace, **_oracle_kwargs(w))
+                                   budgets[b], forced_masks=forced, trace=trace,
+                                   E_bits=None if exact is None else exact[0][b, h * G:(h + 1) * G],
+                                   **okw, **_oracle_kwargs(w))
         for r, st in enumerate(trace):
+            if exact is not None:
+                # the comparison of the merged rows presumes that no merged pair sits at the guard of
+                # its denominator (there 1/2 and a clipped ratio are both within rounding)
+                g12 = st["G12"] if exact[1] == 1 else 0.0
+                gam = st["G11"] + 2.0 * g12 + st["G22"]
+                cond = np.abs(gam) / np.maximum(st["Gabs"][0] + st["Gabs"][1] + 2.0 * st["Gabs"][2], 1e-300)
+                assert cond[forced[r] != 0].min() > 5e-4, "a merged pair is ill conditioned: pick another seed"
             ok, nm, nout = tl.mask_band_ok(forced[r], st["mask"], st["score"], st["R"])
             assert ok, f"unit {(b, h)} round {r}: {nm} mask mismatches, {nout} outside the band"
             flips += nm
@@ -809,3 +827,65 @@ def test_per_head_budgets(kb):
     with pytest.raises(kb.KvsError) as e:
         kb.kvs_merge_layer_per_head(pbad, Kbad, Kbad, dev["counts"], dev["q_win"], seq_len, budget, ws)
     assert e.value.code == 2
+
+
+def test_exact_weights_with_a_supplied_gradient(kb):
+    """kvs_window_stats_exact / kvs_merge_layer_exact: the signed sums G_ij = sum_q E_q^T c_ij and the
+    weights of both exact modes against the oracle (errors measured against the sum of the absolute
+    terms, since the signed sums cancel), merged counts in the statistics, then the whole pass of a
+    small cache with exact weights against the oracle."""
+    import torch
+    w = _small(seed=71, batch=2, n_q_heads=8, n_kv_heads=2, window=40, seq_lens=(900, 517), budgets=(300, 170))
+    data = wl.make_layer(w)
+    rng = np.random.default_rng(71)
+    data["counts"][:] = rng.integers(1, 4, size=data["counts"].shape)
+    E = wl.f32_to_bf16_bits(rng.standard_normal(data["q_win"].shape).astype(np.float32))
+    dev, p, ws = _setup(kb, w, data)
+    e_dev = tl.to_dev_bf16(E)
+    B, Hkv, Nmax, G = w.batch, w.n_kv_heads, w.n_max, w.group
+    f32 = dict(dtype=torch.float32, device="cuda")
+    for r in (0, 1):
+        pr = kb.make_params(dev["K"], dev["V"], w.n_q_heads, w.window, sink=w.sink, first_round=r)
+        for mode in (1, 2):
+            A, gs = torch.zeros((B, Hkv, Nmax), **f32), torch.zeros((B, Hkv, Nmax), **f32)
+            gp, wg, sc = (torch.zeros((B, Hkv, Nmax // 2), **f32) for _ in range(3))
+            mask = torch.zeros((B, Hkv, Nmax // 2), dtype=torch.uint8, device="cuda")
+            kb.kvs_window_stats_exact(pr, dev["K"], dev["V"], dev["counts"], dev["q_win"], e_dev, mode,
+                                      list(w.seq_lens), list(w.budgets), ws, A=A, g_self=gs, g_pair=gp, score=sc,
+                                      w=wg, mask=mask)
+            torch.cuda.synchronize()
+            n_ratio = 0
+            for b in range(B):
+                n = w.seq_lens[b]
+                for h in range(Hkv):
+                    st = oc.round_stats(data["K"][b, h, :n], data["V"][b, h, :n], data["counts"][b, h, :n].astype(np.int64),
+                                        data["q_win"][b, h * G:(h + 1) * G], w.budgets[b], r, weight_mode=mode,
+                                        E_bits=E[b, h * G:(h + 1) * G], **_oracle_kwargs(w))
+                    off, P = st["off"], st["P"]
+                    g11, g22 = gs[b, h, off:off + 2 * P:2].cpu().numpy(), gs[b, h, off + 1:off + 2 * P:2].cpu().numpy()
+                    g12 = gp[b, h, :P].cpu().numpy()
+                    ab = st["Gabs"]
+                    assert np.all(np.abs(g11 - st["G11"]) <= tl.STAT_RTOL * ab[0] + 1e-37)
+                    assert np.all(np.abs(g22 - st["G22"]) <= tl.STAT_RTOL * ab[1] + 1e-37)
+                    assert np.all(np.abs(g12 - st["G12"]) <= tl.STAT_RTOL * ab[2] + 1e-37)
+                    ok, _, plain = tl.rel_close(A[b, h, off:off + 2 * P].cpu().numpy(), st["A"][off:off + 2 * P])
+                    assert ok, plain
+                    ok, nm, nout = tl.mask_band_ok(mask[b, h, :P].cpu().numpy(), st["mask"], st["score"], st["R"])
+                    assert ok, (nm, nout)
+                    c12 = st["G12"] if mode == 1 else 0.0
+                    gam = st["G11"] + 2.0 * c12 + st["G22"]
+                    tot = ab[0] + ab[1] + (2.0 * ab[2] if mode == 1 else 0.0)
+                    dw = np.abs(wg[b, h, :P].cpu().numpy() - st["w"])
+                    clear = np.abs(gam) > 1e-3 * tot            # away from the guard on the denominator
+                    bound = np.minimum(1.0, tl.STAT_RTOL * tot / np.maximum(np.abs(gam), 1e-300)) + 1e-7
+                    assert np.all(dw[clear] <= bound[clear]), float(np.max((dw / bound)[clear]))
+                    assert clear.mean() > 0.95
+                    n_ratio += int(np.sum((st["w"] > 0) & (st["w"] < 1) & (st["w"] != 0.5)))
+            assert n_ratio > 50
+    # the whole pass with exact weights on a fresh small cache
+    # (seed chosen so that no merged pair sits near the guard of its denominator)
+    w2 = _small(seed=76, batch=1, n_q_heads=8, n_kv_heads=2, window=8, seq_lens=(500,), budgets=(140,))
+    d2 = wl.make_layer(w2)
+    E2 = wl.f32_to_bf16_bits(np.random.default_rng(76).standard_normal(d2["q_win"].shape).astype(np.float32))
+    for mode in (1, 2):
+        *_, flips = full_pass_vs_oracle(kb, w2, d2, exact=(E2, mode))

@@ -663,3 +663,67 @@ def test_per_head_budgets_run_every_head_to_its_own_length():
     ref = oc.merge_layer(same, window=W, sink=sink, heads=[0])
     for b in range(B):
         assert all(np.array_equal(x, y) for x, y in zip(out[(b, 0)], ref[(b, 0)]))
+
+
+# ------------------------------------------------------------------ exact weights with a supplied E
+def test_exact_mode_sums_and_weights_against_finite_differences():
+    """weight_mode 1/2: G_ij of every candidate pair must be the sum over the window queries of the
+    scalar in front of q q^T / d_k in that query's Hessian block, taken here from finite differences
+    of textbook attention (causal: query i sees a truncated cache); the weight is
+    (G11 + G12) / (G11 + 2 G12 + G22) [Eq. kstar_weight_final_rewrite], G11 / (G11 + G22) without
+    the coupling [Eq. simplified_k], 1/2 where the denominator is not positive."""
+    r = np.random.default_rng(41)
+    n, d, dv, G, W, sink, recent = 11, 4, 3, 2, 2, 1, 2
+    Kb, Kf = _bf16_exact(r.standard_normal((n, d)) * 0.7)
+    Vb, Vf = _bf16_exact(r.standard_normal((n, dv)) * np.linspace(0.5, 2.5, n)[:, None])
+    Qb, Qf = _bf16_exact(r.standard_normal((G, W, d)))
+    Eb, Ef = _bf16_exact(r.standard_normal((G, W, dv)))
+    kw = dict(window=W, sink=sink, recent=recent, scale=1.0 / math.sqrt(d), causal=True, round_frac=0.5, score_mode=0)
+    st = oc.round_stats(Kb, Vb, np.ones(n, dtype=np.int64), Qb, n - 2, 0, weight_mode=1, E_bits=Eb, **kw)
+    sd = oc.round_stats(Kb, Vb, np.ones(n, dtype=np.int64), Qb, n - 2, 0, weight_mode=2, E_bits=Eb, **kw)
+    s0 = oc.round_stats(Kb, Vb, np.ones(n, dtype=np.int64), Qb, n - 2, 0, **kw)
+    off, P = st["off"], st["P"]
+    assert P == 4 and np.array_equal(st["mask"], s0["mask"]) and np.array_equal(st["score"], s0["score"])
+    kinds = set()
+    for p in range(P):
+        m = off + 2 * p
+        g11 = g22 = g12 = 0.0
+        for g in range(G):
+            for i in range(W):
+                vis = n - W + i + 1
+                g11 += _fd_scalar(Ef[g, i], Qf[g, i], Kf[:vis], Vf[:vis], m, m)
+                g22 += _fd_scalar(Ef[g, i], Qf[g, i], Kf[:vis], Vf[:vis], m + 1, m + 1)
+                g12 += _fd_scalar(Ef[g, i], Qf[g, i], Kf[:vis], Vf[:vis], m, m + 1)
+        assert abs(st["G11"][p] - g11) < 2e-6 and abs(st["G22"][p] - g22) < 2e-6 and abs(st["G12"][p] - g12) < 2e-6
+        for stx, gam, num in ((st, g11 + 2 * g12 + g22, g11 + g12), (sd, g11 + g22, g11)):
+            if gam > 1e-3 * (abs(g11) + abs(g22)):
+                want = min(1.0, max(0.0, num / gam))
+                kinds.add("ratio" if 0.0 < want < 1.0 else "clipped")
+                assert abs(stx["w"][p] - want) < 1e-4, (p, stx["w"][p], want)
+            elif gam < -1e-3 * (abs(g11) + abs(g22)):
+                kinds.add("guarded")
+                assert stx["w"][p] == 0.5
+    assert "ratio" in kinds and "guarded" in kinds
+    # E -> -E flips the sign of every g: pairs with a positive denominator become guarded and the others not
+    sn = oc.round_stats(Kb, Vb, np.ones(n, dtype=np.int64), Qb, n - 2, 0, weight_mode=1,
+                        E_bits=(Eb ^ np.uint16(0x8000)), **kw)
+    assert np.allclose(sn["G11"], -st["G11"]) and np.allclose(sn["G12"], -st["G12"])
+    gam = st["G11"] + 2 * st["G12"] + st["G22"]
+    big = np.abs(gam) > 1e-3 * (np.abs(st["G11"]) + np.abs(st["G22"]))
+    assert np.all((sn["w"][big] == 0.5) == (gam[big] > 0))
+
+
+def test_exact_mode_equals_norm_mode_in_the_aligned_case():
+    """d_v = 1, one-sided residuals, alpha < 1/2, E > 0: the cosines of Eq. cos_sign_relation_supp1
+    are exactly +1, +1, -1, so the exact weights and the gradient-free weights of Eq. kstar_final
+    coincide, through the whole pass of one round."""
+    n, d, Kb, Kf, qb, qf, Vb, Vf = _aligned_tiny_cache(23)
+    Eb = oc.f64_to_bf16(np.full((1, 1, 1), 1.5))
+    kw = dict(window=1, sink=1, recent=2, scale=1.0 / math.sqrt(d), causal=True, round_frac=0.5, score_mode=0)
+    a = oc.round_stats(Kb, Vb, np.ones(n, dtype=np.int64), qb, n - 1, 0, **kw)
+    b = oc.round_stats(Kb, Vb, np.ones(n, dtype=np.int64), qb, n - 1, 0, weight_mode=1, E_bits=Eb, **kw)
+    assert np.allclose(a["w"], b["w"], atol=1e-12) and np.ptp(a["w"]) > 0.05
+    K1, _, _ = oc.merge_unit(Kb, Vb, np.ones(n, dtype=np.int64), qb, n - 1, window=1, sink=1, recent=2, max_rounds=1)
+    K2, _, _ = oc.merge_unit(Kb, Vb, np.ones(n, dtype=np.int64), qb, n - 1, window=1, sink=1, recent=2, max_rounds=1,
+                             weight_mode=1, E_bits=Eb)
+    assert np.array_equal(K1, K2)
