@@ -110,12 +110,41 @@ def ncu_traffic_ratio(kind):
 
 
 def measured_peaks():
+    """HBM copy bandwidth (GB/s) and dense bf16 rates (TFLOP/s: burst, sustained) measured on this
+    pool's B200s; the recipe's earlier measurement if the file is absent."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def measure_sfu_peak(kb, torch, local):
+    """Special-function operations per second of this GPU, from the library's probe kernel (nothing
+    but ex2.approx / sqrt.approx) timed with CUDA events, with the SM clock sampled meanwhile."""
+    sink = torch.zeros(1, dtype=torch.float32, device="cuda")
+    blocks = 148 * 2
+    kb.kvs_probe_sfu(blocks, 2000, sink)                      # warm-up
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.15)
+    sampler.t_begin = time.perf_counter()
+    best = 0.0
+    t_end = time.perf_counter() + 0.6
+    while time.perf_counter() < t_end:
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        ops = kb.kvs_probe_sfu(blocks, 40000, sink)
+        b.record()
+        b.synchronize()
+        best = max(best, ops / (a.elapsed_time(b) * 1e-3))
+    sampler.t_end = time.perf_counter()
+    clk = sampler.stop()
+    return {"ops_per_s": best, "sm_mhz": clk.get("sm_mhz"), "samples": clk.get("samples"),
+            "how": "kvs_probe_sfu: 296 CTAs x 1024 threads x 640000 ex2.approx/sqrt.approx, best launch of 0.6 s"}
 
 
 def plan_rounds(w, oracle_free=True):
@@ -148,6 +177,43 @@ def algorithmic_bytes(w, n_layers):
         "select": pairs * (4 + 1),
         "merge_compact": slots * ROW_BYTES + kept * ROW_BYTES + pairs * 5,
     }, slots
+
+
+def work_counts(w, n_layers):
+    """Arithmetic that the method asks for per step, per kernel kind: tensor-core flops of its
+    contractions (the second figure adds the low-order bf16 terms that keep fp32 accuracy) and
+    special-function operations (one exp2 per (window query, slot) in either kernel; in the
+    statistics one square root per (query, slot) for N1 and one per (query, pair) for N12)."""
+    plans = plan_rounds(w)
+    M = w.group * w.window
+    units = w.n_kv_heads * n_layers
+    el_attn = sum(n for pl in plans for (n, _, _, _) in pl) * units * M
+    el_stats = sum(2 * P for pl in plans for (_, _, P, _) in pl) * units * M
+    return {
+        "attn_partials": {"elements": el_attn, "flops": 512 * el_attn, "flops_with_split": 768 * el_attn, "sfu_ops": 1.0 * el_attn},
+        "hessian_stats": {"elements": el_stats, "flops": 512 * el_stats, "flops_with_split": 768 * el_stats, "sfu_ops": 2.5 * el_stats},
+    }
+
+
+def rooflines(alg_bytes, work, ms, peaks, sfu_ops_per_s):
+    """The three floors of a piece of work that took `ms`: HBM (algorithmic bytes / measured copy
+    bandwidth), bf16 tensor (method flops / measured dense rate) and special function (operations /
+    measured probe rate).  The binding roofline is the one with the largest floor."""
+    out = {}
+    if alg_bytes:
+        f = alg_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+        out["hbm"] = {"floor_ms": f, "frac": f / ms, "achieved": alg_bytes / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    if work and work.get("flops"):
+        pk = peaks["bf16_tflops_sustained"]
+        f = work["flops"] / (pk * 1e12) * 1e3
+        out["tensor"] = {"floor_ms": f, "frac": f / ms, "achieved": work["flops"] / (ms * 1e-3) / 1e12, "peak": pk,
+                         "unit": "TFLOP/s", "frac_of_burst": work["flops"] / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                         "frac_with_split": work["flops_with_split"] / (pk * 1e12) * 1e3 / ms}
+    if work and work.get("sfu_ops") and sfu_ops_per_s:
+        f = work["sfu_ops"] / sfu_ops_per_s * 1e3
+        out["alu"] = {"floor_ms": f, "frac": f / ms, "achieved": work["sfu_ops"] / (ms * 1e-3) / 1e12,
+                      "peak": sfu_ops_per_s / 1e12, "unit": "Tops/s"}
+    return out
 
 
 def run_reference(args, w):
@@ -314,13 +380,46 @@ def run_stream(args):
     launches = kb.lib().kvs_launch_count() - l0
     assert status.item() == 0 and new_len == bud
     ms = total / args.steps
-    print(json.dumps({"metric": "stream_step_ms", "value": ms, "unit": "ms", "higher_is_better": False,
-                      "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup), "data": "synthetic",
-                      "dtype": "bf16", "gpu_launches": int(launches),
-                      "chunk_tokens_per_sec_per_layer": B * chunk / (ms * 1e-3),
-                      "config": {"workload": "streaming step, configs[1] head layout", "layers": L, "batch": B,
-                                 "n_kv_heads": Hkv, "budget": budget, "chunk": chunk, "window": W, "sink": w.sink,
-                                 "calls_per_step": "one kvs_append_and_merge over all layers"}}))
+    rec = {"metric": "stream_step_ms", "value": ms, "unit": "ms", "higher_is_better": False,
+           "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup), "data": "synthetic",
+           "dtype": "bf16", "gpu_launches": int(launches),
+           "chunk_tokens_per_sec_per_layer": B * chunk / (ms * 1e-3),
+           "config": {"workload": "streaming step, configs[1] head layout", "layers": L, "batch": B,
+                      "n_kv_heads": Hkv, "budget": budget, "chunk": chunk, "window": W, "sink": w.sink,
+                      "calls_per_step": "one kvs_append_and_merge over all layers"}}
+    del mK, mV, mC, wK, wV, wC, ws
+    torch.cuda.empty_cache()
+    return rec
+
+
+def weight_mode_report(kb, torch, w):
+    """How far the gradient-free weights of Eq. kstar_final are from the exact weights of
+    Eq. kstar_weight_final_rewrite, and those from the diagonal-only merge of Eq. simplified_k, on
+    round 0 of layer 0 with a synthetic loss gradient E ~ N(0, 1) per window query (with an i.i.d. E
+    the cosine relation that equates the two has no reason to hold: this measures the mechanism on
+    synthetic data, not the paper's claim about real models)."""
+    d = wl.make_layer(w, 0)
+    to = lambda x: torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).cuda().view(torch.bfloat16)
+    K, V, q = to(d["K"]), to(d["V"]), to(d["q_win"])
+    C = torch.from_numpy(d["counts"]).cuda()
+    rng = np.random.default_rng(123)
+    E = to(wl.f32_to_bf16_bits(rng.standard_normal(d["q_win"].shape).astype(np.float32)))
+    p = kb.make_params(K, V, w.n_q_heads, w.window, sink=w.sink, round_frac=w.round_frac)
+    ws = torch.empty(kb.kvs_workspace_size(p, w.n_max, 0), dtype=torch.uint8, device="cuda")
+    B, Hkv, Nmax = K.shape[:3]
+    ww = [torch.zeros((B, Hkv, Nmax // 2), dtype=torch.float32, device="cuda") for _ in range(3)]
+    lens, buds = list(w.seq_lens), list(w.budgets)
+    kb.kvs_window_stats(p, K, V, C, q, lens, buds, ws, w=ww[0])
+    kb.kvs_window_stats_exact(p, K, V, C, q, E, 1, lens, buds, ws, w=ww[1])
+    kb.kvs_window_stats_exact(p, K, V, C, q, E, 2, lens, buds, ws, w=ww[2])
+    torch.cuda.synchronize()
+    P = (w.seq_lens[0] - w.sink - w.window) // 2
+    wn, we, wd = (x[0, :, :P].float().cpu().numpy() for x in ww)
+    return {"pairs": int(wn.size), "E": "synthetic N(0,1), bf16", "round": 0, "layer": 0,
+            "mean_abs_norm_minus_exact": float(np.mean(np.abs(wn - we))),
+            "mean_abs_diag_minus_exact": float(np.mean(np.abs(wd - we))),
+            "exact_guarded_or_clipped_frac": float(np.mean((we == 0.5) | (we == 0.0) | (we == 1.0))),
+            "norm_weight_mean": float(wn.mean()), "norm_weight_std": float(wn.std())}
 
 
 def main():
@@ -335,6 +434,8 @@ def main():
                     help="one kvs_merge_layer call per layer instead of one call over all layers")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the streaming-step timing and the weight-mode comparison of the default line")
     ap.add_argument("--e2e-groups", type=int, default=4,
                     help="end-to-end leg: layer groups whose host copies overlap the other groups' kernels")
     ap.add_argument("--stream", action="store_true",
@@ -344,7 +445,7 @@ def main():
                     help="CPU only: exercise the multi-rank plumbing (gloo) on a small workload and exit")
     args = ap.parse_args()
     if args.stream:
-        run_stream(args)
+        print(json.dumps(run_stream(args)))
         return
     w = wl.config(args.config)
     if args.layers:
@@ -531,45 +632,41 @@ def main():
     prof = kb.kvs_profile_end()
     n_prof = min(args.steps, 2)
     alg, slot_rounds = algorithmic_bytes(w, L)
-    kinds = {k: v for k, v in prof.items() if v[1] > 0}
+    work = work_counts(w, L)
+    kinds = {k: v for k, v in prof.items() if v[1] > 0 and k != "misc"}
     top = max(kinds, key=lambda k: kinds[k][0])
-    peak, peak_src = measured_peaks()
-    top_ms, top_launches = kinds[top]
-    achieved = alg.get(top, 0) * n_prof / (top_ms * 1e-3) / 1e9 if top in alg else None
+    peaks = measured_peaks()
+    # special-function rate of this GPU, measured now, brought to the SM clock the step ran at
+    sfu = measure_sfu_peak(kb, torch, local)
+    clk_scale = (clocks["sm_mhz"] / sfu["sm_mhz"]) if (clocks.get("sm_mhz") and sfu.get("sm_mhz")) else 1.0
+    sfu_rate = sfu["ops_per_s"] * clk_scale
+    per_kernel = {}
+    for k, v in kinds.items():
+        ms_k = v[0] / n_prof
+        per_kernel[k] = {"ms_per_step": ms_k, "launches_per_step": v[1] // n_prof,
+                         "GBps": (alg[k] / (ms_k * 1e-3) / 1e9) if k in alg else None,
+                         "rooflines": rooflines(alg.get(k), work.get(k), ms_k, peaks, sfu_rate)}
+    # The dominant kernel against its three floors (all peaks measured on this machine: copy bandwidth,
+    # cuBLAS bf16 inside a long run, the special-function probe).  The headline is the roofline with
+    # the LARGEST floor: the one that bounds the kernel from below most tightly.
+    top_ms, top_launches = kinds[top][0] / n_prof, kinds[top][1] // n_prof
+    rl = per_kernel[top]["rooflines"]
+    bind = max(rl, key=lambda r: rl[r]["floor_ms"])
     ratio = ncu_traffic_ratio(top)
-    traffic = (ratio * alg.get(top, 0) * n_prof / top_launches) if (ratio and top in alg) else None
-    roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": (achieved / peak) if achieved else None, "traffic": traffic,
-                "peak_source": f"of {peak_src}",
-                "avg_launch_us": 1e3 * top_ms / top_launches,
-                "algorithmic_bytes_per_launch": alg.get(top, 0) * n_prof / top_launches,
-                "per_kernel": {k: {"ms_per_step": v[0] / n_prof, "launches_per_step": v[1] // n_prof,
-                                   "GBps": (alg[k] * n_prof / (v[0] * 1e-3) / 1e9) if k in alg else None}
-                               for k, v in kinds.items()}}
-
-    # The two attention-shaped kernels are, at this window size, limited by the 16-lane special
-    # function pipe rather than by HBM: report that roofline beside the HBM one.  Peak = 148 SMs x
-    # 16 lanes x the maximum SM clock; operations per (window query, slot) element: statistics
-    # 2.5 (one exp2, 1.5 square roots), attention 1.5 (one exp2, half a pack conversion).
-    plans = plan_rounds(w)
-    M = w.group * W
-    sfu_peak = 148 * 16 * (clocks.get("sm_max_mhz") or 1965.0) * 1e6
-    for kind, per_elem, count in (("hessian_stats", 2.5, lambda n, P: 2 * P), ("attn_partials", 1.5, lambda n, P: n)):
-        if kind in kinds:
-            elems = sum(count(n, P) for pl in plans for (n, _, P, _) in pl) * Hkv * L * M
-            ops_per_s = per_elem * elems / (kinds[kind][0] / n_prof * 1e-3)
-            roofline["per_kernel"][kind]["sfu"] = {"bound": "alu", "achieved": ops_per_s / 1e12, "peak": sfu_peak / 1e12,
-                                                   "unit": "Tops/s", "frac": ops_per_s / sfu_peak}
-    # The headline roofline is the one that binds the dominant kernel: where its special-function
-    # fraction exceeds its HBM fraction the kernel is reported as bound by plain arithmetic
-    # ("alu"), with the HBM figures kept beside it.
-    top_sfu = roofline["per_kernel"].get(top, {}).get("sfu")
-    if top_sfu and roofline["frac"] is not None and top_sfu["frac"] > roofline["frac"]:
-        roofline["hbm"] = {"achieved": roofline["achieved"], "peak": roofline["peak"], "unit": "GB/s",
-                           "frac": roofline["frac"], "peak_source": roofline["peak_source"]}
-        roofline.update({"bound": "alu", "achieved": top_sfu["achieved"], "peak": top_sfu["peak"],
-                         "unit": "Tops/s", "frac": top_sfu["frac"],
-                         "peak_source": "148 SMs x 16 special-function lanes x maximum SM clock"})
+    roofline = {"bound": bind, "kernel": top, "achieved": rl[bind]["achieved"], "peak": rl[bind]["peak"],
+                "unit": rl[bind]["unit"], "frac": rl[bind]["frac"],
+                "traffic": (ratio * alg[top] / top_launches) if (ratio and top in alg) else None,
+                "peak_source": ("of measured (special-function probe at %.0f MHz, scaled to the %.0f MHz of the timed region)"
+                                % (sfu["sm_mhz"] or 0, clocks.get("sm_mhz") or 0)) if bind == "alu" else f"of {peaks['source']}",
+                "binding": "largest of the three floors (hbm / tensor / alu)",
+                "floors_ms": {r: rl[r]["floor_ms"] for r in rl}, "fracs": {r: rl[r]["frac"] for r in rl},
+                "kernel_ms_per_step": top_ms, "avg_launch_us": 1e3 * top_ms / top_launches,
+                "algorithmic_bytes_per_launch": alg.get(top, 0) / top_launches,
+                "sfu_probe": sfu, "per_kernel": per_kernel}
+    # the whole step against the same three floors (sums over the kernels)
+    step_work = {key: sum(wk[key] for wk in work.values()) for key in ("flops", "flops_with_split", "sfu_ops")}
+    roofline["step"] = {"ms_per_step": ms_per_step,
+                        "rooflines": rooflines(sum(alg.values()), step_work, ms_per_step, peaks, sfu_rate)}
 
     # ---- end to end through the C ABI with host buffers
     e2e = None
@@ -603,6 +700,13 @@ def main():
                "sample": f"layer 0, sequence 0, KV head 0 only ({n0} tokens, all rounds): {t_unit:.1f} s; "
                          f"scaled to a layer of {Hkv} heads"}
 
+    stream_rec = weights_rec = None
+    if rank == 0 and world == 1 and not args.no_extras:
+        del mK, mV, mC, wK, wV, wC, ws
+        torch.cuda.empty_cache()
+        weights_rec = weight_mode_report(kb, torch, w)
+        stream_rec = run_stream(argparse.Namespace(layers=0, steps=20, warmup=3))
+
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -610,7 +714,9 @@ def main():
                 "config": workload_config(w, args), "clocks": clocks, "e2e": e2e,
                 "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
                 "removed_tokens_per_sec_per_layer":
-                    world * L * sum(n - b for n, b in zip(w.seq_lens, w.budgets)) / (ms_per_step * 1e-3)}
+                    world * L * sum(n - b for n, b in zip(w.seq_lens, w.budgets)) / (ms_per_step * 1e-3),
+                "stream_step_ms": stream_rec["value"] if stream_rec else None, "stream": stream_rec,
+                "weight_modes": weights_rec}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -315,6 +315,16 @@ kvs_status_t kvs_adjacent_cosine(const void* x, int32_t batch, int32_t n_heads, 
 kvs_status_t kvs_debug_set_wait(uint32_t limit_us, uint32_t withhold);
 
 /*
+ * Measurement aid: launches a kernel that executes nothing but special-function operations
+ * (ex2.approx and sqrt.approx, the operations that the softmax and the norms of Eqs. c11_def-c12_def
+ * cost per (query, slot)), `blocks` CTAs of 1024 threads with 16 * iters operations per thread, and
+ * returns the operation count through *ops.  Timed by the caller with CUDA events it gives the
+ * special-function rate of the GPU at hand, the denominator of that roofline in the benchmark.
+ *   sink_dev   DEVICE float[1] (never written in practice)
+ */
+kvs_status_t kvs_probe_sfu(int32_t blocks, int32_t iters, float* sink_dev, uint64_t* ops, void* cuda_stream);
+
+/*
  * Per-kernel device timing for benchmarks.  Between kvs_profile_begin() and
  * kvs_profile_end() every kernel launch of this library is bracketed by CUDA events on the
  * launching stream.  kvs_profile_end() synchronises those events and returns, for each

@@ -25,7 +25,7 @@ EXPORTS = ["kvs_version", "kvs_last_error_string", "kvs_launch_count", "kvs_roun
            "kvs_compact_static", "kvs_static_scratch_bytes", "kvs_append_and_merge",
            "kvs_debug_set_wait", "kvs_adjacent_cosine",
            "kvs_workspace_size_per_head", "kvs_merge_layer_per_head", "kvs_decode_attn_per_head",
-           "kvs_merge_layer_exact", "kvs_window_stats_exact"]
+           "kvs_merge_layer_exact", "kvs_window_stats_exact", "kvs_probe_sfu"]
 
 
 class KvsError(RuntimeError):
@@ -64,7 +64,7 @@ def lib() -> ctypes.CDLL:
                      "kvs_decode_attn", "kvs_window_stats", "kvs_profile_begin", "kvs_profile_end",
                      "kvs_compact_static", "kvs_append_and_merge", "kvs_debug_set_wait", "kvs_adjacent_cosine",
                      "kvs_workspace_size_per_head", "kvs_merge_layer_per_head", "kvs_decode_attn_per_head",
-                     "kvs_merge_layer_exact", "kvs_window_stats_exact"):
+                     "kvs_merge_layer_exact", "kvs_window_stats_exact", "kvs_probe_sfu"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -281,6 +281,13 @@ def kvs_debug_set_wait(limit_us: int = 0, withhold: int = 0) -> None:
     """Time limit of the device-side waits (0: the default of one second) and the test hook that
     makes one kind of wait run out (see kvs.h)."""
     _check(lib().kvs_debug_set_wait(ctypes.c_uint32(limit_us), ctypes.c_uint32(withhold)))
+
+
+def kvs_probe_sfu(blocks: int, iters: int, sink) -> int:
+    """Launch the special-function probe on the current stream; returns the operations it executes."""
+    ops = ctypes.c_uint64(0)
+    _check(lib().kvs_probe_sfu(ctypes.c_int32(blocks), ctypes.c_int32(iters), _ptr(sink), ctypes.byref(ops), _stream()))
+    return int(ops.value)
 
 
 def kvs_profile_begin() -> None:

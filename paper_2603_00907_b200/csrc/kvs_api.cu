@@ -994,6 +994,14 @@ kvs_status_t kvs_adjacent_cosine(const void* x, int32_t batch, int32_t n_heads, 
   return KVS_OK;
 }
 
+kvs_status_t kvs_probe_sfu(int32_t blocks, int32_t iters, float* sink_dev, uint64_t* ops, void* cuda_stream) {
+  if (blocks <= 0 || iters <= 0 || !sink_dev) return fail(KVS_ERR_INVALID_ARG, "bad probe argument");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  CUDA_TRY(launch(KVS_K_MISC, st, [&] { return kvs_launch_sfu_probe(blocks, iters, sink_dev, st); }));
+  if (ops) *ops = (uint64_t)blocks * 1024ull * 16ull * (uint64_t)iters;
+  return KVS_OK;
+}
+
 kvs_status_t kvs_profile_begin(void) {
   g_prof.on = true;
   g_prof.recs.clear();

@@ -174,6 +174,9 @@ struct KvsPerDeviceOnce {
   }
 };
 
+// Special-function probe: `blocks` CTAs of 1024 threads, 16 * iters operations per thread.
+cudaError_t kvs_launch_sfu_probe(int blocks, int iters, float* sink, cudaStream_t st);
+
 // ----------------------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
 __device__ __forceinline__ float bf16lo(uint32_t v) { return __uint_as_float(v << 16); }
