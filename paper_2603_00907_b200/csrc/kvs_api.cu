@@ -168,8 +168,7 @@ void round_plan(const kvs_params_t* p, int n, int budget, int r, int* off, int* 
 size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct WsLayout {
-  size_t part_ml, part_o, qstat, qc2, norms, o, o_hi, o_lo, score, w, mask, tile_prefix, partA, partN1, partN12, partCos,
-      sync, total;
+  size_t part_ml, part_o, qstat, qc2, norms, o, o_hi, o_lo, score, w, mask, tile_prefix, part4, part1, sync, total;
   int splits_max, M_max, pair_stride, tile_stride, counter_stride, nqblk_w, U;
   size_t sync_bytes;
 };
@@ -246,11 +245,10 @@ WsLayout make_layout(const kvs_params_t* p, int n_max, int max_new) {
   L.o_lo = o;    o += align_up((size_t)L.U * L.M_max * KVS_D * sizeof(__nv_bfloat16));
   L.nqblk_w = (Mw + 127) / 128;
   L.counter_stride = n_max / 128 + 2;
-  const size_t nq = L.nqblk_w > 1 ? L.nqblk_w : 0;      // partial sums only with several query blocks
-  L.partA = o;   o += align_up((size_t)L.U * nq * n_max * sizeof(float));
-  L.partN1 = o;  o += align_up((size_t)L.U * nq * n_max * sizeof(float));
-  L.partN12 = o; o += align_up((size_t)L.U * nq * L.pair_stride * sizeof(float));
-  L.partCos = o; o += align_up((size_t)L.U * (nq ? 1 : 0) * L.pair_stride * sizeof(float));
+  // partial sums of every (query block, statistics group): five floats per candidate pair
+  const size_t nsub = (size_t)L.nqblk_w * KVS_STATS_GROUPS;
+  L.part4 = o;   o += align_up((size_t)L.U * nsub * L.pair_stride * sizeof(float4));
+  L.part1 = o;   o += align_up((size_t)L.U * nsub * L.pair_stride * sizeof(float));
   // tickets [KVS_MAX_ROUNDS][U], flags [U][tile_stride], tile counters [U][counter_stride];
   // zeroed once per call
   L.sync = o;
@@ -384,9 +382,8 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
   ta.score = score_out ? score_out : reinterpret_cast<float*>(c.ws + c.L.score);
   ta.w = w_out ? w_out : reinterpret_cast<float*>(c.ws + c.L.w);
   ta.A = A; ta.N1 = N1; ta.N12 = N12; ta.cosv = cosv;
-  ta.partA = reinterpret_cast<float*>(c.ws + c.L.partA);
-  ta.partN1 = reinterpret_cast<float*>(c.ws + c.L.partN1);
-  ta.partN12 = reinterpret_cast<float*>(c.ws + c.L.partN12);
+  ta.part4 = reinterpret_cast<float4*>(c.ws + c.L.part4);
+  ta.part1 = reinterpret_cast<float*>(c.ws + c.L.part1);
   ta.status_dev = c.status_dev;
   ta.wait_us = g_wait_us.load(); ta.debug_stall = g_debug_stall.load();
   CUDA_TRY(launch(KVS_K_STATS, c.st, [&] {

@@ -17,6 +17,7 @@
 #define KVS_MAX_ROUNDS 64
 #define KVS_CTILE 64              // slots per compaction tile (32 candidate pairs)
 #define KVS_SPIN_LIMIT (1 << 22)  // iterations of any device-side wait before it gives up
+#define KVS_STATS_GROUPS 3        // statistics groups per query block: each writes its own partial sums
 
 // ----------------------------------------------------------------------------- kernel kinds
 enum KvsKernelKind {
@@ -98,9 +99,8 @@ struct StatsTcArgs {
   float* N1;
   float* N12;              // optional [U, pair_stride]
   float* cosv;
-  float* partA;            // [U, nqblk, n_max] per-query-block partial sums
-  float* partN1;
-  float* partN12;          // [U, nqblk, pair_stride]
+  float4* part4;           // [U, nqblk * KVS_STATS_GROUPS, pair_stride]: partial (A_l, A_r, N1_l, N1_r) of a pair
+  float* part1;            // [U, nqblk * KVS_STATS_GROUPS, pair_stride]: partial N12
   const float4* pair_norms; // [U, norm_stride] from the attention pass
   int32_t norm_stride;
   int32_t* status_dev;

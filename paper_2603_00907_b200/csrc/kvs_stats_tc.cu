@@ -4,20 +4,23 @@
 // bf16 terms, stay in shared memory) and walks a range of tiles of 128 candidate pairs.
 // A 5-D view of the cache, [128, parity, slot/2, head, sequence], lets TMA bring the left
 // members and the right members of the 128 pairs as two separate row tiles, so that TMEM
-// lane p holds everything of pair p.  For each half of 64 queries one thread issues
+// lane p holds everything of pair p.  For each half of 64 queries
 //   S_l = K_l Q^T, S_r = K_r Q^T                    (logits, fp32 in TMEM)
 //   T_l = Vsum_l (O_hi + O_lo)^T, T_r likewise      (value/output inner products)
-// into one of two TMEM buffers; while the statistics warps reduce one half, the tensor
-// core fills the other.  Each statistics thread owns one pair and a share of the queries and
-// reduces, in registers and with no cross-lane traffic,
+// go into one of two TMEM buffers; while the statistics warps reduce one half, the tensor
+// core fills the other.  Two threads (in two warps) issue the products, one the chains of the
+// left members and one those of the right members: feeding the tensor pipe from one thread costs
+// about as much time per product as the product itself.  Each statistics thread owns one pair
+// and a share of the queries and reduces, in registers and with no cross-lane traffic,
 //   A_j   = sum_q alpha_qj
 //   N1_j  = sum_q alpha |1 - 2 alpha| |vbar_j - o_q|                    [Eqs. c11_def, c22_def]
 //   N12_p = sum_q alpha_j alpha_j+1 |vbar_j + vbar_j+1 - 2 o_q|         [Eq. c12_def]
 // with |vbar_j - o_q|^2 = |vbar_j|^2 - 2 T_jq / c_j + |o_q|^2.  The probability matrix never
 // leaves the SM.  The row norms |vbar|^2, |vbar_l + vbar_r|^2 and the adjacent-key cosine of
 // every pair come from the attention pass that precedes this kernel (it streams the same rows).
-// With one query block the kernel forms score and the merge weight of Eq. kstar_final itself;
-// with several, each block writes its partial sums and a small kernel adds them in block order.
+// Every (query block, statistics group) writes its five sums per pair as a partial; a small
+// kernel adds the partials in a fixed order and forms score and the merge weight of
+// Eq. kstar_final (deterministic, no atomics, no hand-over between warps inside the tile loop).
 // A second instantiation serves the exact weight modes: a supplied loss gradient E (one row per
 // window query) takes the place of the attention output in the T products, and the statistics
 // warps sum the signed scalars g_ij = E^T c_ij instead of the norms [Section 4.2, text before
@@ -39,24 +42,31 @@ constexpr int kOperand = 2 * kHalf;        // a [128 x 128] bf16 operand
 constexpr int kSmemQ = 0, kSmemOhi = kOperand, kSmemOlo = 2 * kOperand;
 constexpr int kSmemKl = 3 * kOperand, kSmemKr = 4 * kOperand, kSmemVl = 5 * kOperand, kSmemVr = 6 * kOperand;
 constexpr int kSmemMisc = 7 * kOperand;
-constexpr int kGroups = 2;                 // statistics groups: a group reduces 64 / kGroups queries of every half
-constexpr int kStatWarps = 4 * kGroups;    // (more warps did not pay: the tensor pipe, not their latency, sets the pace)
-constexpr int kQG = kQH / kGroups;         // queries of a half per group
-constexpr int kThreads = (2 + kStatWarps) * 32;   // warp 0: TMA, warp 1: MMA, warps 2-17: statistics
+constexpr int kGroups = KVS_STATS_GROUPS;  // statistics groups: a group reduces a share of the queries of every half
+constexpr int kChunk = 8;                  // queries per round of TMEM loads
+constexpr bool kDoubleBuffer = kGroups < 4;   // the next chunk's loads in flight while one chunk is reduced
+constexpr int kChunks = kQH / kChunk;      // chunks of a half, dealt out to the groups as evenly as they go
+constexpr int kStatWarps = 4 * kGroups;
+constexpr int kIssuers = 2;
+constexpr int kFirstStat = 1 + kIssuers;   // warp 0: TMA, warps 1-2: product issuers, then the statistics warps
+constexpr int kThreads = (kFirstStat + kStatWarps) * 32;
+static_assert(KVS_STATS_GROUPS == kGroups, "the launcher sizes the partials with KVS_STATS_GROUPS");
 
 struct Misc {
-  uint64_t kfull, vfull, kfree, vfree, tfull[2], tfree[2], qfull, xhand[kGroups - 1][4], xfree[4];
+  uint64_t kfull, vfull, kfree, vfree, tfull[2], tfree[2], qfull;
   uint32_t tmem_base;
   int abort_flag, wait_us;                 // (adjacent: the bounded waits read both through one pointer)
-  float xbuf[kPairs * 5];                  // partial sums of a pair on their way from the last group down to group 0
+  alignas(16) float2 qconst[kQB];          // per query of the block: (-(max + log2 Z), |o|^2 or <E, o>)
 };
 constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc);
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 
-// One lane polls, the warp follows.
+// One lane polls, the warp follows.  The statistics warps wait on the critical path of a tile
+// (the tensor core has usually just finished): they poll instead of letting the hardware suspend
+// them, whose wake-up costs several hundred cycles.
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int lane) {
   int ok = 1;
-  if (lane == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+  if (lane == 0) ok = mbar_wait(bar, parity, abort_flag, true) ? 1 : 0;
   return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 __device__ __forceinline__ void warp_arrive(uint64_t* bar, int lane) {
@@ -79,31 +89,6 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
       : "memory");
 #pragma unroll
   for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-// Score and left-key weight of a pair from its sums over the window queries.  Weight modes:
-//   0: N1j / N1p / N12 are summed norms; w = (N1j - N12) / (N1j - 2 N12 + N1p)            [Eq. kstar_final]
-//   1: they are the signed sums G11, G22, G12 of g_ij = E^T c_ij; w = (G11 + G12) / (G11 + 2 G12 + G22)
-//                                                                            [Eq. kstar_weight_final_rewrite]
-//   2: as 1 with the coupling dropped, w = G11 / (G11 + G22)                              [Eq. simplified_k]
-// A denominator that is not safely positive gives 1/2; the weight is clipped to [0, 1].
-__device__ __forceinline__ void finalize_pair(const StatsTcArgs& a, size_t pi, float Aj, float Ap, float N1j,
-                                              float N1p, float N12, float cosv) {
-  const float mass = Aj + Ap;
-  const float score = (a.score_mode == 0) ? mass * fmaxf(0.f, 1.f - cosv) : mass;
-  float w = 0.5f;
-  if (a.weight_mode == 0) {
-    const float D = N1j - 2.f * N12 + N1p;
-    if (D > 1e-6f * (N1j + N1p) && D < INFINITY) w = fminf(1.f, fmaxf(0.f, (N1j - N12) / D));
-  } else {
-    const float g12 = (a.weight_mode == 2) ? 0.f : N12;
-    const float gamma = N1j + 2.f * g12 + N1p;
-    if (gamma > 1e-6f * (fabsf(N1j) + fabsf(N1p)) && gamma < INFINITY) w = fminf(1.f, fmaxf(0.f, (N1j + g12) / gamma));
-  }
-  a.score[pi] = fabsf(score);
-  a.w[pi] = w;
-  if (a.N12) a.N12[pi] = N12;
-  if (a.cosv) a.cosv[pi] = cosv;
 }
 
 // kExact: a loss gradient E (one bf16 row per window query) takes the place of the attention
@@ -145,21 +130,19 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
     // T product: each operand is requested again as soon as its own buffer is free
     mbar_init(&misc->kfull, 1);
     mbar_init(&misc->vfull, 1);
-    mbar_init(&misc->kfree, 1);            // MMA commit
-    mbar_init(&misc->vfree, 1);            // MMA commit
+    mbar_init(&misc->kfree, kIssuers);     // the issuers' commits
+    mbar_init(&misc->vfree, kIssuers);
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&misc->tfull[s], 1);
+      mbar_init(&misc->tfull[s], kIssuers);
       mbar_init(&misc->tfree[s], kStatWarps);   // statistics warps
     }
     mbar_init(&misc->qfull, 1);
-    for (int q = 0; q < 4; ++q) {          // per TMEM lane quarter: one warp hands over to one warp
-      for (int g = 0; g < kGroups - 1; ++g) mbar_init(&misc->xhand[g][q], 1);
-      mbar_init(&misc->xfree[q], 1);
-    }
     misc->abort_flag = 0;
     misc->wait_us = (int)a.wait_us;
     mbar_fence_init();
   }
+  // the per-query constants of the block (the same for every tile): read from shared memory in the loop
+  if (threadIdx.x < kQB) misc->qconst[threadIdx.x] = a.qc2[(size_t)unit * a.M_pad + qblk * kQB + threadIdx.x];
   if (warp == 1) tmem_alloc(&misc->tmem_base, 512);
   tc_fence_before();
   __syncthreads();
@@ -234,36 +217,31 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
         if (vli > 0) mbar_drain(&misc->vfull, (vli - 1) & 1);
       }
     }
-  } else if (warp == 1) {
-    // ================================================================ MMA issuer
+  } else if (warp < kFirstStat) {
+    // ================================================================ product issuers
+    // warp 1 issues the chains of the left pair members (S_l, T_l), warp 2 those of the right ones
     if (lane == 0) {
-      // (one thread feeds the tensor pipe with 96 products per tile: descriptors are kept as a
-      // constant high word and low words that only need an addition per product)
+      const bool right = warp != 1;
+      // descriptors are kept as a constant high word and low words that only need an addition per product
       constexpr uint32_t idesc = idesc_bf16(kPairs, kQH);
       const uint32_t dhi = (uint32_t)(smem_desc_sw128(0, 16, 1024) >> 32);
       auto dlo = [&](int off_bytes) { return (uint32_t)smem_desc_sw128(smem_u32(smem + off_bytes), 16, 1024); };
       const uint32_t q_lo = dlo(kSmemQ), ohi_lo = dlo(kSmemOhi), olo_lo = dlo(kSmemOlo);
-      const uint32_t kl_lo = dlo(kSmemKl), kr_lo = dlo(kSmemKr), vl_lo = dlo(kSmemVl), vr_lo = dlo(kSmemVr);
+      const uint32_t k_lo = dlo(right ? kSmemKr : kSmemKl), v_lo = dlo(right ? kSmemVr : kSmemVl);
       bool ok = mbar_wait(&misc->qfull, 0, abort_flag);
       for (int li = 0; ok && li < my_tiles; ++li) {
         if (!mbar_wait(&misc->kfull, li & 1, abort_flag)) break;
         for (int hq = 0; hq < nh; ++hq) {
           if (!mbar_wait(&misc->tfree[hq], (li & 1) ^ 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t d0 = tmem + hq * 256;
+          const uint32_t d0 = tmem + hq * 256 + (right ? 64u : 0u);
           const uint32_t qrow = (uint32_t)(hq * (kQH * 128)) >> 4;   // rows 64.. of the query-side operands
           const uint32_t qh = q_lo + qrow, oh = ohi_lo + qrow, ol = olo_lo + qrow;
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk) {
             const uint32_t o = ((kk >> 2) * kHalf + (kk & 3) * 32) >> 4;
-            if (kk == 0) umma_ss<false>(d0, kl_lo, dhi, qh, dhi, idesc);
-            else umma_ss<true>(d0, kl_lo + o, dhi, qh + o, dhi, idesc);
-          }
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t o = ((kk >> 2) * kHalf + (kk & 3) * 32) >> 4;
-            if (kk == 0) umma_ss<false>(d0 + 64, kr_lo, dhi, qh, dhi, idesc);
-            else umma_ss<true>(d0 + 64, kr_lo + o, dhi, qh + o, dhi, idesc);
+            if (kk == 0) umma_ss<false>(d0, k_lo, dhi, qh, dhi, idesc);
+            else umma_ss<true>(d0, k_lo + o, dhi, qh + o, dhi, idesc);
           }
           if (hq == nh - 1) tc_commit(&misc->kfree);
           if (hq == 0 && !mbar_wait(&misc->vfull, li & 1, abort_flag)) { ok = false; break; }
@@ -272,15 +250,8 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
           for (int kk = 0; kk < kTSteps; ++kk) {
             const uint32_t o = (((kk & 7) >> 2) * kHalf + (kk & 3) * 32) >> 4;
             const uint32_t ob = (kk < 8 ? oh : ol) + o;
-            if (kk == 0) umma_ss<false>(d0 + 128, vl_lo, dhi, ob, dhi, idesc);
-            else umma_ss<true>(d0 + 128, vl_lo + o, dhi, ob, dhi, idesc);
-          }
-#pragma unroll
-          for (int kk = 0; kk < kTSteps; ++kk) {
-            const uint32_t o = (((kk & 7) >> 2) * kHalf + (kk & 3) * 32) >> 4;
-            const uint32_t ob = (kk < 8 ? oh : ol) + o;
-            if (kk == 0) umma_ss<false>(d0 + 192, vr_lo, dhi, ob, dhi, idesc);
-            else umma_ss<true>(d0 + 192, vr_lo + o, dhi, ob, dhi, idesc);
+            if (kk == 0) umma_ss<false>(d0 + 128, v_lo, dhi, ob, dhi, idesc);
+            else umma_ss<true>(d0 + 128, v_lo + o, dhi, ob, dhi, idesc);
           }
           tc_commit(&misc->tfull[hq]);
         }
@@ -290,13 +261,18 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
     }
   } else {
     // ================================================================ statistics warps
-    const int grp = (warp - 2) >> 2;                      // queries [kQG grp, kQG grp + kQG) of each half
+    const int grp = (warp - kFirstStat) >> 2;             // its share of the queries of each half
     const int quarter = warp & 3;                         // TMEM lane quarter this warp may read
     const int lane_p = quarter * 32 + lane;               // pair within the tile
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    // chunks [c_begin, c_end) of every half
+    const int c_begin = (grp * kChunks) / kGroups, c_end = ((grp + 1) * kChunks) / kGroups;
     const int32_t* Cb = a.counts + (size_t)unit * a.n_max;
     const float4* norms = a.pair_norms + (size_t)unit * a.norm_stride;
-    const float2* qc = a.qc2 + (size_t)unit * a.M_pad + qblk * kQB;   // per query: (-(max + log2 Z), |o|^2)
+    // the partial sums of this (query block, group)
+    const size_t sub = (size_t)unit * (a.nqblk * kGroups) + (size_t)qblk * kGroups + grp;
+    float4* out4 = a.part4 + sub * a.pair_stride;
+    float* out1 = a.part1 + sub * a.pair_stride;
     // norms and counts of the next tile's pair travel while the current tile is reduced
     float4 nrm_next = make_float4(1.f, 1.f, 1.f, 0.f);
     int cl_next = 1, cr_next = 1;
@@ -307,16 +283,14 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
     for (int li = 0; li < my_tiles; ++li) {
       const int tile = t_begin + li;
       const int p = tile * kPairs + lane_p;               // candidate pair of this thread
-      const bool pair_ok = p < P;
-      const int jl = off + 2 * p;                         // its left slot
       const float4 nrm = nrm_next;
       const float cl = (float)cl_next, cr = (float)cr_next;
       if (li + 1 < my_tiles) {
         const int pn = p + kPairs;
         if (pn < P) { nrm_next = ldg_here(norms + pn); cl_next = ldg_here(Cb + off + 2 * pn); cr_next = ldg_here(Cb + off + 2 * pn + 1); }
       }
-      const float icl = 1.f / cl, icr = 1.f / cr;
-      const float r2l = nrm.x, r2r = nrm.y, pc = nrm.z, cosv = nrm.w;
+      const float icl = __fdividef(1.f, cl), icr = __fdividef(1.f, cr);   // (counts are small integers)
+      const float r2l = nrm.x, r2r = nrm.y, pc = nrm.z;
       const float n2cl = -2.f * cl, n2cr = -2.f * cr, n2il = -2.f * icl, n2ir = -2.f * icr;
 
       // beta = alpha / c = exp2(scale * s - (max + log2 Z)); sums are scaled by the counts at the end
@@ -325,26 +299,21 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
       for (int hq = 0; hq < nh; ++hq) {
         if (!warp_wait(&misc->tfull[hq], li & 1, abort_flag, lane)) { broken = true; break; }
         tc_fence_after();
-        const uint32_t col0 = tmem + lane_addr + hq * 256 + grp * kQG;
-        const float4* qc4 = reinterpret_cast<const float4*>(qc + hq * kQH + grp * kQG);
-        // chunks of 8 queries; the loads of chunk c + 1 are in flight while chunk c is reduced
-        float buf[2][4][8];
+        const uint32_t col0 = tmem + lane_addr + hq * 256;
+        const float4* qc4 = reinterpret_cast<const float4*>(misc->qconst + hq * kQH);
+        // chunks of 8 queries; the loads of the next chunk are in flight while this one is reduced
+        float buf[kDoubleBuffer ? 2 : 1][4][kChunk];
         auto issue = [&](int c, int b) {
-          const uint32_t col = col0 + c * 8;
+          const uint32_t col = col0 + c * kChunk;
           tmem_ld8(col, buf[b][0]);
           tmem_ld8(col + 64, buf[b][1]);
           tmem_ld8(col + 128, buf[b][2]);
           tmem_ld8(col + 192, buf[b][3]);
         };
-        issue(0, 0);
+        auto reduce = [&](int c, int b) {
 #pragma unroll
-        for (int c = 0; c < kQG / 8; ++c) {
-          const int b = c & 1;
-          tmem_ld_wait();
-          if (c + 1 < kQG / 8) issue(c + 1, b ^ 1);
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const float4 cq = __ldg(qc4 + c * 4 + (i >> 1));               // two queries' constants (the same address in every lane)
+          for (int i = 0; i < kChunk; ++i) {
+            const float4 cq = qc4[c * (kChunk / 2) + (i >> 1)];           // two queries' constants (a broadcast read)
             const float ncq = (i & 1) ? cq.z : cq.x;
             const float hq2 = (i & 1) ? cq.w : cq.y;
             const float bl = fast_exp2(fmaf(buf[b][0][i], a.scale_log2, ncq));
@@ -373,45 +342,35 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
               sN12 = fmaf(bl * br, fast_sqrt(fabsf(d12)), sN12);
             }
           }
+        };
+        if constexpr (kDoubleBuffer) {
+          issue(c_begin, 0);
+          for (int c = c_begin; c < c_end; c += 2) {
+            tmem_ld_wait();
+            if (c + 1 < c_end) issue(c + 1, 1);
+            reduce(c, 0);
+            if (c + 1 < c_end) {
+              tmem_ld_wait();
+              if (c + 2 < c_end) issue(c + 2, 0);
+              reduce(c + 1, 1);
+            }
+          }
+        } else {
+          // (with four warps per scheduler the other warps cover the latency of the loads)
+          for (int c = c_begin; c < c_end; ++c) {
+            issue(c, 0);
+            tmem_ld_wait();
+            reduce(c, 0);
+          }
         }
         tc_fence_before();
         warp_arrive(&misc->tfree[hq], lane);                               // this half may be overwritten
       }
       if (broken) break;
-
-      // ---- the sums of a pair travel from the last group down to group 0, which owns the outputs: each
-      //      group adds its own to what it receives (a fixed order, so the result is reproducible)
-      float* x = misc->xbuf + lane_p * 5;
-      if (grp == kGroups - 1) {
-        // the first group must have read the previous tile's sums
-        if (!warp_wait(&misc->xfree[quarter], (li & 1) ^ 1, abort_flag, lane)) break;
-      } else {
-        if (!warp_wait(&misc->xhand[kGroups - 2 - grp][quarter], li & 1, abort_flag, lane)) break;
-        sAl += x[0]; sAr += x[1]; sN1l += x[2]; sN1r += x[3]; sN12 += x[4];
-      }
-      if (grp != 0) {
-        x[0] = sAl; x[1] = sAr; x[2] = sN1l; x[3] = sN1r; x[4] = sN12;
-        warp_arrive(&misc->xhand[kGroups - 1 - grp][quarter], lane);
-      } else {
-        warp_arrive(&misc->xfree[quarter], lane);                          // the buffer may be rewritten
-        const float Al = cl * sAl, Ar = cr * sAr;
-        const float N1l = cl * sN1l, N1r = cr * sN1r;
-        const float N12 = (kExact ? -1.f : 1.f) * cl * cr * sN12;
-        if (pair_ok) {
-          if (a.nqblk == 1) {
-            const size_t pi = (size_t)unit * a.pair_stride + p;
-            if (a.A) { a.A[(size_t)unit * a.n_max + jl] = Al; a.A[(size_t)unit * a.n_max + jl + 1] = Ar; }
-            if (a.N1) { a.N1[(size_t)unit * a.n_max + jl] = N1l; a.N1[(size_t)unit * a.n_max + jl + 1] = N1r; }
-            finalize_pair(a, pi, Al, Ar, N1l, N1r, N12, cosv);
-          } else {
-            // partial sums of this query block; a separate kernel adds the blocks in order
-            const size_t slot_i = ((size_t)unit * a.nqblk + qblk) * a.n_max + jl;
-            const size_t pair_i = ((size_t)unit * a.nqblk + qblk) * a.pair_stride + p;
-            a.partA[slot_i] = Al; a.partA[slot_i + 1] = Ar;
-            a.partN1[slot_i] = N1l; a.partN1[slot_i + 1] = N1r;
-            a.partN12[pair_i] = N12;
-          }
-        }
+      // the sums of this (query block, group) for the pair: a later kernel adds the partials in order
+      if (p < P) {
+        out4[p] = make_float4(cl * sAl, cr * sAr, cl * sN1l, cr * sN1r);
+        out1[p] = (kExact ? -1.f : 1.f) * cl * cr * sN12;
       }
     }
   }
@@ -427,7 +386,13 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
   if (threadIdx.x == 0 && misc->abort_flag && a.status_dev) atomicExch(a.status_dev, (int)KVS_ERR_TIMEOUT);
 }
 
-// Sum of the per-query-block partials in block order, then score and weight of each pair.
+// Sum of the partials of all (query block, statistics group) pairs in a fixed order, then score and
+// left-key weight of each candidate pair.  Weight modes:
+//   0: the sums are norms; w = (N1_l - N12) / (N1_l - 2 N12 + N1_r)                        [Eq. kstar_final]
+//   1: they are the signed sums G11, G22, G12 of g_ij = E^T c_ij; w = (G11 + G12) / (G11 + 2 G12 + G22)
+//                                                                            [Eq. kstar_weight_final_rewrite]
+//   2: as 1 with the coupling dropped, w = G11 / (G11 + G22)                              [Eq. simplified_k]
+// A denominator that is not safely positive gives 1/2; the weight is clipped to [0, 1].
 __global__ void __launch_bounds__(256)
 stats_finalize_kernel(const StatsTcArgs a, const RoundTable tab) {
   const SeqRound sr = tab.s[blockIdx.z];
@@ -436,17 +401,33 @@ stats_finalize_kernel(const StatsTcArgs a, const RoundTable tab) {
   const int p = blockIdx.x * 256 + threadIdx.x;
   if (p >= sr.P) return;
   const int jl = tab.off + 2 * p;
+  const int nsub = a.nqblk * kGroups;
   float Al = 0.f, Ar = 0.f, N1l = 0.f, N1r = 0.f, N12 = 0.f;
-  for (int qb = 0; qb < a.nqblk; ++qb) {
-    const size_t si = ((size_t)unit * a.nqblk + qb) * a.n_max + jl;
-    Al += a.partA[si]; Ar += a.partA[si + 1];
-    N1l += a.partN1[si]; N1r += a.partN1[si + 1];
-    N12 += a.partN12[((size_t)unit * a.nqblk + qb) * a.pair_stride + p];
+  for (int sb = 0; sb < nsub; ++sb) {
+    const size_t i = ((size_t)unit * nsub + sb) * a.pair_stride + p;
+    const float4 v = a.part4[i];
+    Al += v.x; Ar += v.y; N1l += v.z; N1r += v.w;
+    N12 += a.part1[i];
+  }
+  const float cosv = a.pair_norms[(size_t)unit * a.norm_stride + p].w;
+  const float mass = Al + Ar;
+  const float score = (a.score_mode == 0) ? mass * fmaxf(0.f, 1.f - cosv) : mass;
+  float w = 0.5f;
+  if (a.weight_mode == 0) {
+    const float D = N1l - 2.f * N12 + N1r;
+    if (D > 1e-6f * (N1l + N1r) && D < INFINITY) w = fminf(1.f, fmaxf(0.f, (N1l - N12) / D));
+  } else {
+    const float g12 = (a.weight_mode == 2) ? 0.f : N12;
+    const float gamma = N1l + 2.f * g12 + N1r;
+    if (gamma > 1e-6f * (fabsf(N1l) + fabsf(N1r)) && gamma < INFINITY) w = fminf(1.f, fmaxf(0.f, (N1l + g12) / gamma));
   }
   const size_t pi = (size_t)unit * a.pair_stride + p;
+  a.score[pi] = fabsf(score);
+  a.w[pi] = w;
+  if (a.N12) a.N12[pi] = N12;
+  if (a.cosv) a.cosv[pi] = cosv;
   if (a.A) { a.A[(size_t)unit * a.n_max + jl] = Al; a.A[(size_t)unit * a.n_max + jl + 1] = Ar; }
   if (a.N1) { a.N1[(size_t)unit * a.n_max + jl] = N1l; a.N1[(size_t)unit * a.n_max + jl + 1] = N1r; }
-  finalize_pair(a, pi, Al, Ar, N1l, N1r, N12, a.pair_norms[(size_t)unit * a.norm_stride + p].w);
 }
 
 }  // namespace
@@ -465,7 +446,7 @@ cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const
   if (a.weight_mode == 0) hessian_stats_tc<false><<<grid, kThreads, kSmemBytes, st>>>(a, t, tmKp, tmVp, tmQ, tmOhi, tmOlo);
   else hessian_stats_tc<true><<<grid, kThreads, kSmemBytes, st>>>(a, t, tmKp, tmVp, tmQ, tmOhi, tmOlo);
   cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess || a.nqblk == 1) return e;
+  if (e != cudaSuccess) return e;
   int pmax = 0;
   for (int i = 0; i < t.nseq; ++i) pmax = pmax > t.s[i].P ? pmax : t.s[i].P;
   if (pmax <= 0) return cudaSuccess;
