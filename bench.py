@@ -392,6 +392,27 @@ def run_stream(args):
     return rec
 
 
+def other_configs_report(skip):
+    """Device-resident step time of the other benchmark configurations (each in a process of its
+    own, 5 steps after 3 warm-ups, same code path as the headline): every config gets a number from
+    the same run, not only the one the headline is quoted on."""
+    out = {}
+    for c in range(5):
+        if c == skip:
+            continue
+        cmd = [sys.executable, os.path.abspath(__file__), "--config", str(c), "--steps", "5", "--warmup", "3",
+               "--no-e2e", "--no-cpu-baseline", "--no-extras"]
+        try:
+            r = subprocess.run(cmd, capture_output=True, text=True, timeout=600)
+            d = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])
+            out[f"configs[{c}]"] = {"ms_per_step": d["ms_per_step"], "value": d["value"],
+                                    "kernels_ms": {k: v["ms_per_step"] for k, v in d["roofline"]["per_kernel"].items()},
+                                    "sm_mhz": d["clocks"].get("sm_mhz")}
+        except Exception as e:                                   # a failed side measurement must not lose the headline
+            out[f"configs[{c}]"] = {"error": str(e)[:200]}
+    return out
+
+
 def weight_mode_report(kb, torch, w):
     """How far the gradient-free weights of Eq. kstar_final are from the exact weights of
     Eq. kstar_weight_final_rewrite, and those from the diagonal-only merge of Eq. simplified_k, on
@@ -700,12 +721,14 @@ def main():
                "sample": f"layer 0, sequence 0, KV head 0 only ({n0} tokens, all rounds): {t_unit:.1f} s; "
                          f"scaled to a layer of {Hkv} heads"}
 
-    stream_rec = weights_rec = None
+    stream_rec = weights_rec = others_rec = None
     if rank == 0 and world == 1 and not args.no_extras:
         del mK, mV, mC, wK, wV, wC, ws
         torch.cuda.empty_cache()
         weights_rec = weight_mode_report(kb, torch, w)
         stream_rec = run_stream(argparse.Namespace(layers=0, steps=20, warmup=3))
+        torch.cuda.empty_cache()
+        others_rec = other_configs_report(w.config_id)
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -716,7 +739,7 @@ def main():
                 "removed_tokens_per_sec_per_layer":
                     world * L * sum(n - b for n, b in zip(w.seq_lens, w.budgets)) / (ms_per_step * 1e-3),
                 "stream_step_ms": stream_rec["value"] if stream_rec else None, "stream": stream_rec,
-                "weight_modes": weights_rec}
+                "weight_modes": weights_rec, "other_configs": others_rec}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
