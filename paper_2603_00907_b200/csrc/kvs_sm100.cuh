@@ -80,14 +80,16 @@ __device__ __forceinline__ bool mbar_poll(uint64_t* bar, uint32_t parity, uint32
 // Bounded wait: false once the time limit has passed (or when another role already flagged an
 // abort).  `ctl` points at two ints in shared memory: ctl[0] is the CTA's abort flag, ctl[1] the
 // time limit of one wait in microseconds (one second unless the host asked otherwise).
-// These kernels are chains of hand-offs, so the wake-up latency of a wait counts for more than
-// the issue slots its polling takes: a wait on the critical path (`eager`) polls in a tight
-// loop and looks at the clock only between bursts; a role that runs ahead of the others anyway
-// lets the hardware suspend it between attempts.
+// These kernels are chains of hand-offs, so the wake-up latency of a wait counts: a wait on the
+// critical path (`eager`) first polls in a tight loop for a few hundred cycles; after that, and
+// for a role that runs ahead of the others anyway, the hardware suspends the thread between attempts.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* ctl, bool eager = false) {
   if (mbar_try_wait(bar, parity)) return true;
+  // (an eager waiter polls for a short while only: a long wait in a tight loop would take issue
+  // slots from the warps that have work to do)
+  if (eager && mbar_poll(bar, parity, 48)) return true;
   const uint64_t t0 = globaltimer_ns();
-  while (!(eager ? mbar_poll(bar, parity, 256) : mbar_try_wait_hint(bar, parity, 10000u))) {
+  while (!mbar_try_wait_hint(bar, parity, 10000u)) {
     if (ctl[0]) return false;
     if (globaltimer_ns() - t0 > (uint64_t)(uint32_t)ctl[1] * 1000ull) { ctl[0] = 1; return false; }
   }

@@ -56,7 +56,9 @@ struct Misc {
   uint64_t kfull, vfull, kfree, vfree, tfull[2], tfree[2], qfull;
   uint32_t tmem_base;
   int abort_flag, wait_us;                 // (adjacent: the bounded waits read both through one pointer)
-  alignas(16) float2 qconst[kQB];          // per query of the block: (-(max + log2 Z), |o|^2 or <E, o>)
+  // per two queries (2k, 2k+1) of the block: (c_2k, c_2k+1, h_2k, h_2k+1) with c = -(max + log2 Z) and
+  // h = |o|^2 (or <E, o>): neighbours sit side by side for the packed two-float arithmetic
+  alignas(16) float qconst[2 * kQB];
 };
 constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc);
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
@@ -142,7 +144,11 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
     mbar_fence_init();
   }
   // the per-query constants of the block (the same for every tile): read from shared memory in the loop
-  if (threadIdx.x < kQB) misc->qconst[threadIdx.x] = a.qc2[(size_t)unit * a.M_pad + qblk * kQB + threadIdx.x];
+  if (threadIdx.x < kQB) {
+    const float2 c = a.qc2[(size_t)unit * a.M_pad + qblk * kQB + threadIdx.x];
+    misc->qconst[(threadIdx.x >> 1) * 4 + (threadIdx.x & 1)] = c.x;
+    misc->qconst[(threadIdx.x >> 1) * 4 + 2 + (threadIdx.x & 1)] = c.y;
+  }
   if (warp == 1) tmem_alloc(&misc->tmem_base, 512);
   tc_fence_before();
   __syncthreads();
@@ -265,8 +271,6 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
     const int quarter = warp & 3;                         // TMEM lane quarter this warp may read
     const int lane_p = quarter * 32 + lane;               // pair within the tile
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-    // chunks [c_begin, c_end) of every half
-    const int c_begin = (grp * kChunks) / kGroups, c_end = ((grp + 1) * kChunks) / kGroups;
     const int32_t* Cb = a.counts + (size_t)unit * a.n_max;
     const float4* norms = a.pair_norms + (size_t)unit * a.norm_stride;
     // the partial sums of this (query block, group)
@@ -293,14 +297,27 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
       const float r2l = nrm.x, r2r = nrm.y, pc = nrm.z;
       const float n2cl = -2.f * cl, n2cr = -2.f * cr, n2il = -2.f * icl, n2ir = -2.f * icr;
 
-      // beta = alpha / c = exp2(scale * s - (max + log2 Z)); sums are scaled by the counts at the end
-      float sAl = 0.f, sAr = 0.f, sN1l = 0.f, sN1r = 0.f, sN12 = 0.f;
+      // beta = alpha / c = exp2(scale * s - (max + log2 Z)); sums are scaled by the counts at the end.
+      // The arithmetic runs on pairs of neighbouring queries with the packed two-float instructions
+      // (fma/add/mul.f32x2): the kernel is as short of issue slots as of special-function slots, and a
+      // packed instruction takes one slot for two operations.  Every sum is kept as two lanes.
+      float2 sAl = make_float2(0.f, 0.f), sAr = sAl, sN1l = sAl, sN1r = sAl, sN12 = sAl;
+      const float2 sc2 = make_float2(a.scale_log2, a.scale_log2), one2 = make_float2(1.f, 1.f);
+      const float2 n2cl2 = make_float2(n2cl, n2cl), n2cr2 = make_float2(n2cr, n2cr);
+      const float2 n2il2 = make_float2(n2il, n2il), n2ir2 = make_float2(n2ir, n2ir);
+      const float2 icl2 = make_float2(icl, icl), icr2 = make_float2(icr, icr);
+      const float2 r2l2 = make_float2(r2l, r2l), r2r2 = make_float2(r2r, r2r), pc2 = make_float2(pc, pc);
+      const float2 m42 = make_float2(-4.f, -4.f);
       bool broken = false;
       for (int hq = 0; hq < nh; ++hq) {
         if (!warp_wait(&misc->tfull[hq], li & 1, abort_flag, lane)) { broken = true; break; }
         tc_fence_after();
         const uint32_t col0 = tmem + lane_addr + hq * 256;
-        const float4* qc4 = reinterpret_cast<const float4*>(misc->qconst + hq * kQH);
+        const float4* qc4 = reinterpret_cast<const float4*>(misc->qconst + hq * (2 * kQH));
+        // chunks [c_begin, c_end) of every half (2 / 3 / 3 of the eight: letting the short share go round
+        // among the groups measured slower; the group that is done early moves on to the next half
+        // and the groups end up staggered, which spreads their serial phases)
+        const int c_begin = (grp * kChunks) / kGroups, c_end = ((grp + 1) * kChunks) / kGroups;
         // chunks of 8 queries; the loads of the next chunk are in flight while this one is reduced
         float buf[kDoubleBuffer ? 2 : 1][4][kChunk];
         auto issue = [&](int c, int b) {
@@ -312,34 +329,36 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
         };
         auto reduce = [&](int c, int b) {
 #pragma unroll
-          for (int i = 0; i < kChunk; ++i) {
-            const float4 cq = qc4[c * (kChunk / 2) + (i >> 1)];           // two queries' constants (a broadcast read)
-            const float ncq = (i & 1) ? cq.z : cq.x;
-            const float hq2 = (i & 1) ? cq.w : cq.y;
-            const float bl = fast_exp2(fmaf(buf[b][0][i], a.scale_log2, ncq));
-            const float br = fast_exp2(fmaf(buf[b][1][i], a.scale_log2, ncq));
-            sAl += bl;
-            sAr += br;
+          for (int i = 0; i < kChunk; i += 2) {
+            const float4 cq = qc4[c * (kChunk / 2) + (i >> 1)];           // the two queries' constants (a broadcast read)
+            const float2 ncq = make_float2(cq.x, cq.y), hq2 = make_float2(cq.z, cq.w);
+            const float2 el = __ffma2_rn(make_float2(buf[b][0][i], buf[b][0][i + 1]), sc2, ncq);
+            const float2 er = __ffma2_rn(make_float2(buf[b][1][i], buf[b][1][i + 1]), sc2, ncq);
+            const float2 bl = make_float2(fast_exp2(el.x), fast_exp2(el.y));
+            const float2 br = make_float2(fast_exp2(er.x), fast_exp2(er.y));
+            const float2 tl = make_float2(buf[b][2][i], buf[b][2][i + 1]), tr = make_float2(buf[b][3][i], buf[b][3][i + 1]);
+            sAl = __fadd2_rn(sAl, bl);
+            sAr = __fadd2_rn(sAr, br);
+            const float2 al = __ffma2_rn(bl, n2cl2, one2), ar = __ffma2_rn(br, n2cr2, one2);   // 1 - 2 alpha
             if constexpr (kExact) {
               // g11 = alpha (1 - 2 alpha) E^T (vbar_l - o), g12 = -alpha_l alpha_r E^T (vbar_l + vbar_r - 2 o);
               // hq2 holds <E_q, o_q> here (the sign of g12 is applied after the loop)
-              const float gl = bl * fmaf(bl, n2cl, 1.f);                   // beta (1 - 2 alpha)
-              const float gr = br * fmaf(br, n2cr, 1.f);
-              const float hl = fmaf(buf[b][2][i], icl, -hq2);              // E^T (vbar_l - o)
-              const float hr = fmaf(buf[b][3][i], icr, -hq2);
-              sN1l = fmaf(gl, hl, sN1l);
-              sN1r = fmaf(gr, hr, sN1r);
-              sN12 = fmaf(bl * br, hl + hr, sN12);
+              const float2 nh2 = make_float2(-hq2.x, -hq2.y);
+              const float2 hl = __ffma2_rn(tl, icl2, nh2), hr = __ffma2_rn(tr, icr2, nh2);     // E^T (vbar - o)
+              sN1l = __ffma2_rn(__fmul2_rn(bl, al), hl, sN1l);
+              sN1r = __ffma2_rn(__fmul2_rn(br, ar), hr, sN1r);
+              sN12 = __ffma2_rn(__fmul2_rn(bl, br), __fadd2_rn(hl, hr), sN12);
             } else {
-              const float gl = bl * fabsf(fmaf(bl, n2cl, 1.f));            // beta |1 - 2 alpha|
-              const float gr = br * fabsf(fmaf(br, n2cr, 1.f));
-              const float dl = fmaf(buf[b][2][i], n2il, r2l + hq2);        // |vbar_l - o|^2
-              const float dr = fmaf(buf[b][3][i], n2ir, r2r + hq2);
-              sN1l = fmaf(gl, fast_sqrt(fabsf(dl)), sN1l);
-              sN1r = fmaf(gr, fast_sqrt(fabsf(dr)), sN1r);
-              const float u = fmaf(buf[b][2][i], icl, buf[b][3][i] * icr) - hq2;   // <vbar_l + vbar_r, o> - |o|^2
-              const float d12 = fmaf(u, -4.f, pc);                         // |vbar_l + vbar_r - 2 o|^2
-              sN12 = fmaf(bl * br, fast_sqrt(fabsf(d12)), sN12);
+              const float2 gl = make_float2(bl.x * fabsf(al.x), bl.y * fabsf(al.y));          // beta |1 - 2 alpha|
+              const float2 gr = make_float2(br.x * fabsf(ar.x), br.y * fabsf(ar.y));
+              const float2 dl = __ffma2_rn(tl, n2il2, __fadd2_rn(r2l2, hq2));                  // |vbar_l - o|^2
+              const float2 dr = __ffma2_rn(tr, n2ir2, __fadd2_rn(r2r2, hq2));
+              sN1l = __ffma2_rn(gl, make_float2(fast_sqrt(fabsf(dl.x)), fast_sqrt(fabsf(dl.y))), sN1l);
+              sN1r = __ffma2_rn(gr, make_float2(fast_sqrt(fabsf(dr.x)), fast_sqrt(fabsf(dr.y))), sN1r);
+              // <vbar_l + vbar_r, o> - |o|^2, then |vbar_l + vbar_r - 2 o|^2
+              const float2 u = __fadd2_rn(__ffma2_rn(tl, icl2, __fmul2_rn(tr, icr2)), make_float2(-hq2.x, -hq2.y));
+              const float2 d12 = __ffma2_rn(u, m42, pc2);
+              sN12 = __ffma2_rn(__fmul2_rn(bl, br), make_float2(fast_sqrt(fabsf(d12.x)), fast_sqrt(fabsf(d12.y))), sN12);
             }
           }
         };
@@ -369,8 +388,8 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
       if (broken) break;
       // the sums of this (query block, group) for the pair: a later kernel adds the partials in order
       if (p < P) {
-        out4[p] = make_float4(cl * sAl, cr * sAr, cl * sN1l, cr * sN1r);
-        out1[p] = (kExact ? -1.f : 1.f) * cl * cr * sN12;
+        out4[p] = make_float4(cl * (sAl.x + sAl.y), cr * (sAr.x + sAr.y), cl * (sN1l.x + sN1l.y), cr * (sN1r.x + sN1r.y));
+        out1[p] = (kExact ? -1.f : 1.f) * cl * cr * (sN12.x + sN12.y);
       }
     }
   }
