@@ -1,10 +1,11 @@
 // Attention partials on the tensor cores (tcgen05 + TMEM + TMA), queries on TMEM lanes.
 //
-// One CTA owns a block of 128 query rows (Q is staged once and copied into tensor memory) and a contiguous range
+// One CTA owns a block of 128 query rows (Q is staged once in shared memory) and a contiguous range
 // of 128-slot tiles.  K and V tiles travel in two separate two-stage TMA rings; per tile one
 // thread issues
-//   S[q, slot] = Q K_tile^T                         (fp32 in TMEM, double buffered; Q is read from TMEM too,
-//                                                    so that only the K rows cross the shared-memory port)
+//   S[q, slot] = Q K_tile^T                         (fp32 in TMEM, three buffers: the logits run two tiles
+//                                                    ahead of the P V products, so that a softmax team that
+//                                                    has finished a tile finds its next one already formed)
 // Two teams of eight softmax warps take alternate tiles, so that one team's arithmetic overlaps
 // the other team's waits.  Inside a team the two warps of a TMEM lane quarter own the same 32
 // query rows and 64 slot columns each.  A thread reads its logits twice: once for the maximum
@@ -42,9 +43,10 @@ constexpr int kSmemMisc = kSmemStage + 2 * kStage;
 constexpr int kSoftmaxWarps = 16, kNormWarps = 4;
 constexpr int kThreads = (2 + kSoftmaxWarps + kNormWarps) * 32;   // warp 0: TMA, 1: MMA, 2-17: softmax, 18-21: pair norms
 constexpr float kRescaleGap = 8.f;         // log2 units
+constexpr int kSBufs = 3;                  // logit / P' buffers in tensor memory
 
 struct Misc {
-  uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[2], pready[2][2], ofull[2], stabdone[2], qfull, qready;
+  uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[kSBufs], pready[kSBufs][2], ofull[2], stabdone[2], qfull;
   uint32_t tmem_base;
   int abort_flag, wait_us;                 // (adjacent: the bounded waits read both through one pointer)
   float rowmax[2][2][2][kTile];            // per team, tile parity, column half and query row: that thread's maximum logit
@@ -55,7 +57,7 @@ struct Misc {
 constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc);
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 
-constexpr uint32_t kColQ = 256, kColO = 384;   // TMEM columns: two logit buffers of 128, Q (64), O (128)
+constexpr uint32_t kColO = 384;                // TMEM columns: three logit buffers of 128, then O (128)
 
 __device__ __forceinline__ void team_barrier(int team) { asm volatile("bar.sync %0, 256;" ::"r"(team + 1) : "memory"); }
 __device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 3, 512;" ::: "memory"); }
@@ -200,14 +202,15 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       mbar_init(&misc->kfree[s], norm_k ? 1 + kNormWarps : 1);   // MMA commit (+ the pair-norm warps)
       mbar_init(&misc->vfree[s], norm_v ? 1 + kNormWarps : 1);
       mbar_init(&misc->stabdone[s], kSoftmaxWarps / 2);
-      mbar_init(&misc->sfull[s], 1);
       mbar_init(&misc->ofull[s], 1);
+    }
+    for (int b = 0; b < kSBufs; ++b) {
+      mbar_init(&misc->sfull[b], 1);
       // P' is handed over in two halves (the last and the first 32 slots of every thread's 64), so
       // that the P V products of one half run while the other half is still being written
-      for (int hf = 0; hf < 2; ++hf) mbar_init(&misc->pready[s][hf], kSoftmaxWarps / 2);
+      for (int hf = 0; hf < 2; ++hf) mbar_init(&misc->pready[b][hf], kSoftmaxWarps / 2);
     }
     mbar_init(&misc->qfull, 1);
-    mbar_init(&misc->qready, kSoftmaxWarps);
     misc->abort_flag = 0;
     misc->wait_us = (int)a.wait_us;
     mbar_fence_init();
@@ -272,38 +275,43 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       // descriptors are kept as a constant high word and a low word that only needs an addition.
       constexpr uint32_t idesc_s = idesc_bf16(128, 128);                 // Q (K-major) x K tile (K-major)
       constexpr uint32_t idesc_o = idesc_bf16(128, 128, false, true);    // P' (K-major) x V tile (MN-major)
+      const uint64_t qd0 = smem_desc_sw128(smem_u32(smem + kSmemQ), 16, 1024);
       const uint64_t kd0 = smem_desc_sw128(smem_u32(smem + kSmemStage), 16, 1024);
       const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + kSmemStage + kOperand), kHalf, 1024);
       const uint32_t kd_hi = (uint32_t)(kd0 >> 32), vd_hi = (uint32_t)(vd0 >> 32);
-      const uint32_t kd_lo0 = (uint32_t)kd0, vd_lo0 = (uint32_t)vd0;     // stage 0; stage 1 is kStage / 16 further
+      const uint32_t qd_lo = (uint32_t)qd0, kd_lo0 = (uint32_t)kd0, vd_lo0 = (uint32_t)vd0;   // stage 0; stage 1 is kStage / 16 further
+      // The logits of tile li go to buffer li mod 3, which last held P' of tile li - 3: the products
+      // that read it were issued by this thread before.  With three buffers the logits run two
+      // tiles ahead of the P V products, so that a softmax team that has finished tile li finds the
+      // logits of its next tile, li + 2, already formed instead of waiting for P V of tile li.
       auto issue_s = [&](int li) -> bool {
-        const int s = li & 1, k = li >> 1;                 // K stage = logit buffer
-        // the buffer last held P' of tile li - 2, whose products were issued by this thread before
+        const int s = li & 1, k = li >> 1;                 // K stage and its use count
         if (!mbar_wait(&misc->kfull[s], k & 1, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t kd_lo = kd_lo0 + s * (kStage >> 4), ds = tmem + s * 128;
+        const uint32_t kd_lo = kd_lo0 + s * (kStage >> 4), ds = tmem + (uint32_t)(li % kSBufs) * 128;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
-          const uint32_t o = (kk >> 2) * kHalf + (kk & 3) * 32;
-          if (kk == 0) umma_ts<false>(ds, tmem + kColQ, kd_lo, kd_hi, idesc_s);
-          else umma_ts<true>(ds, tmem + kColQ + 8 * kk, kd_lo + (o >> 4), kd_hi, idesc_s);
+          const uint32_t o = ((kk >> 2) * kHalf + (kk & 3) * 32) >> 4;
+          if (kk == 0) umma_ss<false>(ds, qd_lo, kd_hi, kd_lo, kd_hi, idesc_s);
+          else umma_ss<true>(ds, qd_lo + o, kd_hi, kd_lo + o, kd_hi, idesc_s);
         }
-        tc_commit(&misc->sfull[s]);
+        tc_commit(&misc->sfull[li % kSBufs]);
         tc_commit(&misc->kfree[s]);
         return true;
       };
-      bool ok = mbar_wait(&misc->qready, 0, abort_flag);
-      if (ok) tc_fence_after();
+      bool ok = mbar_wait(&misc->qfull, 0, abort_flag);
       ok = ok && issue_s(0);
+      if (ok && my_tiles > 1) ok = issue_s(1);
       for (int li = 0; ok && li < my_tiles; ++li) {
-        // the next tile's logits are queued before this tile's P V products
-        if (li + 1 < my_tiles) ok = issue_s(li + 1);
-        const int s = li & 1, ph = (li >> 1) & 1;          // V stage = logit buffer
+        // the logits of the tile after next are queued before this tile's P V products
+        if (li + 2 < my_tiles) ok = issue_s(li + 2);
+        const int s = li & 1, ph = (li >> 1) & 1;          // V stage and its phase
+        const int b = li % kSBufs, bph = (li / kSBufs) & 1; // P' buffer and its phase
         if (ok && !mbar_wait(&misc->vfull[s], ph, abort_flag)) ok = false;
-        const uint32_t vd_lo = vd_lo0 + s * (kStage >> 4), ps = tmem + s * 128;
+        const uint32_t vd_lo = vd_lo0 + s * (kStage >> 4), ps = tmem + (uint32_t)b * 128;
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
-          if (ok && !mbar_wait(&misc->pready[s][hf], ph, abort_flag)) ok = false;
+          if (ok && !mbar_wait(&misc->pready[b][hf], bph, abort_flag)) ok = false;
           if (!ok) break;
           tc_fence_after();
           const int sub = 1 - hf;                            // the last 32 slots of a thread's 64 come first
@@ -402,25 +410,6 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     float m_stab = 0.f, l = 0.f;
     bool have_stab = false;
     bool alive = true;
-    // Q into tensor memory: row on its lane, two channels per 32-bit column; each of the four
-    // warps of a lane quarter copies 32 channels (rows past the last query were staged as zeros)
-    {
-      const int part = ((warp - 2) >> 2);                  // channels [32 part, 32 part + 32)
-      alive = warp_wait(&misc->qfull, 0, abort_flag, lane);
-      const uint8_t* qrow = smem + kSmemQ + (part >> 1) * kHalf + row * 128;
-      uint32_t qv[16];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int c = (part & 1) * 4 + i;
-        const uint4 v = *reinterpret_cast<const uint4*>(qrow + ((c ^ (row & 7)) << 4));
-        qv[4 * i] = v.x; qv[4 * i + 1] = v.y; qv[4 * i + 2] = v.z; qv[4 * i + 3] = v.w;
-      }
-      tmem_st8(tmem + lane_addr + kColQ + part * 16, qv);
-      tmem_st8(tmem + lane_addr + kColQ + part * 16 + 8, qv + 8);
-      tmem_st_wait();
-      tc_fence_before();
-      warp_arrive(&misc->qready, lane);
-    }
     // (first column half) the count of slot `row` of the team's next tile travels meanwhile
     int cnt_next = 1;
     if (ch == 0 && team_tiles > 0) {
@@ -430,8 +419,13 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     // logits of 32 columns, relative to the stabiliser (one multiply-add), masked where needed
     auto scale32 = [&](int j0, float* x) {
       if (j0 >= 0 && j0 + 31 <= last_free) {
+        // (two columns per instruction: the softmax warps are bound by issue slots)
+        const float2 sc2 = make_float2(a.scale_log2, a.scale_log2), nm2 = make_float2(-m_stab, -m_stab);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) x[i] = fmaf(x[i], a.scale_log2, -m_stab);
+        for (int i = 0; i < 32; i += 2) {
+          const float2 v = __ffma2_rn(make_float2(x[i], x[i + 1]), sc2, nm2);
+          x[i] = v.x; x[i + 1] = v.y;
+        }
       } else {
 #pragma unroll
         for (int i = 0; i < 32; ++i)
@@ -454,7 +448,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     // value cut to bf16 (a byte permute, no conversion); the lo term rounds the exact remainder, so
     // hi + lo carries 16 significant bits.  Returns sum_j c_j P'_j.
     auto emit32 = [&](uint32_t col, const float* x, const float* cnt32) {
-      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+      float2 ls[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
       for (int c = 0; c < 4; c += 2) {
         uint32_t hi[8], lo[8];
@@ -462,26 +456,27 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         for (int c2 = c; c2 < c + 2; ++c2) {
           const float4 ca = *reinterpret_cast<const float4*>(&cnt32[c2 * 8]);
           const float4 cb = *reinterpret_cast<const float4*>(&cnt32[c2 * 8 + 4]);
-          const float cc[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+          const float2 cc[4] = {make_float2(ca.x, ca.y), make_float2(ca.z, ca.w), make_float2(cb.x, cb.y), make_float2(cb.z, cb.w)};
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
             const int i = c2 * 8 + u * 2;
-            const float q0 = fast_exp2(x[i]), q1 = fast_exp2(x[i + 1]);
-            ls[u] = fmaf(cc[2 * u], q0, fmaf(cc[2 * u + 1], q1, ls[u]));
-            const uint32_t b0 = __float_as_uint(q0), b1 = __float_as_uint(q1);
+            const float2 q = make_float2(fast_exp2(x[i]), fast_exp2(x[i + 1]));
+            ls[u] = __ffma2_rn(cc[u], q, ls[u]);                     // (two slots per instruction)
+            const uint32_t b0 = __float_as_uint(q.x), b1 = __float_as_uint(q.y);
             hi[(c2 & 1) * 4 + u] = __byte_perm(b0, b1, 0x7632);
-            lo[(c2 & 1) * 4 + u] = pack_bf16(q0 - __uint_as_float(b0 & 0xffff0000u), q1 - __uint_as_float(b1 & 0xffff0000u));
+            const float2 r = __fadd2_rn(q, make_float2(-__uint_as_float(b0 & 0xffff0000u), -__uint_as_float(b1 & 0xffff0000u)));
+            lo[(c2 & 1) * 4 + u] = pack_bf16(r.x, r.y);
           }
         }
         tmem_st8(col + (c >> 1) * 8, hi);
         tmem_st8(col + 16 + (c >> 1) * 8, lo);
       }
       tmem_st_wait();
-      return (ls[0] + ls[1]) + (ls[2] + ls[3]);
+      return ((ls[0].x + ls[0].y) + (ls[1].x + ls[1].y)) + ((ls[2].x + ls[2].y) + (ls[3].x + ls[3].y));
     };
     for (int j = 0; j < team_tiles; ++j) {
       const int li = 2 * j + team;
-      const int s = li & 1, b = li & 1, ph = j & 1;        // K/V stage, logit buffer and its phase
+      const int s = li & 1, b = li % kSBufs, ph = (li / kSBufs) & 1;   // K/V stage, logit buffer and its phase
       const uint32_t scol = tmem + lane_addr + b * 128 + ch * 64;   // this thread's 64 logit columns
       const int tile_row0 = (t_begin + li) * kTile - shift;
       const int jA = tile_row0 + ch * 64, jB = jA + 32;    // first slots of this thread's two column groups
