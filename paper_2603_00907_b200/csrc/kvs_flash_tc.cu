@@ -41,12 +41,13 @@ constexpr int kStage = 2 * kOperand;       // K tile + V tile
 constexpr int kSmemQ = 0, kSmemStage = kOperand;
 constexpr int kSmemMisc = kSmemStage + 2 * kStage;
 constexpr int kSoftmaxWarps = 16, kNormWarps = 4;
-constexpr int kThreads = (2 + kSoftmaxWarps + kNormWarps) * 32;   // warp 0: TMA, 1: MMA, 2-17: softmax, 18-21: pair norms
+constexpr int kPvWarp = 2 + kSoftmaxWarps + kNormWarps;          // the warp that issues the P V products
+constexpr int kThreads = (kPvWarp + 1) * 32;   // warp 0: TMA, 1: S products, 2-17: softmax, 18-21: pair norms, 22: P V products
 constexpr float kRescaleGap = 8.f;         // log2 units
 constexpr int kSBufs = 3;                  // logit / P' buffers in tensor memory
 
 struct Misc {
-  uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[kSBufs], pready[kSBufs][2], ofull[2], stabdone[2], qfull;
+  uint64_t kfull[2], vfull[2], kfree[2], vfree[2], sfull[kSBufs], pready[kSBufs][2], pvdone[kSBufs], ofull[2], stabdone[2], qfull;
   uint32_t tmem_base;
   int abort_flag, wait_us;                 // (adjacent: the bounded waits read both through one pointer)
   float rowmax[2][2][2][kTile];            // per team, tile parity, column half and query row: that thread's maximum logit
@@ -206,6 +207,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     }
     for (int b = 0; b < kSBufs; ++b) {
       mbar_init(&misc->sfull[b], 1);
+      mbar_init(&misc->pvdone[b], 1);
       // P' is handed over in two halves (the last and the first 32 slots of every thread's 64), so
       // that the P V products of one half run while the other half is still being written
       for (int hf = 0; hf < 2; ++hf) mbar_init(&misc->pready[b][hf], kSoftmaxWarps / 2);
@@ -269,45 +271,47 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
       }
     }
   } else if (warp == 1) {
-    // ================================================================ MMA issuer
+    // ================================================================ issuer of the S products
+    // Two threads in two warps feed the tensor pipe, one the logits and one the P V products: a
+    // single thread needed 110-125 cycles per product here (it shares its scheduler with four busy
+    // softmax warps), the pipe 66, and the softmax teams waited for their logits.
     if (lane == 0) {
-      // One thread feeds the tensor pipe, so every instruction between two products counts: the
-      // descriptors are kept as a constant high word and a low word that only needs an addition.
       constexpr uint32_t idesc_s = idesc_bf16(128, 128);                 // Q (K-major) x K tile (K-major)
-      constexpr uint32_t idesc_o = idesc_bf16(128, 128, false, true);    // P' (K-major) x V tile (MN-major)
       const uint64_t qd0 = smem_desc_sw128(smem_u32(smem + kSmemQ), 16, 1024);
       const uint64_t kd0 = smem_desc_sw128(smem_u32(smem + kSmemStage), 16, 1024);
-      const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + kSmemStage + kOperand), kHalf, 1024);
-      const uint32_t kd_hi = (uint32_t)(kd0 >> 32), vd_hi = (uint32_t)(vd0 >> 32);
-      const uint32_t qd_lo = (uint32_t)qd0, kd_lo0 = (uint32_t)kd0, vd_lo0 = (uint32_t)vd0;   // stage 0; stage 1 is kStage / 16 further
-      // The logits of tile li go to buffer li mod 3, which last held P' of tile li - 3: the products
-      // that read it were issued by this thread before.  With three buffers the logits run two
-      // tiles ahead of the P V products, so that a softmax team that has finished tile li finds the
-      // logits of its next tile, li + 2, already formed instead of waiting for P V of tile li.
-      auto issue_s = [&](int li) -> bool {
+      const uint32_t kd_hi = (uint32_t)(kd0 >> 32), qd_lo = (uint32_t)qd0, kd_lo0 = (uint32_t)kd0;   // stage 1 is kStage / 16 further
+      // The logits of tile li go to buffer li mod 3, which last held P' of tile li - 3: its P V products
+      // must be complete (pvdone).  With three buffers the logits run up to three tiles ahead, so that a
+      // softmax team that has finished a tile finds the logits of its next one already formed.
+      bool ok = mbar_wait(&misc->qfull, 0, abort_flag);
+      for (int li = 0; ok && li < my_tiles; ++li) {
         const int s = li & 1, k = li >> 1;                 // K stage and its use count
-        if (!mbar_wait(&misc->kfull[s], k & 1, abort_flag)) return false;
+        const int b = li % kSBufs, u = li / kSBufs;        // logit buffer and its use count
+        if (u > 0 && !mbar_wait(&misc->pvdone[b], (u - 1) & 1, abort_flag)) break;
+        if (!mbar_wait(&misc->kfull[s], k & 1, abort_flag)) break;
         tc_fence_after();
-        const uint32_t kd_lo = kd_lo0 + s * (kStage >> 4), ds = tmem + (uint32_t)(li % kSBufs) * 128;
+        const uint32_t kd_lo = kd_lo0 + s * (kStage >> 4), ds = tmem + (uint32_t)b * 128;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           const uint32_t o = ((kk >> 2) * kHalf + (kk & 3) * 32) >> 4;
           if (kk == 0) umma_ss<false>(ds, qd_lo, kd_hi, kd_lo, kd_hi, idesc_s);
           else umma_ss<true>(ds, qd_lo + o, kd_hi, kd_lo + o, kd_hi, idesc_s);
         }
-        tc_commit(&misc->sfull[li % kSBufs]);
+        tc_commit(&misc->sfull[b]);
         tc_commit(&misc->kfree[s]);
-        return true;
-      };
-      bool ok = mbar_wait(&misc->qfull, 0, abort_flag);
-      ok = ok && issue_s(0);
-      if (ok && my_tiles > 1) ok = issue_s(1);
+      }
+    }
+  } else if (warp == kPvWarp) {
+    // ================================================================ issuer of the P V products
+    if (lane == 0) {
+      constexpr uint32_t idesc_o = idesc_bf16(128, 128, false, true);    // P' (K-major) x V tile (MN-major)
+      const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + kSmemStage + kOperand), kHalf, 1024);
+      const uint32_t vd_hi = (uint32_t)(vd0 >> 32), vd_lo0 = (uint32_t)vd0;
+      bool ok = true;
       for (int li = 0; ok && li < my_tiles; ++li) {
-        // the logits of the tile after next are queued before this tile's P V products
-        if (li + 2 < my_tiles) ok = issue_s(li + 2);
         const int s = li & 1, ph = (li >> 1) & 1;          // V stage and its phase
         const int b = li % kSBufs, bph = (li / kSBufs) & 1; // P' buffer and its phase
-        if (ok && !mbar_wait(&misc->vfull[s], ph, abort_flag)) ok = false;
+        if (!mbar_wait(&misc->vfull[s], ph, abort_flag)) ok = false;
         const uint32_t vd_lo = vd_lo0 + s * (kStage >> 4), ps = tmem + (uint32_t)b * 128;
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
@@ -333,11 +337,12 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
         if (ok) {
           tc_commit(&misc->ofull[s]);
           tc_commit(&misc->vfree[s]);
+          tc_commit(&misc->pvdone[b]);
         }
       }
     }
   } else if (warp >= 2 + kSoftmaxWarps) {
-    // ================================================================ pair-norm warps
+    // ================================================================ pair-norm warps (18-21)
     if (norm_k || norm_v) {
       const int nw = warp - (2 + kSoftmaxWarps);                 // rows [32 nw, 32 nw + 32) of every tile
       const int off = tab.off;
