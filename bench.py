@@ -89,9 +89,9 @@ class ClockSampler(threading.Thread):
 # carries over to a full launch).  Each entry names the kernel source it was taken on: once that
 # file changes, the figure is stale and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "hessian_stats": (1.06, "kvs_stats_tc.cu", "6aa90ad0e6355729"),
-    "attn_partials": (1.08, "kvs_flash_tc.cu", "f06c90efce487272"),
-    "merge_compact": (0.98, "kvs_compact.cu", "b399e8259464a6e9"),
+    "hessian_stats": (1.12, "kvs_stats_tc.cu", "ede5c0691e1047a3"),
+    "attn_partials": (1.08, "kvs_flash_tc.cu", "b4db793774d8087b"),
+    "merge_compact": (0.98, "kvs_compact.cu", "fd795ce5ffcec3da"),
 }
 
 
