@@ -108,3 +108,39 @@ def test_append_and_merge_rejects_bad_arguments_before_any_cuda_call(lib):
     assert lib.kvs_append_and_merge(*args(16, one)) == 1           # NULL chunk / no room behind 4096 slots
     assert lib.kvs_append_and_merge(*args(0, None)) == 1           # NULL cur_len
     assert b"" != lib.kvs_last_error_string()
+
+
+def test_variant_entry_points_reject_bad_arguments_before_any_cuda_call(lib):
+    """Exact-weight, per-head and similarity entry points: host-detectable errors come back as codes
+    with nothing enqueued (all pointers here are NULL or host dummies, so a launch would fault)."""
+    p = _params()
+    one = (ctypes.c_int32 * 1)(4096)
+    # weight_mode must be 1 or 2; e_win must not be NULL
+    args = lambda mode: (ctypes.byref(p), None, None, None, None, None, mode, one, one, 4096, one, None,
+                         ctypes.c_size_t(0), None, None)
+    assert lib.kvs_merge_layer_exact(*args(0)) == 1
+    assert lib.kvs_merge_layer_exact(*args(3)) == 1
+    assert lib.kvs_merge_layer_exact(*args(1)) == 1          # NULL caches
+    # per-head lengths need heads that tile the sequence stride
+    bad = _params(batch=2, k_stride_b=9 * 4096 * 128)
+    out = ctypes.c_size_t(0)
+    assert lib.kvs_workspace_size_per_head(ctypes.byref(bad), 4096, 0, ctypes.byref(out)) == 2
+    good = _params(batch=2)
+    assert lib.kvs_workspace_size_per_head(ctypes.byref(good), 4096, 0, ctypes.byref(out)) == 0
+    whole = kb.kvs_workspace_size(good, 4096)
+    assert out.value > 0 and out.value != whole               # sized for 16 one-head sequences
+    # similarity: sizes, strides, alignment
+    x = ctypes.c_void_p(0x1000)
+    f = lib.kvs_adjacent_cosine
+    assert f(None, 1, 8, 4096, 8 * 4096 * 128, 4096 * 128, 128, one, x, None) == 1
+    assert f(x, 0, 8, 4096, 8 * 4096 * 128, 4096 * 128, 128, one, x, None) == 1
+    assert f(x, 1, 8, 4096, 8 * 4096 * 128, 4096 * 128, 64, one, x, None) == 1       # row stride < 128
+    assert f(x, 1, 8, 4096, 8 * 4096 * 128, 4096 * 128 + 4, 128, one, x, None) == 1  # stride not a multiple of 8
+    assert f(ctypes.c_void_p(0x1004), 1, 8, 4096, 8 * 4096 * 128, 4096 * 128, 128, one, x, None) == 1
+    big = (ctypes.c_int32 * 1)(5000)
+    assert f(x, 1, 8, 4096, 8 * 4096 * 128, 4096 * 128, 128, big, x, None) == 1      # seq_len > n_max
+    # the wait hook takes three bits
+    assert lib.kvs_debug_set_wait(0, 8) == 1
+    assert lib.kvs_debug_set_wait(0, 0) == 0
+    # the probe wants positive sizes
+    assert lib.kvs_probe_sfu(0, 10, x, None, None) == 1
