@@ -89,7 +89,7 @@ class ClockSampler(threading.Thread):
 # carries over to a full launch).  Each entry names the kernel source it was taken on: once that
 # file changes, the figure is stale and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "hessian_stats": (1.12, "kvs_stats_tc.cu", "ede5c0691e1047a3"),
+    "hessian_stats": (1.12, "kvs_stats_tc.cu", "583c16dcb28baa30"),
     "attn_partials": (1.08, "kvs_flash_tc.cu", "b4db793774d8087b"),
     "merge_compact": (0.98, "kvs_compact.cu", "fd795ce5ffcec3da"),
 }

@@ -57,37 +57,14 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parit
       : "memory");
   return ok != 0;
 }
-// Up to `tries` attempts in one tight loop (each attempt may itself sleep in hardware for a short
-// while).  Returns whether the phase completed.
-__device__ __forceinline__ bool mbar_poll(uint64_t* bar, uint32_t parity, uint32_t tries) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
-      "mov.u32 n, %3;\n"
-      "KVS_POLL:\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "@p bra KVS_POLL_DONE;\n\t"
-      "sub.u32 n, n, 1;\n\t"
-      "setp.ne.u32 q, n, 0;\n\t"
-      "@q bra KVS_POLL;\n"
-      "KVS_POLL_DONE:\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity), "r"(tries)
-      : "memory");
-  return ok != 0;
-}
 // Bounded wait: false once the time limit has passed (or when another role already flagged an
 // abort).  `ctl` points at two ints in shared memory: ctl[0] is the CTA's abort flag, ctl[1] the
-// time limit of one wait in microseconds (one second unless the host asked otherwise).
-// These kernels are chains of hand-offs, so the wake-up latency of a wait counts: a wait on the
-// critical path (`eager`) first polls in a tight loop for a few hundred cycles; after that, and
-// for a role that runs ahead of the others anyway, the hardware suspends the thread between attempts.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* ctl, bool eager = false) {
+// time limit of one wait in microseconds (one second unless the host asked otherwise).  Between
+// attempts the hardware may suspend the thread (suspend-time hint): in these kernels that measured
+// better than a tight polling loop (which takes issue slots from the warps that have work) and far
+// better than nanosleep (wake-up latency on every hand-off).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* ctl) {
   if (mbar_try_wait(bar, parity)) return true;
-  // (an eager waiter polls for a short while only: a long wait in a tight loop would take issue
-  // slots from the warps that have work to do)
-  if (eager && mbar_poll(bar, parity, 48)) return true;
   const uint64_t t0 = globaltimer_ns();
   while (!mbar_try_wait_hint(bar, parity, 10000u)) {
     if (ctl[0]) return false;

@@ -63,12 +63,12 @@ struct Misc {
 constexpr int kSmemBytes = kSmemMisc + (int)sizeof(Misc);
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 
-// One lane polls, the warp follows.  The statistics warps wait on the critical path of a tile
-// (the tensor core has usually just finished): they poll instead of letting the hardware suspend
-// them, whose wake-up costs several hundred cycles.
+// One lane waits, the warp follows.  (Polling in a tight loop instead of letting the hardware
+// suspend the lane measured the same: the statistics warps' waits, about 250 cycles per half, are
+// real waits for the tensor core, not wake-up latency.)
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int lane) {
   int ok = 1;
-  if (lane == 0) ok = mbar_wait(bar, parity, abort_flag, true) ? 1 : 0;
+  if (lane == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
   return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 __device__ __forceinline__ void warp_arrive(uint64_t* bar, int lane) {
