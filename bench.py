@@ -380,7 +380,34 @@ def run_stream(args):
     launches = kb.lib().kvs_launch_count() - l0
     assert status.item() == 0 and new_len == bud
     ms = total / args.steps
-    rec = {"metric": "stream_step_ms", "value": ms, "unit": "ms", "higher_is_better": False,
+    # where the step's time goes, kernel by kernel (two extra steps with per-launch events)
+    kb.kvs_profile_begin()
+    for _ in range(2):
+        restore(); step()
+    torch.cuda.synchronize()
+    kernels_ms = {k: v[0] / 2 for k, v in kb.kvs_profile_end().items() if v[1] > 0}
+    # the same step replayed from a CUDA graph: what is left when the host's launch work is gone
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        restore(); step()                      # (first call on the capturing stream happens outside the capture)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    restore()
+    with torch.cuda.graph(graph):
+        step()
+    graph_total = 0.0
+    for _ in range(args.steps):
+        restore()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); graph.replay(); b.record(); b.synchronize()
+        graph_total += a.elapsed_time(b)
+    assert status.item() == 0
+    graph_ms = graph_total / args.steps
+    del graph
+    rec = {"metric": "stream_step_ms", "value": ms, "graph_replay_ms": graph_ms, "kernels_ms": kernels_ms,
+           "unit": "ms", "higher_is_better": False,
            "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup), "data": "synthetic",
            "dtype": "bf16", "gpu_launches": int(launches),
            "chunk_tokens_per_sec_per_layer": B * chunk / (ms * 1e-3),

@@ -389,6 +389,7 @@ kvs_status_t enqueue_round_stats(const Common& c, const CacheView& view, const v
   CUDA_TRY(launch(KVS_K_STATS, c.st, [&] {
     return kvs_launch_stats_tc(ta, tab, c.tmKp, c.tmVp, c.tmQ, c.weight_mode ? c.tmE : c.tmOhi, c.tmOlo, c.st);
   }));
+  g_launches.fetch_add(1, std::memory_order_relaxed);   // (two kernels behind that call: the statistics and their finalize)
 
   if (do_select) {
     SelectArgs se;

@@ -182,40 +182,30 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
           tma_prefetch_5d(tm, hf * 64, par_r, rho_r0 + p0, h, sr.b);
         }
       };
+      // K of a tile is free again before its Vsum rows are (the last logits come before the last T
+      // product), and the K of the tile after that cannot be free before these Vsum rows have been
+      // used: the requests go out in the fixed order K, V, K, V, ... behind blocking (bounded) waits
       int kli = 0, vli = 0;
-      uint64_t t0 = globaltimer_ns();
-      while (kli < my_tiles || vli < my_tiles) {
-        bool progress = false;
-        if (kli < my_tiles && mbar_try_wait(&misc->kfree, (kli & 1) ^ 1)) {
-          const int p0 = (t_begin + kli) * kPairs;
-          if (!withhold_k) {
-            mbar_expect_tx(&misc->kfull, 2 * kOperand);
-            for (int hf = 0; hf < 2; ++hf) {
-              tma_load_5d(smem + kSmemKl + hf * kHalf, &tmKp, &misc->kfull, hf * 64, par_l, rho_l0 + p0, h, sr.b);
-              tma_load_5d(smem + kSmemKr + hf * kHalf, &tmKp, &misc->kfull, hf * 64, par_r, rho_r0 + p0, h, sr.b);
-            }
-          }
-          if (kli + 1 < my_tiles) prefetch(kli + 1, false);
-          ++kli;
-          progress = true;
-        }
-        if (vli < my_tiles && mbar_try_wait(&misc->vfree, (vli & 1) ^ 1)) {
-          const int p0 = (t_begin + vli) * kPairs;
-          mbar_expect_tx(&misc->vfull, 2 * kOperand);
+      for (int li = 0; li < my_tiles; ++li) {
+        const int p0 = (t_begin + li) * kPairs;
+        if (!mbar_wait(&misc->kfree, (li & 1) ^ 1, abort_flag)) break;
+        if (!withhold_k) {
+          mbar_expect_tx(&misc->kfull, 2 * kOperand);
           for (int hf = 0; hf < 2; ++hf) {
-            tma_load_5d(smem + kSmemVl + hf * kHalf, &tmVp, &misc->vfull, hf * 64, par_l, rho_l0 + p0, h, sr.b);
-            tma_load_5d(smem + kSmemVr + hf * kHalf, &tmVp, &misc->vfull, hf * 64, par_r, rho_r0 + p0, h, sr.b);
+            tma_load_5d(smem + kSmemKl + hf * kHalf, &tmKp, &misc->kfull, hf * 64, par_l, rho_l0 + p0, h, sr.b);
+            tma_load_5d(smem + kSmemKr + hf * kHalf, &tmKp, &misc->kfull, hf * 64, par_r, rho_r0 + p0, h, sr.b);
           }
-          if (vli + 1 < my_tiles) prefetch(vli + 1, true);
-          ++vli;
-          progress = true;
         }
-        if (progress) {
-          t0 = globaltimer_ns();
-        } else {
-          if (*abort_flag) break;
-          if (globaltimer_ns() - t0 > (uint64_t)(uint32_t)misc->wait_us * 1000ull) { *abort_flag = 1; break; }
+        if (li + 1 < my_tiles) prefetch(li + 1, false);
+        ++kli;
+        if (!mbar_wait(&misc->vfree, (li & 1) ^ 1, abort_flag)) break;
+        mbar_expect_tx(&misc->vfull, 2 * kOperand);
+        for (int hf = 0; hf < 2; ++hf) {
+          tma_load_5d(smem + kSmemVl + hf * kHalf, &tmVp, &misc->vfull, hf * 64, par_l, rho_l0 + p0, h, sr.b);
+          tma_load_5d(smem + kSmemVr + hf * kHalf, &tmVp, &misc->vfull, hf * 64, par_r, rho_r0 + p0, h, sr.b);
         }
+        if (li + 1 < my_tiles) prefetch(li + 1, true);
+        ++vli;
       }
       if (*abort_flag) {
         // drain: give the copies already issued a bounded time to land before the CTA leaves

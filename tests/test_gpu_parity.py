@@ -889,3 +889,55 @@ def test_exact_weights_with_a_supplied_gradient(kb):
     E2 = wl.f32_to_bf16_bits(np.random.default_rng(76).standard_normal(d2["q_win"].shape).astype(np.float32))
     for mode in (1, 2):
         *_, flips = full_pass_vs_oracle(kb, w2, d2, exact=(E2, mode))
+
+
+def test_merge_pass_replayed_from_a_cuda_graph(kb):
+    """The merge pass and the decode check, captured once into a CUDA graph and replayed twice on
+    a restored cache, must give bit for bit what the same calls gave when launched directly:
+    everything a call needs on the device travels as kernel arguments or lives in the caller's
+    workspace, nothing depends on host work at launch time."""
+    import torch
+    w = _small(seed=31, seq_lens=(700, 389), budgets=(256, 120), n_decode=4)
+    data = wl.make_layer(w)
+    dev, p, ws = _setup(kb, w, data)
+    B, Hq, T = w.batch, w.n_q_heads, w.n_decode
+    K0, V0, C0 = dev["K"].clone(), dev["V"].clone(), dev["counts"].clone()
+    out = torch.zeros((B, Hq, T, 128), dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def restore():
+        dev["K"].copy_(K0); dev["V"].copy_(V0); dev["counts"].copy_(C0); out.zero_()
+
+    def run():
+        new_len = kb.kvs_merge_layer(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], list(w.seq_lens),
+                                     list(w.budgets), ws, status_dev=status)
+        kb.kvs_decode_attn(p, dev["q_new"], dev["K"], dev["V"], dev["counts"], new_len, out, ws)
+        return new_len
+
+    # launched directly (also the first call on this device, outside any capture)
+    new_len = run()
+    torch.cuda.synchronize()
+    assert status.item() == 0 and new_len == list(w.budgets)
+    ref = [tl.bits_of(dev["K"]), tl.bits_of(dev["V"]), dev["counts"].cpu().numpy(), tl.bits_of(out)]
+    # once more on a side stream, then the capture
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        restore(); run()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    restore()
+    with torch.cuda.graph(graph):
+        assert run() == new_len
+    for _ in range(2):
+        restore()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        got = [tl.bits_of(dev["K"]), tl.bits_of(dev["V"]), dev["counts"].cpu().numpy(), tl.bits_of(out)]
+        for b in range(B):
+            m = new_len[b]
+            for g, r in zip(got[:3], ref[:3]):
+                assert np.array_equal(g[b, :, :m], r[b, :, :m])
+        assert np.array_equal(got[3], ref[3])
