@@ -147,6 +147,31 @@ def measure_sfu_peak(kb, torch, local):
             "how": "kvs_probe_sfu: 296 CTAs x 1024 threads x 640000 ex2.approx/sqrt.approx, best launch of 0.6 s"}
 
 
+def measure_operand_feed(kb, torch):
+    """Cycles per tensor-core product when both operands come from shared memory, from the library's
+    probe on every SM at once: 128 x N x 16 for N = 64 (the statistics kernel's shape; also with
+    the A slice of every second product taken from the collector buffer), 128 and 256.  A product
+    reads 4 KiB of A and N * 32 bytes of B; the narrow ones are bound by that read, which gives
+    the shared-memory bytes per cycle an SM delivers to the tensor core."""
+    blocks, products = 148, 2048
+    out = {}
+    for key, n_cols, reuse in (("n64", 64, False), ("n64_reuse_a", 64, True), ("n128", 128, False), ("n256", 256, False)):
+        cyc = torch.zeros(blocks, dtype=torch.int64, device="cuda")
+        best = None
+        for _ in range(3):
+            kb.kvs_probe_mma(blocks, n_cols, reuse, products, cyc)
+            torch.cuda.synchronize()
+            c = cyc.cpu().numpy()
+            if (c <= 0).any():
+                return None
+            v = float(c.max()) / products
+            best = v if best is None else min(best, v)
+        out[key] = best
+    out["bytes_per_cycle"] = (4096 + 64 * 32) / out["n64"]
+    out["how"] = "kvs_probe_mma: 148 CTAs x 2048 products each, slowest CTA, best of 3 launches"
+    return out
+
+
 def plan_rounds(w, oracle_free=True):
     """(n_r, off, P, R) per round for each sequence, from the closed-form schedule."""
     out = []
@@ -190,8 +215,14 @@ def work_counts(w, n_layers):
     el_attn = sum(n for pl in plans for (n, _, _, _) in pl) * units * M
     el_stats = sum(2 * P for pl in plans for (_, _, P, _) in pl) * units * M
     return {
-        "attn_partials": {"elements": el_attn, "flops": 512 * el_attn, "flops_with_split": 768 * el_attn, "sfu_ops": 1.0 * el_attn},
-        "hessian_stats": {"elements": el_stats, "flops": 512 * el_stats, "flops_with_split": 768 * el_stats, "sfu_ops": 2.5 * el_stats},
+        # shared-memory bytes per (query, slot) AS THE KERNELS ARE BUILT (not a property of the method): a
+        # tile of 128 x 128 of them costs the attention kernel 24 products of 8 resp. 4 KiB of operand reads
+        # plus 64 KiB of TMA fill, the statistics kernel (128 pairs = 256 slots) 96 products of 6 KiB, 128 KiB
+        # of TMA fill and 128 KiB of per-query constants
+        "attn_partials": {"elements": el_attn, "flops": 512 * el_attn, "flops_with_split": 768 * el_attn, "sfu_ops": 1.0 * el_attn,
+                          "smem_bytes": (8 * 8192 + 16 * 4096 + 65536) / 16384 * el_attn},
+        "hessian_stats": {"elements": el_stats, "flops": 512 * el_stats, "flops_with_split": 768 * el_stats, "sfu_ops": 2.5 * el_stats,
+                          "smem_bytes": (96 * 6144 + 131072 + 131072) / 32768 * el_stats},
     }
 
 
@@ -688,6 +719,9 @@ def main():
     sfu = measure_sfu_peak(kb, torch, local)
     clk_scale = (clocks["sm_mhz"] / sfu["sm_mhz"]) if (clocks.get("sm_mhz") and sfu.get("sm_mhz")) else 1.0
     sfu_rate = sfu["ops_per_s"] * clk_scale
+    # shared-memory bandwidth towards the tensor core, measured now; at the SM clock the step ran at
+    feed = measure_operand_feed(kb, torch)
+    smem_Bps = feed["bytes_per_cycle"] * clocks["sm_mhz"] * 1e6 * 148 if (feed and clocks.get("sm_mhz")) else None
     per_kernel = {}
     for k, v in kinds.items():
         ms_k = v[0] / n_prof
@@ -711,6 +745,17 @@ def main():
                 "kernel_ms_per_step": top_ms, "avg_launch_us": 1e3 * top_ms / top_launches,
                 "algorithmic_bytes_per_launch": alg.get(top, 0) / top_launches,
                 "sfu_probe": sfu, "per_kernel": per_kernel}
+    # Beside the three: the shared-memory traffic of the kernel as built (operand reads of the tensor
+    # core, TMA fills, per-query constants) against the bandwidth the probe measured.  It is a floor of
+    # this design, not of the method, so it does not take part in `bound`; it says how much room is
+    # left without a design that moves fewer shared-memory bytes per (query, slot).
+    if smem_Bps and work.get(top, {}).get("smem_bytes"):
+        f = work[top]["smem_bytes"] / smem_Bps * 1e3
+        roofline["operand_feed"] = {"floor_ms": f, "frac": f / top_ms, "achieved": work[top]["smem_bytes"] / (top_ms * 1e-3) / 1e12,
+                                    "peak": smem_Bps / 1e12, "unit": "TB/s (shared memory, all SMs)", "probe": feed,
+                                    "per_kernel": {k: {"floor_ms": work[k]["smem_bytes"] / smem_Bps * 1e3,
+                                                       "frac": work[k]["smem_bytes"] / smem_Bps * 1e3 / per_kernel[k]["ms_per_step"]}
+                                                   for k in per_kernel if work.get(k, {}).get("smem_bytes")}}
     # the whole step against the same three floors (sums over the kernels)
     step_work = {key: sum(wk[key] for wk in work.values()) for key in ("flops", "flops_with_split", "sfu_ops")}
     roofline["step"] = {"ms_per_step": ms_per_step,

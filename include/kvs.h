@@ -325,6 +325,21 @@ kvs_status_t kvs_debug_set_wait(uint32_t limit_us, uint32_t withhold);
 kvs_status_t kvs_probe_sfu(int32_t blocks, int32_t iters, float* sink_dev, uint64_t* ops, void* cuda_stream);
 
 /*
+ * Measurement aid: what one tensor-core product costs when both of its operands are read from
+ * shared memory, which is what bounds the narrow products of the statistics kernel (Eqs.
+ * c11_def-c12_def need S = K Q^T and T = Vsum O^T per candidate pair; the pair members sit on the
+ * 128 accumulator lanes, so every product re-reads a 128 x 16 slice of K or Vsum).  Launches
+ * `blocks` CTAs; one warp of each issues `products` (a multiple of 8, at most 2^20) back-to-back
+ * bf16 products of shape 128 x n_cols x 16, n_cols in {16, 32, 64, 128, 256}, on zero-filled
+ * operands, and writes the cycles from the first issue to the completion of the last into
+ * cycles_dev[block] (-1 if its bounded wait ran out).  With reuse_a != 0 consecutive products
+ * share their A slice in twos and the second takes it from the tensor core's collector buffer.
+ *   cycles_dev   DEVICE int64[blocks]
+ */
+kvs_status_t kvs_probe_mma(int32_t blocks, int32_t n_cols, int32_t reuse_a, int32_t products, int64_t* cycles_dev,
+                           void* cuda_stream);
+
+/*
  * Per-kernel device timing for benchmarks.  Between kvs_profile_begin() and
  * kvs_profile_end() every kernel launch of this library is bracketed by CUDA events on the
  * launching stream.  kvs_profile_end() synchronises those events and returns, for each

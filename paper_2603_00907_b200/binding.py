@@ -25,7 +25,7 @@ EXPORTS = ["kvs_version", "kvs_last_error_string", "kvs_launch_count", "kvs_roun
            "kvs_compact_static", "kvs_static_scratch_bytes", "kvs_append_and_merge",
            "kvs_debug_set_wait", "kvs_adjacent_cosine",
            "kvs_workspace_size_per_head", "kvs_merge_layer_per_head", "kvs_decode_attn_per_head",
-           "kvs_merge_layer_exact", "kvs_window_stats_exact", "kvs_probe_sfu"]
+           "kvs_merge_layer_exact", "kvs_window_stats_exact", "kvs_probe_sfu", "kvs_probe_mma"]
 
 
 class KvsError(RuntimeError):
@@ -64,7 +64,7 @@ def lib() -> ctypes.CDLL:
                      "kvs_decode_attn", "kvs_window_stats", "kvs_profile_begin", "kvs_profile_end",
                      "kvs_compact_static", "kvs_append_and_merge", "kvs_debug_set_wait", "kvs_adjacent_cosine",
                      "kvs_workspace_size_per_head", "kvs_merge_layer_per_head", "kvs_decode_attn_per_head",
-                     "kvs_merge_layer_exact", "kvs_window_stats_exact", "kvs_probe_sfu"):
+                     "kvs_merge_layer_exact", "kvs_window_stats_exact", "kvs_probe_sfu", "kvs_probe_mma"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -288,6 +288,13 @@ def kvs_probe_sfu(blocks: int, iters: int, sink) -> int:
     ops = ctypes.c_uint64(0)
     _check(lib().kvs_probe_sfu(ctypes.c_int32(blocks), ctypes.c_int32(iters), _ptr(sink), ctypes.byref(ops), _stream()))
     return int(ops.value)
+
+
+def kvs_probe_mma(blocks: int, n_cols: int, reuse_a: bool, products: int, cycles) -> None:
+    """Launch the operand-feed probe on the current stream; `cycles` is a device int64[blocks] that
+    receives each CTA's elapsed cycles for its `products` tensor-core products (-1: wait ran out)."""
+    _check(lib().kvs_probe_mma(ctypes.c_int32(blocks), ctypes.c_int32(n_cols), ctypes.c_int32(1 if reuse_a else 0),
+                               ctypes.c_int32(products), _ptr(cycles), _stream()))
 
 
 def kvs_profile_begin() -> None:

@@ -1000,6 +1000,19 @@ kvs_status_t kvs_probe_sfu(int32_t blocks, int32_t iters, float* sink_dev, uint6
   return KVS_OK;
 }
 
+kvs_status_t kvs_probe_mma(int32_t blocks, int32_t n_cols, int32_t reuse_a, int32_t products, int64_t* cycles_dev,
+                           void* cuda_stream) {
+  const bool n_ok = n_cols == 16 || n_cols == 32 || n_cols == 64 || n_cols == 128 || n_cols == 256;
+  if (blocks <= 0 || blocks > 65535 || !n_ok || products < 8 || products > (1 << 20) || (products & 7) || !cycles_dev)
+    return fail(KVS_ERR_INVALID_ARG, "bad probe argument");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  CUDA_TRY(launch(KVS_K_MISC, st, [&] {
+    return kvs_launch_mma_probe(blocks, n_cols, reuse_a ? 1 : 0, products, g_wait_us.load(),
+                                reinterpret_cast<long long*>(cycles_dev), st);
+  }));
+  return KVS_OK;
+}
+
 kvs_status_t kvs_profile_begin(void) {
   g_prof.on = true;
   g_prof.recs.clear();

@@ -231,7 +231,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     // one thread streams both rings.  Stages come free in a fixed order (the logits of tile t + 1 are
     // queued before the P V products of tile t), so the thread sleeps on one barrier at a time:
     // K(0), K(1), V(0), K(2), V(1), ...
-    if (lane == 0) {
+    if (elect_one()) {
       prefetch_tmap(&tmK); prefetch_tmap(&tmV); prefetch_tmap(&tmQ);
       mbar_expect_tx(&misc->qfull, kOperand);
       for (int hf = 0; hf < 2; ++hf)
@@ -275,7 +275,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     // Two threads in two warps feed the tensor pipe, one the logits and one the P V products: a
     // single thread needed 110-125 cycles per product here (it shares its scheduler with four busy
     // softmax warps), the pipe 66, and the softmax teams waited for their logits.
-    if (lane == 0) {
+    if (elect_one()) {
       constexpr uint32_t idesc_s = idesc_bf16(128, 128);                 // Q (K-major) x K tile (K-major)
       const uint64_t qd0 = smem_desc_sw128(smem_u32(smem + kSmemQ), 16, 1024);
       const uint64_t kd0 = smem_desc_sw128(smem_u32(smem + kSmemStage), 16, 1024);
@@ -303,7 +303,7 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
     }
   } else if (warp == kPvWarp) {
     // ================================================================ issuer of the P V products
-    if (lane == 0) {
+    if (elect_one()) {
       constexpr uint32_t idesc_o = idesc_bf16(128, 128, false, true);    // P' (K-major) x V tile (MN-major)
       const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + kSmemStage + kOperand), kHalf, 1024);
       const uint32_t vd_hi = (uint32_t)(vd0 >> 32), vd_lo0 = (uint32_t)vd0;

@@ -176,6 +176,10 @@ struct KvsPerDeviceOnce {
 
 // Special-function probe: `blocks` CTAs of 1024 threads, 16 * iters operations per thread.
 cudaError_t kvs_launch_sfu_probe(int blocks, int iters, float* sink, cudaStream_t st);
+// Operand-feed probe: `blocks` CTAs, each `products` (a multiple of 8) tcgen05 products of shape
+// 128 x n_cols x 16 with both operands in shared memory; cycles[block] = elapsed cycles or -1.
+cudaError_t kvs_launch_mma_probe(int blocks, int n_cols, int reuse_a, int products, uint32_t limit_us,
+                                 long long* cycles, cudaStream_t st);
 
 // ----------------------------------------------------------------------------- device helpers
 #ifdef __CUDACC__

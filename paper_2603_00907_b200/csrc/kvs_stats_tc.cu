@@ -164,7 +164,7 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
 
   if (warp == 0) {
     // ================================================================ TMA producer
-    if (lane == 0) {
+    if (elect_one()) {
       prefetch_tmap(&tmKp); prefetch_tmap(&tmVp); prefetch_tmap(&tmQ); prefetch_tmap(&tmOhi); prefetch_tmap(&tmOlo);
       mbar_expect_tx(&misc->qfull, (kExact ? 2 : 3) * kOperand);
       for (int hf = 0; hf < 2; ++hf) {
@@ -216,7 +216,7 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
   } else if (warp < kFirstStat) {
     // ================================================================ product issuers
     // warp 1 issues the chains of the left pair members (S_l, T_l), warp 2 those of the right ones
-    if (lane == 0) {
+    if (elect_one()) {
       const bool right = warp != 1;
       // descriptors are kept as a constant high word and low words that only need an addition per product
       constexpr uint32_t idesc = idesc_bf16(kPairs, kQH);
@@ -297,7 +297,7 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
       const float2 n2il2 = make_float2(n2il, n2il), n2ir2 = make_float2(n2ir, n2ir);
       const float2 icl2 = make_float2(icl, icl), icr2 = make_float2(icr, icr);
       const float2 r2l2 = make_float2(r2l, r2l), r2r2 = make_float2(r2r, r2r), pc2 = make_float2(pc, pc);
-      const float2 m42 = make_float2(-4.f, -4.f);
+      const float2 four2 = make_float2(4.f, 4.f), n4il2 = make_float2(2.f * n2il, 2.f * n2il), n4ir2 = make_float2(2.f * n2ir, 2.f * n2ir);
       bool broken = false;
       for (int hq = 0; hq < nh; ++hq) {
         if (!warp_wait(&misc->tfull[hq], li & 1, abort_flag, lane)) { broken = true; break; }
@@ -345,9 +345,8 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
               const float2 dr = __ffma2_rn(tr, n2ir2, __fadd2_rn(r2r2, hq2));
               sN1l = __ffma2_rn(gl, make_float2(fast_sqrt(fabsf(dl.x)), fast_sqrt(fabsf(dl.y))), sN1l);
               sN1r = __ffma2_rn(gr, make_float2(fast_sqrt(fabsf(dr.x)), fast_sqrt(fabsf(dr.y))), sN1r);
-              // <vbar_l + vbar_r, o> - |o|^2, then |vbar_l + vbar_r - 2 o|^2
-              const float2 u = __fadd2_rn(__ffma2_rn(tl, icl2, __fmul2_rn(tr, icr2)), make_float2(-hq2.x, -hq2.y));
-              const float2 d12 = __ffma2_rn(u, m42, pc2);
+              // |vbar_l + vbar_r - 2 o|^2 = |vbar_l + vbar_r|^2 + 4 |o|^2 - 4 <vbar_l, o> - 4 <vbar_r, o>
+              const float2 d12 = __ffma2_rn(tl, n4il2, __ffma2_rn(tr, n4ir2, __ffma2_rn(hq2, four2, pc2)));
               sN12 = __ffma2_rn(__fmul2_rn(bl, br), make_float2(fast_sqrt(fabsf(d12.x)), fast_sqrt(fabsf(d12.y))), sN12);
             }
           }

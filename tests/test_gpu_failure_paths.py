@@ -223,3 +223,23 @@ def test_odd_capacity_without_protected_suffix_is_refused(kb):
     p1 = kb.make_params(dev["K"], dev["V"], w.n_q_heads, w.window, sink=w.sink, recent=1, causal=False)
     assert kb.kvs_merge_layer(p1, dev["K"], dev["V"], dev["counts"], dev["q_win"], [301], [100], ws) == [100]
     torch.cuda.synchronize()
+
+
+def test_operand_feed_probe_reports_sane_cycles(kb):
+    """The tensor-core operand-feed probe ends by itself and reports what the arithmetic allows at
+    the least: a 128 x 256 x 16 product cannot take fewer than 128 cycles (4096 multiply-adds per
+    cycle), a 128 x 64 x 16 one not fewer than 32; taking the A slice from the collector buffer
+    for every second product must not make the narrow products slower."""
+    import torch
+    blocks, products = 4, 512
+    out = {}
+    for n_cols, reuse in ((256, False), (64, False), (64, True)):
+        cyc = torch.zeros(blocks, dtype=torch.int64, device="cuda")
+        kb.kvs_probe_mma(blocks, n_cols, reuse, products, cyc)
+        torch.cuda.synchronize()
+        c = cyc.cpu().numpy()
+        assert (c > 0).all(), c
+        out[(n_cols, reuse)] = c.max() / products
+    assert 120 <= out[(256, False)] < 400, out
+    assert 30 <= out[(64, False)] < 200, out
+    assert out[(64, True)] <= out[(64, False)] * 1.05, out

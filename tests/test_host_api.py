@@ -144,3 +144,8 @@ def test_variant_entry_points_reject_bad_arguments_before_any_cuda_call(lib):
     assert lib.kvs_debug_set_wait(0, 0) == 0
     # the probe wants positive sizes
     assert lib.kvs_probe_sfu(0, 10, x, None, None) == 1
+    pm = lib.kvs_probe_mma
+    assert pm(1, 48, 0, 64, x, None) == 1           # a column count the products do not come in
+    assert pm(1, 64, 0, 12, x, None) == 1           # not a multiple of 8
+    assert pm(0, 64, 0, 64, x, None) == 1
+    assert pm(1, 64, 0, 64, None, None) == 1
