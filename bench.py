@@ -45,10 +45,33 @@ class ClockSampler(threading.Thread):
 
     def __init__(self, index: int):
         super().__init__(daemon=True)
-        self.index, self.rows, self.proc = index, [], None
+        self.index, self.rows, self.proc, self.halt = index, [], None, False
         self.t_begin = self.t_end = None            # timed region (perf_counter)
 
     def run(self):
+        # NVML read-outs every 20 ms where the Python binding is there (a 0.4 s timed region then gets
+        # some twenty samples), else nvidia-smi's own loop, which delivers a sample every 150-200 ms
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            mx = pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM)
+            bits = [(getattr(pynvml, "nvmlClocksEventReasonHwSlowdown", 0x8), 3),
+                    (getattr(pynvml, "nvmlClocksEventReasonHwThermalSlowdown", 0x40), 4),
+                    (getattr(pynvml, "nvmlClocksEventReasonSwThermalSlowdown", 0x20), 5),
+                    (getattr(pynvml, "nvmlClocksEventReasonSwPowerCap", 0x4), 6)]
+            get_reasons = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                pynvml.nvmlDeviceGetCurrentClocksThrottleReasons
+            while not self.halt:
+                r = get_reasons(h)
+                row = [str(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)), str(mx), "", "", "", "", ""]
+                for bit, col in bits:
+                    row[col] = "Active" if (r & bit) else "Not Active"
+                self.rows.append((time.perf_counter(), row))
+                time.sleep(0.02)
+            return
+        except Exception:
+            pass
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
@@ -60,6 +83,7 @@ class ClockSampler(threading.Thread):
             pass
 
     def stop(self):
+        self.halt = True
         if self.proc is not None:
             self.proc.terminate()
         self.join(timeout=2)
@@ -89,8 +113,8 @@ class ClockSampler(threading.Thread):
 # carries over to a full launch).  Each entry names the kernel source it was taken on: once that
 # file changes, the figure is stale and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "hessian_stats": (1.12, "kvs_stats_tc.cu", "583c16dcb28baa30"),
-    "attn_partials": (1.08, "kvs_flash_tc.cu", "b4db793774d8087b"),
+    "hessian_stats": (1.12, "kvs_stats_tc.cu", "fdd6b1e73179566b"),
+    "attn_partials": (1.08, "kvs_flash_tc.cu", "cfd013b3dd16c78d"),
     "merge_compact": (0.98, "kvs_compact.cu", "fd795ce5ffcec3da"),
 }
 
