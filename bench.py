@@ -780,6 +780,11 @@ def main():
                                     "per_kernel": {k: {"floor_ms": work[k]["smem_bytes"] / smem_Bps * 1e3,
                                                        "frac": work[k]["smem_bytes"] / smem_Bps * 1e3 / per_kernel[k]["ms_per_step"]}
                                                    for k in per_kernel if work.get(k, {}).get("smem_bytes")}}
+    # what the step spends outside the five kernel kinds: small launches (append, clears) and the
+    # gaps between dependent launches
+    all_ms = sum(v[0] for v in prof.values()) / n_prof
+    roofline["misc_kernels_ms_per_step"] = (prof["misc"][0] / n_prof) if "misc" in prof else 0.0
+    roofline["between_launches_ms_per_step"] = ms_per_step - all_ms
     # the whole step against the same three floors (sums over the kernels)
     step_work = {key: sum(wk[key] for wk in work.values()) for key in ("flops", "flops_with_split", "sfu_ops")}
     roofline["step"] = {"ms_per_step": ms_per_step,
