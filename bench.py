@@ -539,7 +539,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the streaming-step timing and the weight-mode comparison of the default line")
-    ap.add_argument("--e2e-groups", type=int, default=4,
+    ap.add_argument("--e2e-groups", type=int, default=16,
                     help="end-to-end leg: layer groups whose host copies overlap the other groups' kernels")
     ap.add_argument("--stream", action="store_true",
                     help="time the streaming step instead (budget 2048 + chunk 512, all layers of configs[1] "
