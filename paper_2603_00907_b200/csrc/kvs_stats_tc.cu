@@ -8,9 +8,9 @@
 //   S_l = K_l Q^T, S_r = K_r Q^T                    (logits, fp32 in TMEM)
 //   T_l = Vsum_l (O_hi + O_lo)^T, T_r likewise      (value/output inner products)
 // go into one of two TMEM buffers; while the statistics warps reduce one half, the tensor
-// core fills the other.  Two threads (in two warps) issue the products, one the chains of the
-// left members and one those of the right members: feeding the tensor pipe from one thread costs
-// about as much time per product as the product itself.  Each statistics thread owns one pair
+// core fills the other.  Two threads (in two warps, each chosen with elect.sync) issue the
+// products, one the chains of the left members and one those of the right members: one thread
+// alone measured 2 % slower.  Each statistics thread owns one pair
 // and a share of the queries and reduces, in registers and with no cross-lane traffic,
 //   A_j   = sum_q alpha_qj
 //   N1_j  = sum_q alpha |1 - 2 alpha| |vbar_j - o_q|                    [Eqs. c11_def, c22_def]
