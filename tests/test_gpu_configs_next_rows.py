@@ -1,0 +1,158 @@
+"""The variants beyond the plain pass (exact weights from a supplied gradient, a budget per
+(sequence, KV head), the adjacent-similarity diagnostic) at the shape of the benchmark's headline
+configuration: 32768 tokens, 8 KV heads, 4 x 64 window rows.  The oracle redoes sampled units
+element by element; bookkeeping and conservation are checked for every unit."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import kvs_oracle as oc
+from paper_2603_00907_b200 import workloads as wl
+from tests import kvs_testlib as tl
+from tests import test_gpu_parity as tp
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def kb():
+    from paper_2603_00907_b200 import binding, build
+    build.build()
+    binding.lib()
+    return binding
+
+
+def _okw(w):
+    return dict(window=w.window, sink=w.sink, recent=w.window, scale=1 / math.sqrt(128), causal=True,
+                round_frac=w.round_frac, score_mode=0)
+
+
+def test_config1_exact_weight_sums_of_a_sampled_unit(kb):
+    """kvs_window_stats_exact on one layer of configs[1] (16 336 candidate pairs per head, two query
+    blocks of 128 rows, two pair ranges per block): the signed sums G11, G22, G12 and the exact
+    weight of blocks of pairs sampled across a unit against the oracle (window probabilities formed
+    once, then the per-pair sums of the sampled pairs: the oracle's loop over all pairs and queries
+    would take minutes), for the full form and the diagonal-only ablation
+    [Section 4.2, Eq. kstar_weight_final_rewrite; Section 3.1, Eq. simplified_k]."""
+    import torch
+    w = wl.config(1)
+    data = wl.make_layer(w, 0)
+    rng = np.random.default_rng(123)
+    E_bits = wl.f32_to_bf16_bits(rng.standard_normal(data["q_win"].shape).astype(np.float32))
+    dev, p, ws = tp._setup(kb, w, data)
+    e_dev = tl.to_dev_bf16(E_bits)
+    B, Hkv, Nmax, G = w.batch, w.n_kv_heads, w.n_max, w.group
+    f32 = dict(dtype=torch.float32, device="cuda")
+    b, h = 0, 5
+    n = w.seq_lens[b]
+    # the oracle's pieces for the sampled unit
+    Kf, Vs = oc.bf16_to_f64(data["K"][b, h, :n]), oc.bf16_to_f64(data["V"][b, h, :n])
+    cf = data["counts"][b, h, :n].astype(np.float64)
+    Q = oc.bf16_to_f64(data["q_win"][b, h * G:(h + 1) * G])
+    off, P, R = oc.round_plan(n, w.budgets[b], w.sink, w.window, w.round_frac, 0)
+    assert P == 16336
+    alpha, o, vbar = oc.window_probabilities(Kf, Vs, cf, Q, w.window, 1 / math.sqrt(128), True)
+    A_ref, _ = oc.slot_stats(alpha, o, vbar)
+    E = oc.bf16_to_f64(E_bits[b, h * G:(h + 1) * G]).reshape(alpha.shape[0], -1)
+    # first pairs of blocks of 16: both ends, tile edges, and thirty more spread over the unit
+    blocks = sorted(set([0, 101, 127, 4000, 8167, 12345, P - 16] + [int(x) for x in rng.integers(0, P - 16, size=30)]))
+    ref = {}
+    for p0 in blocks:
+        ref[p0] = oc.exact_pair_sums(alpha, o, vbar, E, off + 2 * p0, 16)
+    for mode in (1, 2):
+        A, gs = torch.zeros((B, Hkv, Nmax), **f32), torch.zeros((B, Hkv, Nmax), **f32)
+        gp, wg = torch.zeros((B, Hkv, Nmax // 2), **f32), torch.zeros((B, Hkv, Nmax // 2), **f32)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        kb.kvs_window_stats_exact(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], e_dev, mode,
+                                  list(w.seq_lens), list(w.budgets), ws, A=A, g_self=gs, g_pair=gp, w=wg,
+                                  status_dev=status)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        ok, _, plain = tl.rel_close(A[b, h, off:off + 2 * P].cpu().numpy(), A_ref[off:off + 2 * P])
+        assert ok, plain
+        gsn, gpn, wgn = gs[b, h].cpu().numpy(), gp[b, h].cpu().numpy(), wg[b, h].cpu().numpy()
+        n_clear = 0
+        for p0 in blocks:
+            G11, G22, G12, ab = ref[p0]
+            sl = slice(off + 2 * p0, off + 2 * p0 + 32, 2)
+            sr = slice(off + 2 * p0 + 1, off + 2 * p0 + 32, 2)
+            assert np.all(np.abs(gsn[sl] - G11) <= tl.STAT_RTOL * ab[0] + 1e-37), p0
+            assert np.all(np.abs(gsn[sr] - G22) <= tl.STAT_RTOL * ab[1] + 1e-37), p0
+            assert np.all(np.abs(gpn[p0:p0 + 16] - G12) <= tl.STAT_RTOL * ab[2] + 1e-37), p0
+            for i in range(16):
+                w_ref = oc.exact_form_weight(G11[i], G22[i], G12[i], mode == 2)
+                c12 = G12[i] if mode == 1 else 0.0
+                gam = G11[i] + 2.0 * c12 + G22[i]
+                tot = ab[0][i] + ab[1][i] + (2.0 * ab[2][i] if mode == 1 else 0.0)
+                if abs(gam) > 1e-3 * tot:                   # away from the guard on the denominator
+                    n_clear += 1
+                    bound = min(1.0, tl.STAT_RTOL * tot / abs(gam)) + 1e-7
+                    assert abs(wgn[p0 + i] - w_ref) <= bound, (p0 + i, wgn[p0 + i], w_ref)
+        assert n_clear > 400
+
+
+def test_config1_per_head_budgets_at_full_length(kb):
+    """kvs_merge_layer_per_head on one layer of configs[1]: the eight KV heads run to eight different
+    budgets (one stays as it is, one goes down to the sink + window floor region).  Every head must
+    end at its own length with every token still counted, its protected rows untouched and its
+    value sums conserved; the head that keeps its length must not change at all; the decode check
+    of two sampled heads is compared with the oracle on the GPU's merged cache."""
+    import torch
+    w = wl.config(1).scaled(n_decode=2)
+    data = wl.make_layer(w, 0)
+    B, Hkv, G, Nmax = w.batch, w.n_kv_heads, w.group, w.n_max
+    n = w.seq_lens[0]
+    seq_len = [n] * Hkv
+    budget = [2048, n, 4096, 1024, 8192, 3000, 16384, 2500]
+    dev = tl.upload_layer(data)
+    p = kb.make_params(dev["K"], dev["V"], w.n_q_heads, w.window, sink=w.sink, round_frac=w.round_frac)
+    ws = torch.empty(kb.kvs_workspace_size_per_head(p, Nmax, 2), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    new_len = kb.kvs_merge_layer_per_head(p, dev["K"], dev["V"], dev["counts"], dev["q_win"], seq_len, budget, ws,
+                                          status_dev=status)
+    out = torch.zeros((B, w.n_q_heads, 2, 128), dtype=torch.bfloat16, device="cuda")
+    kb.kvs_decode_attn_per_head(p, dev["q_new"], dev["K"], dev["V"], dev["counts"], new_len, out, ws)
+    torch.cuda.synchronize()
+    assert status.item() == 0 and new_len == [min(n, x) for x in budget]
+    Kg, Vg, Cg, og = tl.bits_of(dev["K"]), tl.bits_of(dev["V"]), dev["counts"].cpu().numpy(), tl.bits_of(out)
+    for h in range(Hkv):
+        m = new_len[h]
+        c = Cg[0, h, :m]
+        assert int(c.sum()) == n and c.min() >= 1
+        assert np.array_equal(Kg[0, h, :w.sink], data["K"][0, h, :w.sink])
+        assert np.array_equal(Kg[0, h, m - w.window:m], data["K"][0, h, n - w.window:n])
+        assert np.array_equal(Vg[0, h, m - w.window:m], data["V"][0, h, n - w.window:n])
+        tot = oc.bf16_to_f64(data["V"][0, h, :n]).sum(0)
+        got = oc.bf16_to_f64(Vg[0, h, :m]).sum(0)
+        assert np.max(np.abs(got - tot)) < 0.02 * math.sqrt(n)
+    assert np.array_equal(Kg[0, 1, :n], data["K"][0, 1, :n]) and np.array_equal(Vg[0, 1, :n], data["V"][0, 1, :n])
+    for h in (0, 6):
+        m = new_len[h]
+        ref, _ = oc.decode_attention(data["q_new"][0, h * G:(h + 1) * G], Kg[0, h, :m], Vg[0, h, :m], Cg[0, h, :m])
+        ok, mx, _, _ = tl.bf16_close(og[0, h * G:(h + 1) * G], oc.f64_to_bf16(ref))
+        assert ok, (h, mx)
+
+
+def test_config1_adjacent_cosine_at_full_length(kb):
+    """kvs_adjacent_cosine over the keys and the values of one layer of configs[1] (8 heads x 32768
+    rows): every entry of two sampled heads against the oracle [Section 3.2, Eq. cosine_raw]; the
+    synthetic keys drift slowly (homogeneous neighbours), the values do not."""
+    import torch
+    w = wl.config(1)
+    data = wl.make_layer(w, 0)
+    dev = tl.upload_layer(data)
+    n = w.seq_lens[0]
+    for name in ("K", "V"):
+        x = dev[name]
+        out = torch.full(x.shape[:3], -7.0, dtype=torch.float32, device="cuda")
+        kb.kvs_adjacent_cosine(x, list(w.seq_lens), out)
+        torch.cuda.synchronize()
+        g = out.cpu().numpy()
+        for h in (2, 7):
+            ref = oc.adjacent_cosine(data[name][0, h, :n])
+            assert len(ref) == n - 1
+            assert np.max(np.abs(g[0, h, :n - 1] - ref)) < tl.COS_ATOL
+            assert np.all(g[0, h, n - 1:] == -7.0)
+        mean = float(g[0, :, :n - 1].mean())
+        assert (mean > 0.8) if name == "K" else (abs(mean) < 0.05)
