@@ -156,3 +156,64 @@ def test_config1_adjacent_cosine_at_full_length(kb):
             assert np.all(g[0, h, n - 1:] == -7.0)
         mean = float(g[0, :, :n - 1].mean())
         assert (mean > 0.8) if name == "K" else (abs(mean) < 0.05)
+
+
+def test_streaming_step_at_the_papers_operating_point(kb):
+    """One streaming step in the paper's setting [Section 5.1: budget 2048, chunk 512, sink 32] with
+    configs[1]'s head layout, four layers folded into the batch as the benchmark's --stream leg
+    passes them: kvs_append_and_merge must equal, bit for bit, a device copy of the chunk followed by
+    the single-round calls, and two sampled units must match the oracle's append_and_merge that
+    follows the GPU's near-cutoff choices (2560 -> 2048 is one round of 512 merges)."""
+    import torch
+    budget, chunk, L = 2048, 512, 4
+    w1 = wl.config(1).scaled(seq_lens=(budget + chunk,), budgets=(budget,))
+    per_layer = wl.make_layers_parallel(w1, range(L))
+    data = {k: np.concatenate([d[k] for d in per_layer], axis=0) for k in ("K", "V", "counts", "q_win", "q_new")}
+    w = w1.scaled(batch=L, seq_lens=(budget + chunk,) * L, budgets=(budget,) * L)
+    B, Hkv, G, W, Nmax = w.batch, w.n_kv_heads, w.group, w.window, w.n_max
+    assert Nmax >= budget + chunk
+    plan = oc.full_plan(budget + chunk, budget, w.sink, W, w.round_frac)
+    assert len(plan) == 1 and plan[0][3] == chunk
+    cK, cV = data["K"][:, :, budget:budget + chunk].copy(), data["V"][:, :, budget:budget + chunk].copy()
+    dev, p, ws = tp._setup(kb, w, data)         # through the streaming entry point
+    dev2, _, ws2 = tp._setup(kb, w, data)       # the same step from existing calls
+    dcK, dcV = tl.to_dev_bf16(cK), tl.to_dev_bf16(cV)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    # (the cache holds 2048 slots; what lies behind them is overwritten by the chunk)
+    for d in (dev, dev2):
+        d["K"][:, :, budget:] = 0
+        d["V"][:, :, budget:] = 0
+    cur, bud = [budget] * B, [budget] * B
+    new_len = kb.kvs_append_and_merge(p, dev["K"], dev["V"], dev["counts"], dcK, dcV, dev["q_win"], cur, bud, ws,
+                                      status_dev=status)
+    dev2["K"][:, :, budget:budget + chunk] = dcK
+    dev2["V"][:, :, budget:budget + chunk] = dcV
+    dev2["counts"][:, :, budget:budget + chunk] = 1
+    n_list = [budget + chunk] * B
+    mask = torch.zeros((B, Hkv, Nmax // 2), dtype=torch.uint8, device="cuda")
+    kb.kvs_window_stats(p, dev2["K"], dev2["V"], dev2["counts"], dev2["q_win"], n_list, bud, ws2, mask=mask)
+    n2 = kb.kvs_merge_layer(p, dev2["K"], dev2["V"], dev2["counts"], dev2["q_win"], n_list, bud, ws2)
+    torch.cuda.synchronize()
+    assert status.item() == 0 and new_len == n2 == bud
+    Kg, Vg, Cg = tl.bits_of(dev["K"]), tl.bits_of(dev["V"]), dev["counts"].cpu().numpy()
+    assert np.array_equal(Kg[:, :, :budget], tl.bits_of(dev2["K"])[:, :, :budget])
+    assert np.array_equal(Vg[:, :, :budget], tl.bits_of(dev2["V"])[:, :, :budget])
+    assert np.array_equal(Cg[:, :, :budget], dev2["counts"].cpu().numpy()[:, :, :budget])
+    assert np.all(Cg[:, :, :budget].sum(-1) == budget + chunk)
+    gm = mask.cpu().numpy()
+    flips = 0
+    for (b, h) in ((0, 0), (3, 6)):
+        trace = []
+        Ko, Vo, Co = oc.append_and_merge(data["K"][b, h, :budget], data["V"][b, h, :budget],
+                                         data["counts"][b, h, :budget].astype(np.int64), cK[b, h], cV[b, h],
+                                         data["q_win"][b, h * G:(h + 1) * G], budget,
+                                         forced_masks=[gm[b, h, :plan[0][2]]], trace=trace,
+                                         window=W, sink=w.sink, round_frac=w.round_frac)
+        ok, nm, nout = tl.mask_band_ok(gm[b, h, :plan[0][2]], trace[0]["mask"], trace[0]["score"], trace[0]["R"])
+        assert ok, ((b, h), nm, nout)
+        flips += nm
+        assert np.array_equal(Cg[b, h, :budget], Co)
+        okk, mxk, _, _ = tl.bf16_close(Kg[b, h, :budget], Ko)
+        okv, mxv, _, _ = tl.bf16_close(Vg[b, h, :budget], Vo)
+        assert okk and okv, ((b, h), mxk, mxv)
+    print(f"streaming step: band flips followed: {flips}")
