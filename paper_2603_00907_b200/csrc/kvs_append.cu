@@ -10,6 +10,8 @@ namespace {
 
 __global__ void __launch_bounds__(256)
 append_chunk_kernel(const AppendArgs a, const RoundTable tab) {
+  kvs_pdl_launch_dependents();
+  kvs_pdl_wait();
   const int seq = blockIdx.z;
   const SeqRound sr = tab.s[seq];
   const int h = blockIdx.y;
@@ -35,6 +37,5 @@ append_chunk_kernel(const AppendArgs a, const RoundTable tab) {
 
 cudaError_t kvs_launch_append(const AppendArgs& a, const RoundTable& t, cudaStream_t st) {
   dim3 grid((a.chunk_len + 7) / 8, a.c.Hkv, t.nseq);
-  append_chunk_kernel<<<grid, 256, 0, st>>>(a, t);
-  return cudaGetLastError();
+  return kvs_launch_chained(append_chunk_kernel, grid, dim3(256), 0, st, a, t);
 }

@@ -14,6 +14,8 @@ constexpr int kCombineRows = 8;
 
 __global__ void __launch_bounds__(kCombineRows * 32)
 combine_partials(const CombineArgs a, const RoundTable tab) {
+  kvs_pdl_launch_dependents();
+  kvs_pdl_wait();
   const int seq = blockIdx.z;
   const SeqRound sr = tab.s[seq];
   if (sr.n <= 0) return;
@@ -85,6 +87,5 @@ combine_partials(const CombineArgs a, const RoundTable tab) {
 cudaError_t kvs_launch_combine(const CombineArgs& a, const RoundTable& t, cudaStream_t st) {
   const int rows = a.qc2 ? a.M_pad : a.M;
   dim3 grid((rows + kCombineRows - 1) / kCombineRows, a.Hkv, t.nseq);
-  combine_partials<<<grid, kCombineRows * 32, 0, st>>>(a, t);
-  return cudaGetLastError();
+  return kvs_launch_chained(combine_partials, grid, dim3(kCombineRows * 32), 0, st, a, t);
 }

@@ -97,6 +97,8 @@ __global__ void __launch_bounds__(kThreads, 2)
 merge_compact_kernel(const CompactArgs a, const RoundTable tab) {
   extern __shared__ __align__(128) uint8_t smem[];
   Shared* sh = reinterpret_cast<Shared*>(smem + kStages * kStageBytes);
+  kvs_pdl_launch_dependents();
+  kvs_pdl_wait();
 
   const int seq = blockIdx.z;
   const SeqRound sr = tab.s[seq];
@@ -322,6 +324,5 @@ cudaError_t kvs_launch_compact(const CompactArgs& a, const RoundTable& t, cudaSt
     if (c > per_unit) per_unit = c;
   }
   dim3 grid(per_unit, a.c.Hkv, t.nseq);
-  merge_compact_kernel<<<grid, kThreads, kSmemBytes, st>>>(a, t);
-  return cudaGetLastError();
+  return kvs_launch_chained(merge_compact_kernel, grid, dim3(kThreads), kSmemBytes, st, a, t);
 }

@@ -176,12 +176,15 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
   const int t_begin = min(ntiles, split * a.tiles_per_split);
   const int t_end = min(ntiles, t_begin + a.tiles_per_split);
   const int my_tiles = t_end - t_begin;
-  if (n <= 0) return;
+  kvs_pdl_launch_dependents();
+  if (n <= 0) { kvs_pdl_wait(); return; }
   if (smem_u32(smem) & 1023u) {                        // the swizzled tiles need a 1024-byte aligned base
+    kvs_pdl_wait();
     if (threadIdx.x == 0 && a.status_dev) atomicExch(a.status_dev, (int)KVS_ERR_CUDA);
     return;
   }
   if (my_tiles <= 0) {
+    kvs_pdl_wait();
     // an empty key range still owes its (empty) partial to the combine
     if (warp >= 2 && warp < 6) {
       const int row = (warp & 3) * 32 + lane, m = qblk * 128 + row;
@@ -221,6 +224,8 @@ flash_partial_tc(const FlashTcArgs a, const RoundTable tab, const __grid_constan
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  // (everything above runs while the kernel before this one may still be draining)
+  kvs_pdl_wait();
   const uint32_t tmem = __shfl_sync(0xffffffffu, misc->tmem_base, 0);   // (uniform for the compiler too)
   volatile int* abort_flag = &misc->abort_flag;
   // test hook: the producer requests no K tile, so that the waits on them run out
@@ -622,6 +627,5 @@ cudaError_t kvs_launch_flash_tc(const FlashTcArgs& a, const RoundTable& t, const
   });
   if (ce != cudaSuccess) return ce;
   dim3 grid(a.nqblk * a.splits, a.Hkv, t.nseq);
-  flash_partial_tc<<<grid, kThreads, kSmemBytes, st>>>(a, t, tmK, tmV, tmQ);
-  return cudaGetLastError();
+  return kvs_launch_chained(flash_partial_tc, grid, dim3(kThreads), kSmemBytes, st, a, t, tmK, tmV, tmQ);
 }

@@ -174,6 +174,34 @@ struct KvsPerDeviceOnce {
   }
 };
 
+// Launch of a kernel of the round chain with programmatic dependent launch: the kernel may be
+// scheduled while the kernel before it in the stream is still draining (its set-up then overlaps
+// that kernel's last CTAs and the launch latency), and it calls kvs_pdl_wait() before it touches
+// global memory -- EVERY CTA does, also one that has nothing to do, so that a kernel never completes
+// before its predecessor and the chain stays ordered end to end.
+#ifdef __CUDACC__
+template <typename... KArgs, typename... Args>
+inline cudaError_t kvs_launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                      Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+// Device side: let the next kernel of the stream be scheduled (it will wait for this grid to
+// complete before it reads anything) ...
+__device__ __forceinline__ void kvs_pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+// ... and wait until the kernels before this one have completed and their writes are visible.
+__device__ __forceinline__ void kvs_pdl_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+#endif
+
 // Special-function probe: `blocks` CTAs of 1024 threads, 16 * iters operations per thread.
 cudaError_t kvs_launch_sfu_probe(int blocks, int iters, float* sink, cudaStream_t st);
 // Operand-feed probe: `blocks` CTAs, each `products` (a multiple of 8) tcgen05 products of shape

@@ -12,6 +12,8 @@ namespace {
 
 __global__ void __launch_bounds__(1024)
 select_pairs_kernel(const SelectArgs a, const RoundTable tab) {
+  kvs_pdl_launch_dependents();
+  kvs_pdl_wait();
   const int seq = blockIdx.y;
   const SeqRound sr = tab.s[seq];
   const int n = sr.n;
@@ -174,6 +176,5 @@ select_pairs_kernel(const SelectArgs a, const RoundTable tab) {
 
 cudaError_t kvs_launch_select(const SelectArgs& a, const RoundTable& t, cudaStream_t st) {
   dim3 grid(a.Hkv, t.nseq);
-  select_pairs_kernel<<<grid, 1024, 0, st>>>(a, t);
-  return cudaGetLastError();
+  return kvs_launch_chained(select_pairs_kernel, grid, dim3(1024), 0, st, a, t);
 }

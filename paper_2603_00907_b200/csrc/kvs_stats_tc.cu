@@ -115,8 +115,10 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
   const int ntiles = (P + kPairs - 1) / kPairs;
   const int t_begin = min(ntiles, split * a.tiles_per_split);
   const int t_end = min(ntiles, t_begin + a.tiles_per_split);
-  if (sr.n <= 0 || t_begin >= t_end) return;          // uniform over the CTA
+  kvs_pdl_launch_dependents();
+  if (sr.n <= 0 || t_begin >= t_end) { kvs_pdl_wait(); return; }   // uniform over the CTA
   if (smem_u32(smem) & 1023u) {                        // the swizzled tiles need a 1024-byte aligned base
+    kvs_pdl_wait();
     if (threadIdx.x == 0 && a.status_dev) atomicExch(a.status_dev, (int)KVS_ERR_CUDA);
     return;
   }
@@ -143,13 +145,15 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
     misc->wait_us = (int)a.wait_us;
     mbar_fence_init();
   }
+  if (warp == 1) tmem_alloc(&misc->tmem_base, 512);
+  // (everything above runs while the kernel before this one may still be draining)
+  kvs_pdl_wait();
   // the per-query constants of the block (the same for every tile): read from shared memory in the loop
   if (threadIdx.x < kQB) {
     const float2 c = a.qc2[(size_t)unit * a.M_pad + qblk * kQB + threadIdx.x];
     misc->qconst[(threadIdx.x >> 1) * 4 + (threadIdx.x & 1)] = c.x;
     misc->qconst[(threadIdx.x >> 1) * 4 + 2 + (threadIdx.x & 1)] = c.y;
   }
-  if (warp == 1) tmem_alloc(&misc->tmem_base, 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -403,6 +407,8 @@ hessian_stats_tc(const StatsTcArgs a, const RoundTable tab, const __grid_constan
 // A denominator that is not safely positive gives 1/2; the weight is clipped to [0, 1].
 __global__ void __launch_bounds__(256)
 stats_finalize_kernel(const StatsTcArgs a, const RoundTable tab) {
+  kvs_pdl_launch_dependents();
+  kvs_pdl_wait();
   const SeqRound sr = tab.s[blockIdx.z];
   if (sr.n <= 0) return;
   const int unit = sr.b * a.Hkv + blockIdx.y;
@@ -451,14 +457,13 @@ cudaError_t kvs_launch_stats_tc(const StatsTcArgs& a, const RoundTable& t, const
   });
   if (ce != cudaSuccess) return ce;
   dim3 grid(a.nqblk * a.splits, a.Hkv, t.nseq);
-  if (a.weight_mode == 0) hessian_stats_tc<false><<<grid, kThreads, kSmemBytes, st>>>(a, t, tmKp, tmVp, tmQ, tmOhi, tmOlo);
-  else hessian_stats_tc<true><<<grid, kThreads, kSmemBytes, st>>>(a, t, tmKp, tmVp, tmQ, tmOhi, tmOlo);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = (a.weight_mode == 0)
+      ? kvs_launch_chained(hessian_stats_tc<false>, grid, dim3(kThreads), kSmemBytes, st, a, t, tmKp, tmVp, tmQ, tmOhi, tmOlo)
+      : kvs_launch_chained(hessian_stats_tc<true>, grid, dim3(kThreads), kSmemBytes, st, a, t, tmKp, tmVp, tmQ, tmOhi, tmOlo);
   if (e != cudaSuccess) return e;
   int pmax = 0;
   for (int i = 0; i < t.nseq; ++i) pmax = pmax > t.s[i].P ? pmax : t.s[i].P;
   if (pmax <= 0) return cudaSuccess;
   dim3 fgrid((pmax + 255) / 256, a.Hkv, t.nseq);
-  stats_finalize_kernel<<<fgrid, 256, 0, st>>>(a, t);
-  return cudaGetLastError();
+  return kvs_launch_chained(stats_finalize_kernel, fgrid, dim3(256), 0, st, a, t);
 }
