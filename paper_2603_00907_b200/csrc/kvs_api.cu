@@ -178,8 +178,13 @@ struct WsLayout {
 // write-back.  The cut k that minimises  waves(items * k) * (ceil(tiles / k) + 2)  is taken (the
 // smaller k when two are within 1 %): 512 items of 256 tiles: k = 2 (7 half-length waves instead
 // of 4 full ones); 64 items of 1024 tiles: k = 9 (576 CTAs in 4 waves of 114 tiles instead of 128
-// CTAs of 512 tiles on 148 SMs); 8 items of 16 tiles: k = 16.
+// CTAs of 512 tiles on 148 SMs); 8 items of 16 tiles: k = 16.  When the CTAs need more than one
+// wave, a range is not made shorter than 16 tiles: the pipeline of a CTA (three logit buffers, two
+// K/V stages) takes a few tiles to fill, which the model's constant does not cover -- 512 items of
+// 20 tiles ran 2.4 % faster uncut (4 waves of 20 tiles) than cut in two (7 waves of 10), while a
+// larger constant instead slowed the long ragged items of the other workloads by up to 6 %.
 constexpr int kNumSMs = 148;
+constexpr int kMinRangeTiles = 16;  // (see above)
 constexpr int kMaxTcSplits = 16;    // per item (more only while items * k <= 148); the attention partials are sized for it
 
 int balanced_splits(int items, int ntiles, int* tiles_per_split) {
@@ -192,6 +197,7 @@ int balanced_splits(int items, int ntiles, int* tiles_per_split) {
   for (int k = 1; k <= kmax; ++k) {
     const int tps = (ntiles + k - 1) / k;
     const int ctas = items * ((ntiles + tps - 1) / tps);      // ranges that are not empty
+    if (k > 1 && tps < kMinRangeTiles && ctas > kNumSMs) continue;
     const double cost = (double)((ctas + kNumSMs - 1) / kNumSMs) * (tps + 2);
     if (cost < best_cost * 0.99) { best_cost = cost; best = k; }
   }
